@@ -1,0 +1,359 @@
+"""CPU oracle for the tree-verification step (TEST INFRASTRUCTURE, not product).
+
+Plain, slow, fp64 numpy restatement of what one teacher tree-verification
+step of EAGLE-3-style tree speculative decoding computes, written from the
+paper's problem statement.  It shares no code with the CUDA library and must
+only be imported by tests, the smoke check and the bench's CPU-baseline legs.
+Every function cites the passage it follows.  Nothing here is blocked, fused
+or reordered beyond the definitions; a library matmul / exp / max serves as a
+step where the definition is a sum, an exponential or a maximum.
+
+Conventions (same index algebra as Section 3.2 with N = M + 1 rows):
+  * node 0 is the root (the last sampled token, row 0 of the paper's
+    (M+1)-row tensors); ``parent[0] = -1`` is the only sentinel and is
+    remapped to 0 before any gather (dummy-root indexing);
+  * ``valid[i] = i < n_nodes``; padded slots carry device-defined fill
+    (parent 0, depth 0) and never influence active outputs;
+  * bf16 data arrive as uint16 bit patterns and are decoded here.
+
+Parity status: every function below is pinned by tests/test_oracle_pins.py
+(brute force, closed forms, library routines, special trees); none is
+"parity unpinned".
+"""
+import numpy as np
+
+# status bits reported per sequence
+ST_BAD_TREE = 1          # a structural invariant of Section 3.2 failed
+ST_BAD_INDEX = 2         # a path / node index outside [-1, n_nodes)
+ST_CAPACITY = 4          # commit would run past the cache capacity
+ST_TIMEOUT = 8           # (device only) a bounded wait expired
+ST_PATHS_TRUNCATED = 16  # more leaves than path rows; non-fatal
+ST_FATAL = ST_BAD_TREE | ST_BAD_INDEX | ST_CAPACITY | ST_TIMEOUT
+
+
+def decode_bf16(bits):
+    """bf16 bit patterns -> float64, exactly (bf16 is the upper half of an fp32)."""
+    b = np.asarray(bits, dtype=np.uint16)
+    return (b.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+# ---------------------------------------------------------------------------
+# Section 3.2: tensorisation (dummy-root remap, depth, ancestor table, invariants)
+# ---------------------------------------------------------------------------
+def tensorize_one(parent, n, Dcap):
+    """One sequence.  Returns (ok, safe_parent, depth, A) with A of shape
+    [Dcap+1, Nmax]; on an invariant failure ok is False and the arrays are zero.
+
+    Dummy-root indexing: safe_parent[i] = 0 where parent[i] is the sentinel
+    (Section 3.2, "Dummy-root indexing").  Ancestor table: A[0,i] = i,
+    A[l+1,i] = safe_parent[A[l,i]] (Section 3.2, "Ancestor tables").
+    Invariants (Section 3.2, "Structural invariants"): range, depth
+    consistency / acyclicity (parent chain reaches 0 within depth steps),
+    validity closure; plus our topological-order reading parent[i] < i and
+    the caller's depth bound.
+    """
+    Nmax = len(parent)
+    sp = np.zeros(Nmax, dtype=np.int32)
+    depth = np.zeros(Nmax, dtype=np.int32)
+    A = np.zeros((Dcap + 1, Nmax), dtype=np.int32)
+    zero = (False, np.zeros_like(sp), np.zeros_like(depth), np.zeros_like(A))
+    if n < 1 or n > Nmax:
+        return zero
+    if parent[0] != -1:
+        return zero
+    for i in range(1, n):
+        p = int(parent[i])
+        if p < 0 or p >= n:          # range
+            return zero
+        if p >= i:                   # topological order (our reading)
+            return zero
+        sp[i] = p
+    # padded slots: device-defined fill, parent 0 / depth 0, whatever the input holds
+    for i in range(1, n):
+        # depth by a capped parent walk: steps until row 0 is reached
+        cur, steps = i, 0
+        while cur != 0 and steps <= n:
+            cur = int(sp[cur])
+            steps += 1
+        if cur != 0:                 # acyclicity
+            return zero
+        depth[i] = steps
+    for i in range(1, n):
+        if not depth[sp[i]] < depth[i]:   # depth consistency
+            return zero
+        if depth[i] > Dcap:
+            return zero
+        if not sp[i] < n:                 # validity closure (valid => parent valid)
+            return zero
+    for i in range(Nmax):
+        A[0, i] = i
+    for l in range(Dcap):
+        for i in range(Nmax):
+            A[l + 1, i] = sp[A[l, i]]
+    for i in range(1, n):
+        if A[depth[i], i] != 0:
+            return zero
+    return True, sp, depth, A
+
+
+def build_mask(parent, n_nodes, Dcap, Pcap):
+    """Tree tensorisation + mask for a batch (Sections 2.4, 3.2, 3.3).
+
+    vis[b,i,j] = valid[i] and valid[j] and (exists l in [0,Dcap]: A[l,i] == j)
+    is the ancestor-or-self predicate of Section 3.3 combined with the
+    no-leak padding rule.  Returns a dict:
+      anc_bits[B,Nmax,W] u32 (bit j%32 of word j//32 of row i), dense[B,1,Nmax,Nmax] u8,
+      depth[B,Nmax], anc_table[B,Dcap+1,Nmax], retrieve[B,Pcap,Dcap+1] (-1 padded),
+      n_paths[B], status[B].
+    Candidate-path rows: one per leaf, leaves in increasing node id, root
+    first, -1 after the leaf.
+    """
+    parent = np.asarray(parent)
+    B, Nmax = parent.shape
+    W = (Nmax + 31) // 32
+    out = {
+        "anc_bits": np.zeros((B, Nmax, W), dtype=np.uint32),
+        "dense": np.zeros((B, 1, Nmax, Nmax), dtype=np.uint8),
+        "depth": np.zeros((B, Nmax), dtype=np.int32),
+        "anc_table": np.zeros((B, Dcap + 1, Nmax), dtype=np.int32),
+        "retrieve": np.full((B, Pcap, Dcap + 1), -1, dtype=np.int32),
+        "n_paths": np.zeros(B, dtype=np.int32),
+        "status": np.zeros(B, dtype=np.int32),
+    }
+    for b in range(B):
+        n = int(n_nodes[b])
+        ok, sp, depth, A = tensorize_one(parent[b], n, Dcap)
+        if not ok:
+            out["status"][b] = ST_BAD_TREE
+            continue
+        out["depth"][b] = depth
+        out["anc_table"][b] = A
+        for i in range(n):
+            for j in range(n):
+                seen = False
+                for l in range(Dcap + 1):
+                    if A[l, i] == j:
+                        seen = True
+                if seen:
+                    out["dense"][b, 0, i, j] = 1
+                    out["anc_bits"][b, i, j // 32] |= np.uint32(1) << np.uint32(j % 32)
+        # root-to-leaf rows
+        has_child = np.zeros(n, dtype=bool)
+        for i in range(1, n):
+            has_child[sp[i]] = True
+        row = 0
+        for leaf in range(n):
+            if has_child[leaf]:
+                continue
+            if row >= Pcap:
+                out["status"][b] |= ST_PATHS_TRUNCATED
+                break
+            dl = int(depth[leaf])
+            for l in range(dl + 1):
+                out["retrieve"][b, row, dl - l] = A[l, leaf]
+            row += 1
+        out["n_paths"][b] = row
+    return out
+
+
+# ---------------------------------------------------------------------------
+# Sections 2.3, 3.3: tree attention (the attention sub-step of TeacherTreeEval)
+# ---------------------------------------------------------------------------
+def tree_attention(q_bits, k_cache_bits, v_cache_bits, k_tree_bits, v_tree_bits,
+                   prefix_len, n_nodes, vis, scale):
+    """Every valid node i, query head h (KV head h // G) attends the committed
+    prefix rows [0, S_b) and the tree keys j with vis[b,i,j] (context
+    correctness, Section 3.3): softmax with max subtraction over
+    scale * <q, k>, times V.  Shapes: q[B,Nmax,Hq,d], caches[B,Hkv,Scap,d],
+    tree K/V[B,Nmax,Hkv,d], vis[B,Nmax,Nmax] (0/1).
+    Returns out[B,Nmax,Hq,d] f64 and lse[B,Hq,Nmax] f64; rows without any
+    visible key (padded rows) give zeros and -inf.
+    """
+    q = decode_bf16(q_bits)
+    B, Nmax, Hq, d = q.shape
+    Hkv = k_cache_bits.shape[1]
+    G = Hq // Hkv
+    out = np.zeros((B, Nmax, Hq, d), dtype=np.float64)
+    lse = np.full((B, Hq, Nmax), -np.inf, dtype=np.float64)
+    for b in range(B):
+        S = int(prefix_len[b])
+        n = int(n_nodes[b])
+        for h in range(Hq):
+            hk = h // G
+            keys = np.concatenate([decode_bf16(k_cache_bits[b, hk, :S]),
+                                   decode_bf16(k_tree_bits[b, :, hk])], axis=0)
+            vals = np.concatenate([decode_bf16(v_cache_bits[b, hk, :S]),
+                                   decode_bf16(v_tree_bits[b, :, hk])], axis=0)
+            x = scale * (q[b, :, h, :] @ keys.T)                    # [Nmax, S+Nmax]
+            see = np.zeros((Nmax, S + Nmax), dtype=bool)
+            see[:n, :S] = True
+            see[:, S:] = np.asarray(vis[b], dtype=bool)
+            see[n:, :] = False
+            for i in range(Nmax):
+                cols = np.flatnonzero(see[i])
+                if cols.size == 0:
+                    continue
+                xi = x[i, cols]
+                m = xi.max()
+                p = np.exp(xi - m)
+                l = p.sum()
+                out[b, i, h, :] = (p / l) @ vals[cols]
+                lse[b, h, i] = m + np.log(l)
+    return out, lse
+
+
+# ---------------------------------------------------------------------------
+# Sections 2.5, 3.2: accelerator-safe path gather
+# ---------------------------------------------------------------------------
+def safe_gather(retrieve, tokens, n_nodes):
+    """Sentinel -> dummy index 0 *before* the gather, guarded by a validity
+    flag (Section 2.5; Section 3.2 "Dummy-root indexing", "Padding and batch
+    semantics").  retrieve[B,P,Dp1], tokens[B,Nmax].
+    Returns safe_idx, cand (tokens[safe_idx]), ok, status[B].
+    """
+    retrieve = np.asarray(retrieve)
+    B, P, Dp1 = retrieve.shape
+    safe = np.zeros_like(retrieve)
+    cand = np.zeros_like(retrieve)
+    ok = np.zeros(retrieve.shape, dtype=bool)
+    status = np.zeros(B, dtype=np.int32)
+    for b in range(B):
+        n = int(n_nodes[b])
+        for p in range(P):
+            for j in range(Dp1):
+                r = int(retrieve[b, p, j])
+                good = 0 <= r < n
+                if r < -1 or r >= n:
+                    status[b] |= ST_BAD_INDEX
+                s = r if good else 0
+                assert 0 <= s < tokens.shape[1]      # every dereferenced index is in range
+                safe[b, p, j] = s
+                ok[b, p, j] = good
+                cand[b, p, j] = tokens[b, s]
+    return safe, cand, ok, status
+
+
+# ---------------------------------------------------------------------------
+# Section 2.1: greedy teacher choice; Section 2.3: acceptance along one path
+# ---------------------------------------------------------------------------
+def argmax_rows(logits_bits, n_nodes):
+    """am[b,i] = the lowest v with logits[b,i,v] equal to the row maximum
+    (greedy selection of Section 2.1, temperature 0 as in Section 5); -1 for
+    padded rows.  Comparison is on the decoded float values, so -0.0 == +0.0."""
+    B, Nmax, V = logits_bits.shape
+    am = np.full((B, Nmax), -1, dtype=np.int32)
+    for b in range(B):
+        for i in range(int(n_nodes[b])):
+            row = decode_bf16(logits_bits[b, i])
+            top = row.max()
+            am[b, i] = np.flatnonzero(row == top)[0]
+    return am
+
+
+def greedy_accept(retrieve, tokens, n_nodes, am):
+    """Longest accepted prefix over all candidate rows (Section 2.3: accepted
+    nodes form a single root-to-leaf path prefix; greedy rule, Section 5).
+
+    A draft node on a row is accepted when its token equals the teacher's
+    argmax at the previous node of the row and all earlier nodes of the row
+    were accepted; remapped (-1) slots never match because of the validity
+    guard.  Ties between rows go to the lowest row.
+    Returns accept_len[B], best_path[B], accepted_nodes[B,Dp1] (first A+1
+    entries, rest 0), next_token[B] (teacher argmax at the last accepted
+    node), safe_idx, cand, status.
+    """
+    safe, cand, ok, status = safe_gather(retrieve, tokens, n_nodes)
+    B, P, Dp1 = safe.shape
+    accept_len = np.zeros(B, dtype=np.int32)
+    best_path = np.zeros(B, dtype=np.int32)
+    accepted = np.zeros((B, Dp1), dtype=np.int32)
+    next_token = np.zeros(B, dtype=np.int32)
+    for b in range(B):
+        best_a, best_p = 0, 0
+        for p in range(P):
+            a = 0
+            for j in range(1, Dp1):
+                if ok[b, p, j] and ok[b, p, j - 1] and cand[b, p, j] == am[b, safe[b, p, j - 1]]:
+                    a = j
+                else:
+                    break
+            if a > best_a:
+                best_a, best_p = a, p
+        accept_len[b] = best_a
+        best_path[b] = best_p
+        if P > 0:
+            for j in range(best_a + 1):
+                accepted[b, j] = safe[b, best_p, j]
+        next_token[b] = am[b, accepted[b, best_a]]
+    return {"accept_len": accept_len, "best_path": best_path, "accepted_nodes": accepted,
+            "next_token": next_token, "safe_idx": safe, "candidates": cand, "ok": ok,
+            "status": status}
+
+
+# ---------------------------------------------------------------------------
+# Section 3.1: path-index commit, prefix-sharing fast reorder
+# ---------------------------------------------------------------------------
+def kv_commit(k_cache, v_cache, k_tree, v_tree, accepted_nodes, accept_len, prefix_len,
+              status_in=None):
+    """The committed prefix keeps its order and only the accepted segment is
+    gathered behind it (Section 3.1, "Prefix-sharing fast reorder"):
+    cache[l,b,h,S_b+j,:] = tree[l,b,accepted_nodes[b,j],h,:] for j = 0..A_b,
+    then prefix_len[b] += A_b + 1.  Works on copies; all other bytes are
+    unchanged.  A sequence whose incoming status is fatal, whose segment
+    would pass the capacity or whose node list leaves [0,Nmax) is skipped and
+    flagged.  Arrays are raw uint16 (any dtype works: this is a byte copy).
+    """
+    kc, vc = k_cache.copy(), v_cache.copy()
+    L, B, Hkv, Scap, d = kc.shape
+    Nmax = k_tree.shape[2]
+    Dp1 = accepted_nodes.shape[1]
+    new_len = np.array(prefix_len, dtype=np.int32).copy()
+    status = np.zeros(B, dtype=np.int32) if status_in is None else np.array(status_in, dtype=np.int32).copy()
+    for b in range(B):
+        if status[b] & ST_FATAL:
+            continue
+        S, A = int(prefix_len[b]), int(accept_len[b])
+        if A < 0 or A >= Dp1 or any(not (0 <= int(accepted_nodes[b, j]) < Nmax) for j in range(A + 1)):
+            status[b] |= ST_BAD_INDEX
+            continue
+        if S < 0 or S + A + 1 > Scap:
+            status[b] |= ST_CAPACITY
+            continue
+        for l in range(L):
+            for h in range(Hkv):
+                for j in range(A + 1):
+                    node = int(accepted_nodes[b, j])
+                    kc[l, b, h, S + j, :] = k_tree[l, b, node, h, :]
+                    vc[l, b, h, S + j, :] = v_tree[l, b, node, h, :]
+        new_len[b] = S + A + 1
+    return kc, vc, new_len, status
+
+
+def verify_step(case_np, scale, Dcap=None, Pcap=None, use_given_retrieve=True):
+    """One whole step in the paper's order: tensorise + mask, attention per
+    layer, safe gather + argmax + accept, commit (Section 3 call order)."""
+    parent, n_nodes = case_np["parent"], case_np["n_nodes"]
+    Dp1 = case_np["retrieve"].shape[2]
+    mk = build_mask(parent, n_nodes, Dp1 - 1 if Dcap is None else Dcap,
+                    case_np["retrieve"].shape[1] if Pcap is None else Pcap)
+    L = case_np["q"].shape[0]
+    outs, lses = [], []
+    for l in range(L):
+        o, s = tree_attention(case_np["q"][l], case_np["k_cache"][l], case_np["v_cache"][l],
+                              case_np["k_tree"][l], case_np["v_tree"][l],
+                              case_np["prefix_len"], n_nodes, mk["dense"][:, 0], scale)
+        outs.append(o)
+        lses.append(s)
+    res = {"mask": mk, "out": np.stack(outs), "lse": np.stack(lses)}
+    if "logits" in case_np:
+        am = argmax_rows(case_np["logits"], n_nodes)
+        retrieve = case_np["retrieve"] if use_given_retrieve else mk["retrieve"]
+        acc = greedy_accept(retrieve, case_np["tokens"], n_nodes, am)
+        status = mk["status"] | acc["status"]
+        kc, vc, new_len, status = kv_commit(case_np["k_cache"], case_np["v_cache"],
+                                            case_np["k_tree"], case_np["v_tree"],
+                                            acc["accepted_nodes"], acc["accept_len"],
+                                            case_np["prefix_len"], status)
+        res.update({"argmax": am, "accept": acc, "k_cache": kc, "v_cache": vc,
+                    "prefix_len": new_len, "status": status})
+    return res
