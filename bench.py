@@ -1,0 +1,354 @@
+#!/usr/bin/env python
+"""Benchmark of the tree-verification step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+One step = one pass of the whole hot path over one batch of synthetic input:
+tree_build_mask, tree_verify_attn for every layer, tree_accept, kv_commit.
+Prints one JSON line (rank 0).  With --gpus N (launched under torchrun) every
+rank runs its own batch of the same shape (sequence sharding, no data-path
+collective) and the value is the aggregate over ranks, timed as the max over
+ranks.  --impl reference times the fp64 CPU oracle on a bounded sample.
+"""
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from workloads import CONFIGS, get_config, make_case, bf16_bits  # noqa: E402
+
+METRIC = "tree_verify_steps_per_sec"
+UNIT = "steps/s"
+# DRAM bytes per tree_verify_attn launch measured by ncu (dram__bytes_read.sum + dram__bytes_write.sum),
+# per workload; None until a capture exists (see profiles/).
+NCU_TRAFFIC_BYTES = {}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return float(p["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
+
+    def __init__(self, index, period_s=0.004):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            try:
+                uuid = "GPU-" + str(torch.cuda.get_device_properties(index).uuid)
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid)
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.period = period_s
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+        }
+        get_reasons = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or getattr(
+            nv, "nvmlDeviceGetCurrentClocksThrottleReasons")
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = get_reasons(self.h)
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        if self._thread is not None:
+            self._stop.set()
+            self._thread.join()
+        return {"sm_mhz": float(np.median(self.samples)) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def attn_algorithmic_bytes(cfg, prefix_len):
+    """K and V once over prefix + tree keys, Q in and O out, per layer (bf16)."""
+    keys = int(np.sum(prefix_len.astype(np.int64) + cfg.N))
+    return 2 * 2 * cfg.Hkv * cfg.d * keys + 2 * 2 * cfg.B * cfg.N * cfg.Hq * cfg.d
+
+
+def attn_flops(cfg, prefix_len):
+    keys = int(np.sum(prefix_len.astype(np.int64) + cfg.N))
+    return 4 * cfg.Hq * cfg.N * cfg.d * keys
+
+
+# --------------------------------------------------------------------------- oracle legs
+def oracle_sample_seconds(cfg, seed):
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload and
+    scales each stage to a full step.  Returns (estimated seconds per full step, description, threads)."""
+    from oracle import tree_verify_oracle as orc
+    small = cfg.scaled(L=1, B=min(cfg.B, 4), V=min(cfg.V, 65536) if cfg.V else 0)
+    case = make_case(small, seed, device="cpu")
+    from workloads import case_to_numpy
+    cn = case_to_numpy(case)
+    Dp1 = cn["retrieve"].shape[2]
+    t0 = time.perf_counter()
+    mk = orc.build_mask(cn["parent"], cn["n_nodes"], Dp1 - 1, cn["retrieve"].shape[1])
+    t_mask = time.perf_counter() - t0
+    # attention: one layer, the sampled sequences, all KV heads
+    hk_n = small.Hkv
+    G = small.Hq // small.Hkv
+    t0 = time.perf_counter()
+    orc.tree_attention(cn["q"][0][:, :, :hk_n * G], cn["k_cache"][0][:, :hk_n], cn["v_cache"][0][:, :hk_n],
+                       cn["k_tree"][0][:, :, :hk_n], cn["v_tree"][0][:, :, :hk_n], cn["prefix_len"],
+                       cn["n_nodes"], mk["dense"][:, 0], small.d ** -0.5)
+    t_attn = time.perf_counter() - t0
+    keys_sample = float(np.sum(cn["prefix_len"].astype(np.int64) + small.N)) * hk_n
+    # full-step key count uses the expected prefix length of the config
+    keys_full = cfg.B * ((cfg.S_lo + cfg.S_hi) / 2 + cfg.N) * cfg.Hkv * cfg.L
+    est = t_mask * cfg.B / small.B + t_attn * keys_full / keys_sample
+    desc = (f"oracle on {small.B} of {cfg.B} sequences: mask; attention of 1 layer x {hk_n} KV heads "
+            f"(scaled by keys x heads x layers)")
+    if cfg.V:
+        t0 = time.perf_counter()
+        am = orc.argmax_rows(cn["logits"], cn["n_nodes"])
+        t_arg = time.perf_counter() - t0
+        t0 = time.perf_counter()
+        acc = orc.greedy_accept(cn["retrieve"], cn["tokens"], cn["n_nodes"], am)
+        t_acc = time.perf_counter() - t0
+        t0 = time.perf_counter()
+        orc.kv_commit(cn["k_cache"], cn["v_cache"], cn["k_tree"], cn["v_tree"], acc["accepted_nodes"],
+                      acc["accept_len"], cn["prefix_len"])
+        t_com = time.perf_counter() - t0
+        est += t_arg * (cfg.B * cfg.V) / (small.B * small.V) + t_acc * cfg.B / small.B + t_com * cfg.B * cfg.L / small.B
+        desc += f"; argmax over {small.V} of {cfg.V} logits per row; accept; commit of 1 layer"
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    return est, desc, threads
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    for _ in range(args.warmup):
+        pass      # the oracle has no warm-up state; a warm-up step would only repeat the sample
+    ests = []
+    t_all = time.perf_counter()
+    for s in range(args.steps):
+        est, desc, threads = oracle_sample_seconds(cfg, args.seed + s)
+        ests.append(est)
+        if time.perf_counter() - t_all > 120:
+            break
+    sec = float(np.mean(ests))
+    value = 1.0 / sec
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": len(ests), "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "B": cfg.B, "L": cfg.L, "N": cfg.N, "Hq": cfg.Hq, "Hkv": cfg.Hkv,
+                   "d": cfg.d, "V": cfg.V, "prefix": [cfg.S_lo, cfg.S_hi]},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------- CUDA arm
+def run_ours(args, cfg):
+    import paper_2603_08088_b200 as tv
+    from paper_2603_08088_b200 import dist as tvd
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the treeverify library has no CPU path")
+    rank, world, local = tvd.init_from_env("nccl")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    tv.load()
+    scale = cfg.d ** -0.5
+    case = make_case(cfg, args.seed + rank, device=dev)
+    P, Dp1 = case["retrieve"].shape[1], cfg.D + 1
+    given_rows = cfg.P > 0
+    buf = tv.StepBuffers(cfg.L, cfg.B, cfg.N, cfg.Hq, cfg.Hkv, cfg.d, cfg.Scap, cfg.V, P, Dp1, device=dev)
+    prefix0 = case["prefix_len"].clone()
+    S_host = prefix0.cpu().numpy()
+    has_accept = cfg.V > 0
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def one_step(marks=None):
+        # the commit advances prefix_len; every step starts from the same committed state
+        case["prefix_len"].copy_(prefix0)
+        if marks is not None:
+            marks[0].record()
+        tv.tree_build_mask(case["parent"], case["n_nodes"], Dp1 - 1, buf.retrieve.shape[1], buf.anc_bits,
+                           buf.status, retrieve_indices=None if given_rows else buf.retrieve, n_paths=buf.n_paths)
+        if marks is not None:
+            marks[1].record()
+        for l in range(cfg.L):
+            tv.tree_verify_attn(case["q"][l], case["k_cache"][l], case["v_cache"][l], case["k_tree"][l],
+                                case["v_tree"][l], case["prefix_len"], case["n_nodes"], buf.anc_bits, scale,
+                                buf.out[l], buf.attn_ws, buf.status)
+        if marks is not None:
+            marks[2].record()
+        if has_accept:
+            rows = case["retrieve"] if given_rows else buf.retrieve
+            tv.tree_accept(case["logits"], case["tokens"], rows, case["n_nodes"], buf.argmax_tok, buf.accept_len,
+                           buf.best_path, buf.accepted_nodes, buf.next_token, buf.accept_ws, buf.status)
+            tv.kv_commit(case["k_cache"], case["v_cache"], case["k_tree"], case["v_tree"], buf.accepted_nodes,
+                         buf.accept_len, case["prefix_len"], buf.status)
+        if marks is not None:
+            marks[3].record()
+
+    for _ in range(max(args.warmup, 3)):
+        one_step()
+    torch.cuda.synchronize()
+    status = buf.status.cpu().numpy()
+    if (status & 15).any():
+        raise SystemExit(f"bench.py: fatal per-sequence status after warm-up: {status}")
+
+    sampler = ClockSampler(local)
+    marks = [[ev() for _ in range(4)] for _ in range(args.steps)]
+    tvd.barrier()
+    torch.cuda.synchronize()
+    launches0 = tv.tv_launch_count()
+    sampler.start()
+    t_start, t_end = ev(), ev()
+    t_start.record()
+    for s in range(args.steps):
+        one_step(marks[s])
+    t_end.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    launches = tv.tv_launch_count() - launches0
+    tvd.barrier()
+    elapsed_ms = tvd.max_over_ranks(t_start.elapsed_time(t_end), dev)
+    total_steps = tvd.sum_over_ranks(args.steps, dev)
+    attn_ms = sum(m[1].elapsed_time(m[2]) for m in marks) / (args.steps * cfg.L)
+    tail_us = sum(m[2].elapsed_time(m[3]) for m in marks) / args.steps * 1e3
+    mask_us = sum(m[0].elapsed_time(m[1]) for m in marks) / args.steps * 1e3
+    mean_accept = float(buf.accept_len.float().mean().item()) if has_accept else None
+
+    # ---- end-to-end through the host-buffer entry point (rank-local, timed with the host clock around
+    # the call, which returns after the stream has drained)
+    e2e = None
+    if has_accept:
+        torch.cuda.synchronize()
+        pin = lambda t: t.cpu().contiguous().pin_memory()
+        host = {k: pin(case[k]) for k in ("parent", "n_nodes", "tokens", "q", "k_tree", "v_tree", "logits")}
+        host["retrieve_indices"] = pin(case["retrieve"]) if given_rows else None
+        host["P"] = P
+        host["out"] = torch.empty(cfg.L, cfg.B, cfg.N, cfg.Hq, cfg.d, dtype=torch.bfloat16).pin_memory()
+        for k, shape in (("accept_len", (cfg.B,)), ("accepted_nodes", (cfg.B, Dp1)), ("next_token", (cfg.B,)),
+                         ("status", (cfg.B,))):
+            host[k] = torch.zeros(shape, dtype=torch.int32).pin_memory()
+        staging = torch.empty(tv.tv_step_staging_bytes(cfg.L, cfg.B, cfg.N, cfg.Hq, cfg.Hkv, cfg.d, cfg.Scap,
+                                                       cfg.V, P, Dp1), dtype=torch.uint8, device=dev)
+        h2d = sum(host[k].numel() * host[k].element_size() for k in
+                  ("parent", "n_nodes", "tokens", "q", "k_tree", "v_tree", "logits"))
+        if given_rows:
+            h2d += host["retrieve_indices"].numel() * 4
+        d2h = sum(host[k].numel() * host[k].element_size() for k in
+                  ("out", "accept_len", "accepted_nodes", "next_token", "status"))
+        e2e_steps = max(3, min(args.steps, 10))
+        for _ in range(2):
+            case["prefix_len"].copy_(prefix0)
+            tv.tv_verify_step_host(host, case["k_cache"], case["v_cache"], case["prefix_len"], staging, scale, cfg.V)
+        tvd.barrier()
+        e0, e1 = ev(), ev()
+        e0.record()
+        for _ in range(e2e_steps):
+            case["prefix_len"].copy_(prefix0)
+            tv.tv_verify_step_host(host, case["k_cache"], case["v_cache"], case["prefix_len"], staging, scale, cfg.V)
+        e1.record()
+        torch.cuda.synchronize()
+        e2e_ms = tvd.max_over_ranks(e0.elapsed_time(e1), dev)
+        e2e = {"value": tvd.sum_over_ranks(e2e_steps, dev) / (e2e_ms * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e2e_steps,
+               "ms_per_step": e2e_ms / e2e_steps}
+        if (host["status"].numpy() & 15).any():
+            raise SystemExit(f"bench.py: fatal status from the host-buffer step: {host['status'].numpy()}")
+
+    if rank != 0:
+        return
+    peak, peak_kind = measured_peaks()
+    alg_bytes = attn_algorithmic_bytes(cfg, S_host)
+    achieved = alg_bytes / (attn_ms * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": total_steps / (elapsed_ms * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": elapsed_ms / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": cfg.name, "B": cfg.B, "L": cfg.L, "N": cfg.N, "D": cfg.D, "Hq": cfg.Hq,
+                   "Hkv": cfg.Hkv, "d": cfg.d, "V": cfg.V, "prefix": [cfg.S_lo, cfg.S_hi],
+                   "sum_prefix": int(S_host.sum()), "parallelism": f"sequence-sharded x{world}",
+                   "l2": "inputs larger than L2 (each step streams the whole KV cache and the logits)"},
+        "sequence_steps_per_sec": total_steps * cfg.B / (elapsed_ms * 1e-3),
+        "stage_us": {"mask": mask_us, "attn_per_layer": attn_ms * 1e3, "accept_commit": tail_us},
+        "mean_accept_len": mean_accept,
+        "roofline": {"bound": "hbm", "kernel": "tree_verify_attn", "achieved": achieved, "peak": peak,
+                     "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                     "traffic": NCU_TRAFFIC_BYTES.get(cfg.name), "algorithmic_bytes_per_launch": alg_bytes,
+                     "avg_launch_us": attn_ms * 1e3,
+                     "tensor_tflops": attn_flops(cfg, S_host) / (attn_ms * 1e-3) / 1e12},
+        "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e,
+    }
+    if args.cpu_baseline:
+        sec, desc, threads = oracle_sample_seconds(cfg, args.seed)
+        line["cpu_baseline"] = {"value": 1.0 / sec, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                "sample": desc, "est_seconds_per_step": sec}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="full_step_32l", choices=[c.name for c in CONFIGS])
+    ap.add_argument("--seed", type=int, default=4000)
+    ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    args = ap.parse_args()
+    cfg = get_config(args.workload)
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        if int(os.environ.get("WORLD_SIZE", "1")) > 1:
+            args.cpu_baseline = False      # the CPU baseline is reported at N=1 only
+        run_ours(args, cfg)
+    try:
+        import torch.distributed as dist
+        if dist.is_initialized():
+            dist.destroy_process_group()
+    except Exception:
+        pass
+
+
+if __name__ == "__main__":
+    main()

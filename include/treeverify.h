@@ -1,0 +1,246 @@
+/*
+ * treeverify - the teacher tree-verification step of EAGLE-3-style tree
+ * speculative decoding, as a C-ABI library of sm_100a CUDA kernels.
+ *
+ * One step = tree_build_mask, then tree_verify_attn once per layer, then
+ * tree_accept, then kv_commit, all enqueued on one stream.  No call
+ * synchronises, allocates or keeps state (except tv_verify_step_host, which
+ * waits for its own copies); every launch is asynchronous on the stream given.
+ *
+ * Conventions
+ *   - Pointers are DEVICE pointers owned by the caller unless a parameter is
+ *     marked "host".  Arrays are dense, row-major, last index fastest.
+ *   - tv_bf16 is the raw 16-bit pattern of a bfloat16.
+ *   - Node 0 of every tree is the root (the last sampled token): it is a
+ *     real query row with its own K/V and logits, parent[0] = -1 is the only
+ *     sentinel, and 0 is the dummy index every sentinel is remapped to
+ *     before a gather (Section 3.2, "Dummy-root indexing", with N = M + 1).
+ *   - n_nodes[b] <= Nmax nodes of sequence b are active; slots past it are
+ *     padding and can never influence an active output (Section 3.2,
+ *     "Padding and batch semantics"; Section 3.3, "No leakage to padded slots").
+ *   - Return value: TV_OK or a TV_ERR_* code for errors the host can see
+ *     (nothing is launched then); tv_last_error() gives a message.
+ *   - Data-dependent errors are reported per sequence in status[B] (device,
+ *     bit field TV_ST_*).  tree_build_mask overwrites status[b]; the other
+ *     calls OR into it.  A sequence with a fatal bit gets no commit.
+ */
+#ifndef TREEVERIFY_H_
+#define TREEVERIFY_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define TV_API __attribute__((visibility("default")))
+#else
+#define TV_API
+#endif
+
+typedef uint16_t tv_bf16;
+typedef void* tv_stream;      /* a cudaStream_t; NULL is the legacy default stream */
+
+enum {
+  TV_OK = 0,
+  TV_ERR_INVALID_ARG = 1,     /* NULL pointer, bad dimension, unsupported shape, misalignment */
+  TV_ERR_CUDA = 2,            /* a launch, copy or tensor-map encode failed */
+  TV_ERR_WORKSPACE = 3        /* workspace smaller than tv_*_workspace_bytes says */
+};
+
+enum {
+  TV_ST_BAD_TREE = 1,         /* a structural invariant of the tree failed (fatal) */
+  TV_ST_BAD_INDEX = 2,        /* a path / node index outside its range (fatal) */
+  TV_ST_CAPACITY = 4,         /* the accepted segment does not fit the cache (fatal) */
+  TV_ST_TIMEOUT = 8,          /* a bounded wait inside a kernel expired (fatal) */
+  TV_ST_PATHS_TRUNCATED = 16  /* more leaves than path rows; the first Pcap were kept */
+};
+
+/* Message of the last TV_ERR_* returned on this host thread ("" if none). */
+TV_API const char* tv_last_error(void);
+
+/* Library version, major*100 + minor. */
+TV_API int tv_version(void);
+
+/* Number of kernels this library has launched in this process so far
+ * (diagnostics: lets a caller verify that its work ran in these kernels). */
+TV_API unsigned long long tv_launch_count(void);
+
+/*
+ * Tree tensorisation and tree mask (Section 3.2: dummy-root remap, depth,
+ * ancestor table A[0,k]=k, A[l+1,k]=parent~(A[l,k]), structural invariants;
+ * Section 2.4 / 3.3: node k sees node j iff j is an ancestor of k or k itself
+ * and both are valid).
+ *
+ *   parent[B,Nmax]  in  parent[b,0] must be -1; 0 <= parent[b,i] < i for
+ *                       1 <= i < n_nodes[b] (topological order); slots past
+ *                       n_nodes[b] are ignored.
+ *   n_nodes[B]      in  1..Nmax
+ *   Dcap                largest depth (edges from the root) a node may have
+ *   Pcap                rows of retrieve_indices
+ *   anc_bits[B,Nmax,W]  out, W = ceil(Nmax/32): bit (j%32) of word j/32 of
+ *                       row i is set iff i sees j.  Required.
+ *   dense_mask[B,1,Nmax,Nmax] out or NULL: 1 = visible, 0 = masked (the
+ *                       additive mask of Section 2.4 is visible ? 0 : -inf).
+ *   depth[B,Nmax]       out or NULL
+ *   anc_table[B,Dcap+1,Nmax] out or NULL; every entry is in [0,Nmax).
+ *   retrieve_indices[B,Pcap,Dcap+1] out or NULL: one row per leaf, leaves in
+ *                       increasing node id, root first, -1 after the leaf and
+ *                       in unused rows.
+ *   n_paths[B]          out or NULL (required with retrieve_indices)
+ *   status[B]           out: 0, TV_ST_BAD_TREE (all outputs of the sequence
+ *                       zero, its retrieve rows -1) or TV_ST_PATHS_TRUNCATED.
+ * Limits: 1 <= Nmax <= 1024, 0 <= Dcap < Nmax.
+ */
+TV_API int tree_build_mask(const int32_t* parent, const int32_t* n_nodes,
+                    int B, int Nmax, int Dcap, int Pcap,
+                    uint32_t* anc_bits, uint8_t* dense_mask, int32_t* depth,
+                    int32_t* anc_table, int32_t* retrieve_indices, int32_t* n_paths,
+                    int32_t* status, tv_stream stream);
+
+/* Scratch needed by tree_verify_attn for these dimensions (bytes). */
+TV_API size_t tv_attn_workspace_bytes(int B, int Nmax, int Hq, int Hkv, int d, int Scap);
+
+/*
+ * Tree attention of one layer: the attention sub-step of TeacherTreeEval
+ * (Section 2.3) under the tree mask (Section 3.3).  Every active node i and
+ * query head h (KV head h / (Hq/Hkv)) attends the committed prefix rows
+ * [0, prefix_len[b]) of the cache and the tree keys j whose bit is set in
+ * anc_bits[b,i]; softmax of scale * <q,k> with fp32 accumulation.
+ *
+ *   q[B,Nmax,Hq,d]                 in  bf16
+ *   k_cache,v_cache[B,Hkv,Scap,d]  in  bf16, one layer; never written
+ *                                      (state safety, Section 3.3); rows at
+ *                                      or past prefix_len[b] are ignored even
+ *                                      if they hold NaN.
+ *   k_tree,v_tree[B,Nmax,Hkv,d]    in  bf16, the speculative ("branch") K/V
+ *   prefix_len[B], n_nodes[B]      in
+ *   anc_bits[B,Nmax,W]             in  from tree_build_mask
+ *   out[B,Nmax,Hq,d]               out bf16; padded rows are written as 0
+ *   lse[B,Hq,Nmax]                 out or NULL, fp32 log-sum-exp of the
+ *                                      scaled scores; -inf for padded rows
+ *   workspace                      device scratch, 256-byte aligned, at least
+ *                                      tv_attn_workspace_bytes(...) bytes
+ *   status[B]                      in/out: TV_ST_TIMEOUT is ORed in if a
+ *                                      bounded wait expired (outputs invalid)
+ * Limits: d in {64,128}; Nmax <= 128; Hq % Hkv == 0; all tensors 16-byte
+ * aligned; 0 <= prefix_len[b] <= Scap.
+ */
+TV_API int tree_verify_attn(const tv_bf16* q,
+                     const tv_bf16* k_cache, const tv_bf16* v_cache,
+                     const tv_bf16* k_tree, const tv_bf16* v_tree,
+                     const int32_t* prefix_len, const int32_t* n_nodes,
+                     const uint32_t* anc_bits,
+                     int B, int Nmax, int Hq, int Hkv, int d, int Scap, float scale,
+                     tv_bf16* out, float* lse,
+                     void* workspace, size_t workspace_bytes,
+                     int32_t* status, tv_stream stream);
+
+/* Scratch needed by tree_accept (bytes). */
+TV_API size_t tv_accept_workspace_bytes(int B, int Nmax, int V);
+
+/*
+ * Safe path gather, teacher argmax and greedy acceptance.
+ *   - gather (Section 2.5; Section 3.2): an index r of a candidate row is
+ *     usable iff 0 <= r < n_nodes[b]; every other value is remapped to the
+ *     dummy index 0 BEFORE tokens[] is read, and the slot is excluded from
+ *     acceptance by its validity flag.  r < -1 or r >= n_nodes[b] also
+ *     raises TV_ST_BAD_INDEX.
+ *   - argmax (greedy selection, Section 2.1, temperature 0 as in Section 5):
+ *     the lowest v that maximises logits[b,i,v]; values compare as floats;
+ *     inputs are NaN-free by contract (a NaN never wins).
+ *   - accept (Section 2.3): along each row, node j is accepted while its
+ *     token equals the teacher argmax at node j-1 of the row; the longest
+ *     accepted prefix over all rows wins, ties go to the lowest row.
+ *
+ *   logits[B,Nmax,V]          in  bf16
+ *   tokens[B,Nmax]            in  draft token of every node (node 0: the last sampled token)
+ *   retrieve_indices[B,P,Dp1] in  left-aligned root-to-leaf rows, -1 padded
+ *   argmax_tok[B,Nmax]        out (-1 for padded rows)
+ *   safe_idx,candidates[B,P,Dp1] out or NULL
+ *   accept_len[B]             out accepted draft tokens, 0..Dp1-1 (root and bonus token not counted)
+ *   best_path[B]              out winning row
+ *   accepted_nodes[B,Dp1]     out first accept_len+1 entries = root..last accepted node, rest 0
+ *   next_token[B]             out teacher argmax at the last accepted node (the bonus token)
+ *   workspace                 device scratch >= tv_accept_workspace_bytes(B,Nmax,V), 16-byte aligned
+ *   status[B]                 in/out
+ */
+TV_API int tree_accept(const tv_bf16* logits, const int32_t* tokens,
+                const int32_t* retrieve_indices, const int32_t* n_nodes,
+                int B, int Nmax, int V, int P, int Dp1,
+                int32_t* argmax_tok, int32_t* safe_idx, int32_t* candidates,
+                int32_t* accept_len, int32_t* best_path, int32_t* accepted_nodes,
+                int32_t* next_token,
+                void* workspace, size_t workspace_bytes,
+                int32_t* status, tv_stream stream);
+
+/*
+ * Path-index commit with the prefix-sharing fast reorder (Section 3.1): the
+ * committed prefix keeps its place and only the accepted segment is gathered
+ * behind it, in place, for all layers in one call:
+ *   cache[l,b,h,prefix_len[b]+j,:] = tree[l,b,accepted_nodes[b,j],h,:], j = 0..accept_len[b]
+ *   prefix_len[b] += accept_len[b] + 1
+ * A chain tree makes this the length-based commit of Section 3.1.
+ *
+ *   k_cache,v_cache   in/out [L,B,Hkv,Scap,d] with layer stride cache_layer_stride (elements)
+ *   k_tree,v_tree     in     [L,B,Nmax,Hkv,d] with layer stride tree_layer_stride (elements)
+ *   accepted_nodes[B,Dp1], accept_len[B]  in (device; read by the kernel)
+ *   prefix_len[B]     in/out
+ *   status[B]         in/out: a sequence with a fatal bit already set is
+ *                     skipped; TV_ST_CAPACITY if the segment would pass Scap,
+ *                     TV_ST_BAD_INDEX if accept_len or a node id is out of
+ *                     range; such a sequence is left untouched.
+ * Must follow the last tree_verify_attn of the step on the same stream.
+ * Limits: d*2 bytes a multiple of 16; tensors 16-byte aligned.
+ */
+TV_API int kv_commit(tv_bf16* k_cache, tv_bf16* v_cache,
+              const tv_bf16* k_tree, const tv_bf16* v_tree,
+              const int32_t* accepted_nodes, const int32_t* accept_len,
+              int32_t* prefix_len,
+              int L, int B, int Nmax, int Hkv, int d, int Scap, int Dp1,
+              int64_t cache_layer_stride, int64_t tree_layer_stride,
+              int32_t* status, tv_stream stream);
+
+/*
+ * One whole verification step driven from HOST buffers (Section 3 call
+ * order: tensorise + mask, attention per layer, gather + accept, commit).
+ * Per-step inputs are copied host->device into `staging`, the four calls
+ * above run, and the per-step results are copied back; the call returns after
+ * the stream has drained.  The KV cache and prefix_len stay resident on the
+ * device (they are the committed state, not a per-step input).
+ */
+typedef struct tv_step_host_args {
+  /* host, pinned memory recommended */
+  const int32_t* parent;            /* [B,Nmax] */
+  const int32_t* n_nodes;           /* [B] */
+  const int32_t* tokens;            /* [B,Nmax] */
+  const int32_t* retrieve_indices;  /* [B,P,Dp1] or NULL: use the rows tree_build_mask emits */
+  const tv_bf16* q;                 /* [L,B,Nmax,Hq,d] */
+  const tv_bf16* k_tree;            /* [L,B,Nmax,Hkv,d] */
+  const tv_bf16* v_tree;            /* [L,B,Nmax,Hkv,d] */
+  const tv_bf16* logits;            /* [B,Nmax,V] */
+  tv_bf16* out;                     /* [L,B,Nmax,Hq,d] host out */
+  int32_t* accept_len;              /* [B] host out */
+  int32_t* accepted_nodes;          /* [B,Dp1] host out */
+  int32_t* next_token;              /* [B] host out */
+  int32_t* status;                  /* [B] host out */
+  /* device, resident */
+  tv_bf16* k_cache;                 /* [L,B,Hkv,Scap,d] */
+  tv_bf16* v_cache;
+  int32_t* prefix_len;              /* [B] in/out */
+  void* staging;                    /* device scratch >= tv_step_staging_bytes(...) , 256-byte aligned */
+  size_t staging_bytes;
+  int L, B, Nmax, Hq, Hkv, d, Scap, V, P, Dp1;
+  float scale;
+  tv_stream stream;
+} tv_step_host_args;
+
+TV_API size_t tv_step_staging_bytes(int L, int B, int Nmax, int Hq, int Hkv, int d, int Scap, int V, int P, int Dp1);
+TV_API int tv_verify_step_host(const tv_step_host_args* args);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TREEVERIFY_H_ */

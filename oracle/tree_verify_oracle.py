@@ -96,7 +96,7 @@ def tensorize_one(parent, n, Dcap):
     return True, sp, depth, A
 
 
-def build_mask(parent, n_nodes, Dcap, Pcap):
+def build_mask(parent, n_nodes, Dcap, Pcap, emit_paths=True):
     """Tree tensorisation + mask for a batch (Sections 2.4, 3.2, 3.3).
 
     vis[b,i,j] = valid[i] and valid[j] and (exists l in [0,Dcap]: A[l,i] == j)
@@ -106,7 +106,8 @@ def build_mask(parent, n_nodes, Dcap, Pcap):
       depth[B,Nmax], anc_table[B,Dcap+1,Nmax], retrieve[B,Pcap,Dcap+1] (-1 padded),
       n_paths[B], status[B].
     Candidate-path rows: one per leaf, leaves in increasing node id, root
-    first, -1 after the leaf.
+    first, -1 after the leaf.  With emit_paths=False no rows are written
+    (they stay -1), n_paths is the leaf count and nothing can be truncated.
     """
     parent = np.asarray(parent)
     B, Nmax = parent.shape
@@ -144,6 +145,9 @@ def build_mask(parent, n_nodes, Dcap, Pcap):
         row = 0
         for leaf in range(n):
             if has_child[leaf]:
+                continue
+            if not emit_paths:
+                row += 1
                 continue
             if row >= Pcap:
                 out["status"][b] |= ST_PATHS_TRUNCATED
@@ -335,7 +339,8 @@ def verify_step(case_np, scale, Dcap=None, Pcap=None, use_given_retrieve=True):
     parent, n_nodes = case_np["parent"], case_np["n_nodes"]
     Dp1 = case_np["retrieve"].shape[2]
     mk = build_mask(parent, n_nodes, Dp1 - 1 if Dcap is None else Dcap,
-                    case_np["retrieve"].shape[1] if Pcap is None else Pcap)
+                    case_np["retrieve"].shape[1] if Pcap is None else Pcap,
+                    emit_paths=not (use_given_retrieve and "logits" in case_np))
     L = case_np["q"].shape[0]
     outs, lses = [], []
     for l in range(L):

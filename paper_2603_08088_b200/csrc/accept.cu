@@ -1,0 +1,248 @@
+// tree_accept: teacher argmax over the vocabulary (an HBM-bound scan of the
+// logits), the accelerator-safe path gather (Section 2.5 / 3.2) and greedy
+// acceptance along root-to-leaf rows (Section 2.3).
+//
+// Phase 1 (argmax_scan_kernel) streams logits[B,Nmax,V] once with 16-byte
+// loads; every CTA reduces one vocabulary chunk of one row to a (value,
+// index) pair in scratch.  Phase 2 (accept_kernel), one CTA per sequence,
+// folds the chunk pairs in index order, then remaps, gathers and compares.
+// Ties resolve to the lowest index at every level of the reduction.
+#include "common.cuh"
+
+#include <cuda_bf16.h>
+
+namespace {
+
+constexpr int kScanThreads = 256;
+constexpr int kVecPerThread = 4;                                   // 16-byte loads in flight per thread
+constexpr int kChunkElems = kScanThreads * kVecPerThread * 8;      // 8192 logits per CTA
+
+struct ArgPair {
+  float val;
+  int32_t idx;
+};
+
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t bits16) {
+  return __uint_as_float(bits16 << 16);
+}
+
+// (v, i) beats (bv, bi) when it is larger, or equal with a lower index.
+__device__ __forceinline__ void take_better(float& bv, int& bi, float v, int i) {
+  if (v > bv || (v == bv && i < bi)) {
+    bv = v;
+    bi = i;
+  }
+}
+
+__device__ __forceinline__ float vec8_max(const uint4& u) {
+  const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+  __nv_bfloat162 m = __hmax2(__hmax2(h[0], h[1]), __hmax2(h[2], h[3]));
+  const float r = fmaxf(__low2float(m), __high2float(m));   // max of a NaN and x is x
+  return r == r ? r : -INFINITY;                            // an all-NaN vector can never win
+}
+
+__global__ void __launch_bounds__(kScanThreads)
+argmax_scan_kernel(const tv_bf16* __restrict__ logits, const int32_t* __restrict__ n_nodes,
+                   int Nmax, int V, int n_chunks, ArgPair* __restrict__ partial) {
+  const int row = blockIdx.y;            // b * Nmax + i
+  const int b = row / Nmax, i = row - b * Nmax;
+  if (i >= n_nodes[b]) return;           // padded row: never read
+  const int chunk = blockIdx.x;
+  const int c0 = chunk * kChunkElems;
+  const int c1 = min(V, c0 + kChunkElems);
+  const tv_bf16* base = logits + (size_t)row * V;
+  const int tid = threadIdx.x;
+
+  float best = -INFINITY;
+  int best_i = 0x7fffffff;
+
+  const bool vec_ok = ((V & 7) == 0) && ((reinterpret_cast<uintptr_t>(logits) & 15u) == 0);
+  if (vec_ok) {
+    const uint4* vbase = reinterpret_cast<const uint4*>(base);
+    const int v0 = c0 >> 3, v1 = c1 >> 3;      // vector range of this chunk
+    uint4 u[kVecPerThread];
+    int vi[kVecPerThread];
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+      vi[k] = v0 + k * kScanThreads + tid;
+      u[k] = vi[k] < v1 ? __ldg(vbase + vi[k]) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
+    }
+    int best_vec = -1;
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+      const float m = vec8_max(u[k]);
+      if (vi[k] < v1 && (m > best || best_vec < 0)) {   // increasing index order: strict > keeps the first
+        best = m;
+        best_vec = k;
+      }
+    }
+    if (best_vec >= 0) {
+      uint4 w = u[0];
+#pragma unroll
+      for (int k = 1; k < kVecPerThread; ++k) if (best_vec == k) w = u[k];
+      const uint32_t e[4] = {w.x, w.y, w.z, w.w};
+      float bv = -INFINITY;
+      int bi = 0x7fffffff;
+#pragma unroll
+      for (int t = 0; t < 8; ++t) {
+        const uint32_t bits = (t & 1) ? (e[t >> 1] >> 16) : (e[t >> 1] & 0xffffu);
+        float f = bf16_bits_to_float(bits);
+        f = f == f ? f : -INFINITY;
+        take_better(bv, bi, f, t);
+      }
+      int vsel = vi[0];
+#pragma unroll
+      for (int k = 1; k < kVecPerThread; ++k) if (best_vec == k) vsel = vi[k];
+      best = bv;
+      best_i = vsel * 8 + bi;
+    }
+  } else {
+    for (int v = c0 + tid; v < c1; v += kScanThreads) {
+      float f = bf16_bits_to_float(base[v]);
+      f = f == f ? f : -INFINITY;
+      take_better(best, best_i, f, v);
+    }
+  }
+
+  // warp, then block reduction with the same rule
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, best, off);
+    const int oi = __shfl_xor_sync(0xffffffffu, best_i, off);
+    take_better(best, best_i, ov, oi);
+  }
+  __shared__ float sv[kScanThreads / 32];
+  __shared__ int si[kScanThreads / 32];
+  if ((tid & 31) == 0) {
+    sv[tid >> 5] = best;
+    si[tid >> 5] = best_i;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    for (int w = 1; w < kScanThreads / 32; ++w) take_better(best, best_i, sv[w], si[w]);
+    ArgPair out;
+    out.val = best;
+    out.idx = best_i;
+    partial[(size_t)row * n_chunks + chunk] = out;
+  }
+}
+
+__global__ void __launch_bounds__(256)
+accept_kernel(const ArgPair* __restrict__ partial, int n_chunks,
+              const int32_t* __restrict__ tokens, const int32_t* __restrict__ retrieve,
+              const int32_t* __restrict__ n_nodes,
+              int Nmax, int P, int Dp1,
+              int32_t* __restrict__ argmax_tok, int32_t* __restrict__ safe_idx,
+              int32_t* __restrict__ candidates, int32_t* __restrict__ accept_len,
+              int32_t* __restrict__ best_path, int32_t* __restrict__ accepted_nodes,
+              int32_t* __restrict__ next_token, int32_t* __restrict__ status) {
+  extern __shared__ int32_t am[];          // [Nmax] teacher argmax of this sequence
+  __shared__ unsigned long long best_key;  // (accepted length << 32) | ~row : max = longest, then lowest row
+  __shared__ int bad_index;
+  const int b = blockIdx.x;
+  const int tid = threadIdx.x, nt = blockDim.x;
+  int n = n_nodes[b];
+  n = n < 0 ? 0 : (n > Nmax ? Nmax : n);
+  if (tid == 0) {
+    best_key = 0xffffffffull;              // length 0, row 0
+    bad_index = 0;
+  }
+  for (int i = tid; i < Nmax; i += nt) {
+    int tok = -1;
+    if (i < n) {
+      const ArgPair* pp = partial + ((size_t)b * Nmax + i) * n_chunks;
+      float bv = pp[0].val;
+      int bi = pp[0].idx;
+      for (int c = 1; c < n_chunks; ++c) take_better(bv, bi, pp[c].val, pp[c].idx);
+      tok = bi;
+    }
+    am[i] = tok;
+    argmax_tok[(size_t)b * Nmax + i] = tok;
+  }
+  __syncthreads();
+
+  const int32_t* rows = retrieve + (size_t)b * P * Dp1;
+  const int32_t* tok_b = tokens + (size_t)b * Nmax;
+  for (int p = tid; p < P; p += nt) {
+    int a = 0;
+    bool chain = true;
+    bool prev_ok = false;
+    int prev_safe = 0;
+    for (int j = 0; j < Dp1; ++j) {
+      const int r = rows[p * Dp1 + j];
+      const bool ok = r >= 0 && r < n;
+      if (r < -1 || r >= n) bad_index = 1;
+      const int s = ok ? r : 0;            // remap BEFORE the gather: s is always in [0, Nmax)
+      const int cand = tok_b[s];
+      if (safe_idx) safe_idx[((size_t)b * P + p) * Dp1 + j] = s;
+      if (candidates) candidates[((size_t)b * P + p) * Dp1 + j] = cand;
+      if (j > 0 && chain) {
+        if (ok && prev_ok && cand == am[prev_safe]) a = j;
+        else chain = false;
+      }
+      prev_ok = ok;
+      prev_safe = s;
+    }
+    const unsigned long long key = ((unsigned long long)a << 32) | (unsigned long long)(0xffffffffu - (unsigned)p);
+    atomicMax(&best_key, key);
+  }
+  __syncthreads();
+  const int A = (int)(best_key >> 32);
+  const int pstar = (int)(0xffffffffu - (unsigned)(best_key & 0xffffffffull));
+  for (int j = tid; j < Dp1; j += nt) {
+    int node = 0;
+    if (j <= A && P > 0) {
+      const int r = rows[pstar * Dp1 + j];
+      node = (r >= 0 && r < n) ? r : 0;
+    }
+    accepted_nodes[(size_t)b * Dp1 + j] = node;
+    if (j == A) next_token[b] = am[node];
+  }
+  if (tid == 0) {
+    accept_len[b] = A;
+    best_path[b] = pstar;
+    if (bad_index) atomicOr(&status[b], TV_ST_BAD_INDEX);
+  }
+}
+
+int scan_chunks(int V) { return (V + kChunkElems - 1) / kChunkElems; }
+
+}  // namespace
+
+extern "C" size_t tv_accept_workspace_bytes(int B, int Nmax, int V) {
+  if (B <= 0 || Nmax <= 0 || V <= 0) return 16;
+  return (size_t)B * Nmax * scan_chunks(V) * sizeof(ArgPair);
+}
+
+extern "C" int tree_accept(const tv_bf16* logits, const int32_t* tokens,
+                           const int32_t* retrieve_indices, const int32_t* n_nodes,
+                           int B, int Nmax, int V, int P, int Dp1,
+                           int32_t* argmax_tok, int32_t* safe_idx, int32_t* candidates,
+                           int32_t* accept_len, int32_t* best_path, int32_t* accepted_nodes,
+                           int32_t* next_token,
+                           void* workspace, size_t workspace_bytes,
+                           int32_t* status, tv_stream stream) {
+  TV_REQUIRE(logits && tokens && n_nodes && argmax_tok && accept_len && best_path && accepted_nodes &&
+                 next_token && status && workspace,
+             "tree_accept: NULL required pointer");
+  TV_REQUIRE(B >= 0 && Nmax >= 1 && Nmax <= 8192 && V >= 1 && P >= 0 && Dp1 >= 1,
+             "tree_accept: need B >= 0, 1 <= Nmax <= 8192, V >= 1, P >= 0, Dp1 >= 1");
+  TV_REQUIRE(P == 0 || retrieve_indices, "tree_accept: retrieve_indices is NULL with P > 0");
+  TV_REQUIRE(B * (long long)Nmax <= 65535, "tree_accept: B*Nmax exceeds 65535 rows");
+  TV_REQUIRE((reinterpret_cast<uintptr_t>(workspace) & 7u) == 0, "tree_accept: workspace must be 8-byte aligned");
+  if (workspace_bytes < tv_accept_workspace_bytes(B, Nmax, V))
+    return tv::fail(TV_ERR_WORKSPACE, "tree_accept: workspace of %zu bytes, need %zu", workspace_bytes,
+                    tv_accept_workspace_bytes(B, Nmax, V));
+  if (B == 0) return TV_OK;
+  const int n_chunks = scan_chunks(V);
+  ArgPair* partial = static_cast<ArgPair*>(workspace);
+  cudaStream_t s = (cudaStream_t)stream;
+  argmax_scan_kernel<<<dim3(n_chunks, B * Nmax), kScanThreads, 0, s>>>(logits, n_nodes, Nmax, V, n_chunks, partial);
+  TV_CUDA_OK(cudaGetLastError());
+  accept_kernel<<<B, 256, Nmax * sizeof(int32_t), s>>>(partial, n_chunks, tokens, retrieve_indices, n_nodes,
+                                                        Nmax, P, Dp1, argmax_tok, safe_idx, candidates,
+                                                        accept_len, best_path, accepted_nodes, next_token, status);
+  TV_CUDA_OK(cudaGetLastError());
+  tv::count_launches(2);
+  return TV_OK;
+}

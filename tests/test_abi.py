@@ -1,0 +1,62 @@
+"""The C-ABI library builds, loads without a GPU and exports every symbol the
+header declares; host-visible argument errors are reported before any launch."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2603_08088_b200 as tv
+from paper_2603_08088_b200 import build as tv_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    tv_build.build()
+    return tv.load()
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "treeverify.h")).read()
+    return re.findall(r"^TV_API\s+[\w\s\*]+?\b(\w+)\(", text, flags=re.M)
+
+
+def test_header_symbols_are_exported(lib):
+    names = _declared_symbols()
+    assert set(names) >= {"tree_build_mask", "tree_verify_attn", "tree_accept", "kv_commit",
+                          "tv_verify_step_host", "tv_last_error"}
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in treeverify.h but not exported"
+    assert set(names) == set(tv.EXPORTS)
+
+
+def test_version_and_size_queries(lib):
+    assert tv.tv_version() >= 100
+    assert tv.tv_accept_workspace_bytes(16, 60, 153600) >= 16 * 60 * 8
+    assert tv.tv_attn_workspace_bytes(16, 60, 32, 8, 128, 4224) >= 256
+    assert tv.tv_step_staging_bytes(2, 2, 15, 4, 2, 64, 256, 1024, 8, 5) > 0
+
+
+def test_null_and_bad_dims_are_rejected_without_a_launch(lib):
+    rc = lib.tree_build_mask(None, None, 1, 8, 3, 4, None, None, None, None, None, None, None, None)
+    assert rc == 1 and b"NULL" in lib.tv_last_error()
+    one = ctypes.c_void_p(0x1000)
+    rc = lib.tree_build_mask(one, one, 1, 4096, 3, 4, one, None, None, None, None, None, one, None)
+    assert rc == 1 and b"Nmax" in lib.tv_last_error()
+    rc = lib.kv_commit(one, one, one, one, one, one, one, 1, 1, 8, 2, 12, 64, 4, 0, 0, one, None)
+    assert rc == 1
+    rc = lib.tree_accept(one, one, one, one, 1, 8, 100, 2, 3, one, None, None, one, one, one, one, one, 0, one, None)
+    assert rc == 3     # workspace too small
+    rc = lib.tree_verify_attn(one, one, one, one, one, one, one, one, 1, 200, 4, 2, 64, 64, 1.0, one, None,
+                              one, 1 << 30, one, None)
+    assert rc == 1     # Nmax > 128
+
+
+def test_missing_library_fails_loudly(monkeypatch):
+    from paper_2603_08088_b200 import binding
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", "/nonexistent/libtreeverify.so")
+    with pytest.raises(ImportError):
+        binding.load()

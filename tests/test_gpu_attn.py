@@ -1,0 +1,211 @@
+"""tree_verify_attn on the GPU against the fp64 oracle (max-abs 2e-2), plus the
+checks that pin the mask through the whole kernel: closed forms, leak canaries,
+NaN-poisoned padding, non-ancestor perturbation, state safety."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2603_08088_b200 as tv
+from oracle import tree_verify_oracle as orc
+from workloads import (CONFIGS, make_case, case_to_numpy, bf16_bits, random_parent_tree, topk_expansion_tree,
+                       chain_tree)
+from gpu_util import to_device, f32, assert_attention_close, oracle_attention_slice, ATTN_ATOL
+
+pytestmark = pytest.mark.gpu
+
+
+def gpu_attention(case, layer=0, simt=False):
+    """case: device tensors.  Returns (out, lse, anc_bits, dense) for one layer."""
+    L, B, N, Hq, d = case["q"].shape
+    Hkv, Scap = case["k_cache"].shape[2], case["k_cache"].shape[3]
+    dev = case["q"].device
+    W = (N + 31) // 32
+    bits = torch.zeros(B, N, W, dtype=torch.int32, device=dev)
+    dense = torch.zeros(B, 1, N, N, dtype=torch.uint8, device=dev)
+    status = torch.zeros(B, dtype=torch.int32, device=dev)
+    tv.tree_build_mask(case["parent"], case["n_nodes"], N - 1, 1, bits, status, dense_mask=dense)
+    out = torch.full((B, N, Hq, d), 3.0, dtype=torch.bfloat16, device=dev)
+    lse = torch.full((B, Hq, N), 3.0, dtype=torch.float32, device=dev)
+    scale = d ** -0.5
+    if simt:
+        tv.tv_debug_attn_simt(case["q"][layer], case["k_cache"][layer], case["v_cache"][layer],
+                              case["k_tree"][layer], case["v_tree"][layer], case["prefix_len"],
+                              case["n_nodes"], bits, scale, out, lse=lse)
+    else:
+        ws = torch.zeros(max(256, tv.tv_attn_workspace_bytes(B, N, Hq, Hkv, d, Scap)), dtype=torch.uint8, device=dev)
+        tv.tree_verify_attn(case["q"][layer], case["k_cache"][layer], case["v_cache"][layer],
+                            case["k_tree"][layer], case["v_tree"][layer], case["prefix_len"],
+                            case["n_nodes"], bits, scale, out, ws, status, lse=lse)
+    torch.cuda.synchronize()
+    assert (status.cpu().numpy() == 0).all(), f"status {status.cpu().numpy()}"
+    return out, lse, bits, dense
+
+
+def oracle_attention(case_np, dense, layer=0):
+    d = case_np["q"].shape[-1]
+    return orc.tree_attention(case_np["q"][layer], case_np["k_cache"][layer], case_np["v_cache"][layer],
+                              case_np["k_tree"][layer], case_np["v_tree"][layer], case_np["prefix_len"],
+                              case_np["n_nodes"], dense[:, 0], d ** -0.5)
+
+
+SMALL = [
+    # name, base config, overrides: several key tiles, ragged tails, both head dims, G in {1,2,4}
+    ("tiny_full", 0, {}),
+    ("d64_g2_ragged", 0, dict(B=3, S_lo=0, S_hi=300, Scap=320, N=15)),
+    ("d128_g1", 1, dict(Hq=4, Hkv=4, S_lo=129, S_hi=129, Scap=256, N=60)),
+    ("d128_g4_ragged", 2, dict(B=4, Hq=8, Hkv=2, S_lo=1, S_hi=700, Scap=768, N=64)),
+    ("d128_g4_n128", 3, dict(B=2, Hq=8, Hkv=2, S_lo=383, S_hi=385, Scap=512, N=128)),
+    ("d128_g4_n60", 4, dict(B=3, L=2, Hq=8, Hkv=2, S_lo=100, S_hi=520, Scap=640, V=0)),
+]
+
+
+@pytest.mark.parametrize("name,ci,over", SMALL, ids=[s[0] for s in SMALL])
+@pytest.mark.parametrize("simt", [False, True], ids=["tc", "simt"])
+def test_attention_parity_small(name, ci, over, simt):
+    cfg = CONFIGS[ci].scaled(**over)
+    case = make_case(cfg, seed=1000 * ci + 1, ragged_nodes=(cfg.B > 1), with_logits=False)
+    # rows past the prefix and padded tree slots hold NaN: they must never reach an output
+    S = case["prefix_len"].numpy()
+    n = case["n_nodes"].numpy()
+    nan = torch.tensor(float("nan"), dtype=torch.bfloat16)
+    for b in range(cfg.B):
+        case["k_cache"][:, b, :, S[b]:] = nan
+        case["v_cache"][:, b, :, S[b]:] = nan
+        case["k_tree"][:, b, n[b]:] = nan
+        case["v_tree"][:, b, n[b]:] = nan
+        case["q"][:, b, n[b]:] = nan
+    dcase = to_device(case)
+    case_np = case_to_numpy(case)
+    for layer in range(cfg.L):
+        out, lse, bits, dense = gpu_attention(dcase, layer, simt=simt)
+        ref_out, ref_lse = oracle_attention(case_np, dense.cpu().numpy(), layer)
+        assert_attention_close(out, lse, ref_out, ref_lse, name)
+        got = f32(out)
+        for b in range(cfg.B):                       # padded rows are exact zeros / -inf
+            assert (got[b, n[b]:] == 0).all()
+            assert np.isneginf(f32(lse)[b, :, n[b]:]).all()
+
+
+def _tree_case(parent, S, Hq, Hkv, d, Scap, seed, std=1.0):
+    N = len(parent)
+    cfg = CONFIGS[0].scaled(B=1, Hq=Hq, Hkv=Hkv, d=d, S_lo=S, S_hi=S, Scap=Scap, N=N, D=min(3, N - 1), std=std, V=0)
+    case = make_case(cfg, seed=seed, with_logits=False)
+    case["parent"] = torch.from_numpy(parent[None].astype(np.int32))
+    return case
+
+
+@pytest.mark.parametrize("S", [0, 1, 16, 200])
+@pytest.mark.parametrize("d", [64, 128])
+def test_closed_form_zero_keys_pins_the_visible_count(S, d):
+    """K = 0 => lse = ln(S + depth + 1) and out = mean of the visible V rows."""
+    rng = np.random.default_rng(S + d)
+    parent = topk_expansion_tree(40, 6, 4, rng)
+    case = _tree_case(parent, S, 4, 2, d, 256, seed=S)
+    case["k_cache"].zero_()
+    case["k_tree"].zero_()
+    out, lse, bits, dense = gpu_attention(to_device(case))
+    ref_out, ref_lse = oracle_attention(case_to_numpy(case), dense.cpu().numpy())
+    vis = dense.cpu().numpy()[0, 0]
+    want = np.log(S + vis.sum(1))
+    assert np.abs(f32(lse)[0] - want[None, :]).max() < 1e-4
+    assert np.abs(ref_lse[0] - want[None, :]).max() < 1e-12
+    assert_attention_close(out, lse, ref_out, ref_lse, "zero keys")
+
+
+@pytest.mark.parametrize("S", [0, 1, 16])
+def test_leak_canary_one_hot_values(S):
+    """Tree V rows are 100 * e_j and tree keys score alike, so a leaked
+    non-ancestor or a missing ancestor moves the output by far more than 2e-2."""
+    rng = np.random.default_rng(40 + S)
+    N, d = 60, 64
+    parent = topk_expansion_tree(N, 6, 10, rng)
+    case = _tree_case(parent, S, 2, 1, d, 64, seed=S + 9)
+    case["v_tree"].zero_()
+    for j in range(N):
+        case["v_tree"][0, 0, j, 0, j % d] = 100.0
+    case["v_cache"].zero_()
+    case["k_tree"].zero_()
+    case["k_cache"].zero_()
+    out, lse, bits, dense = gpu_attention(to_device(case))
+    ref_out, ref_lse = oracle_attention(case_to_numpy(case), dense.cpu().numpy())
+    vis = dense.cpu().numpy()[0, 0].astype(np.float64)
+    want = np.zeros((N, d))
+    for i in range(N):
+        for j in np.flatnonzero(vis[i]):
+            want[i, j % d] += 100.0 / (S + vis[i].sum())
+    assert np.abs(ref_out[0, :, 0] - want).max() < 1e-9
+    got = f32(out)[0]
+    for h in range(2):
+        assert np.abs(got[:, h] - want).max() <= 0.26      # 100/k rounded to bf16: half-ulp of 64..128 is 0.25
+    # a leak of one key would shift some entry by >= 100/(S+8) > 4
+
+
+def test_non_ancestor_perturbation_leaves_rows_bit_identical():
+    rng = np.random.default_rng(5)
+    parent = topk_expansion_tree(64, 7, 8, rng)
+    case = _tree_case(parent, 300, 8, 2, 128, 512, seed=3, std=128 ** -0.5)
+    dcase = to_device(case)
+    out1, lse1, bits, dense = gpu_attention(dcase)
+    vis = dense.cpu().numpy()[0, 0]
+    victim = 63
+    dcase["k_tree"][0, 0, victim] = 30.0
+    dcase["v_tree"][0, 0, victim] = -50.0
+    out2, lse2, _, _ = gpu_attention(dcase)
+    a, b = bf16_bits(out1), bf16_bits(out2)
+    unaffected = np.flatnonzero(vis[:, victim] == 0)
+    assert len(unaffected) >= 50
+    assert np.array_equal(a[0, unaffected], b[0, unaffected])
+    assert np.array_equal(f32(lse1)[0][:, unaffected], f32(lse2)[0][:, unaffected])
+    assert not np.array_equal(a[0, victim], b[0, victim])
+
+
+def test_state_safety_cache_and_inputs_are_not_written():
+    cfg = CONFIGS[2].scaled(B=2, Hq=8, Hkv=2, S_lo=200, S_hi=400, Scap=512)
+    dcase = to_device(make_case(cfg, seed=8, with_logits=False))
+    before = {k: dcase[k].clone() for k in ("k_cache", "v_cache", "k_tree", "v_tree", "q", "prefix_len")}
+    gpu_attention(dcase)
+    for k, v in before.items():
+        assert torch.equal(v, dcase[k]), f"{k} was modified by tree_verify_attn"
+
+
+def test_chain_tree_is_causal_attention_and_one_node_is_decode():
+    for N in (1, 37):
+        case = _tree_case(chain_tree(N), 150, 4, 4, 128, 256, seed=N, std=0.3)
+        out, lse, bits, dense = gpu_attention(to_device(case))
+        cn = case_to_numpy(case)
+        q = torch.from_numpy(orc.decode_bf16(cn["q"][0]))[0].permute(1, 0, 2)
+        k = torch.cat([torch.from_numpy(orc.decode_bf16(cn["k_cache"][0]))[0, :, :150],
+                       torch.from_numpy(orc.decode_bf16(cn["k_tree"][0]))[0].permute(1, 0, 2)], 1)
+        v = torch.cat([torch.from_numpy(orc.decode_bf16(cn["v_cache"][0]))[0, :, :150],
+                       torch.from_numpy(orc.decode_bf16(cn["v_tree"][0]))[0].permute(1, 0, 2)], 1)
+        allow = torch.ones(N, 150 + N).tril(diagonal=150).bool()
+        ref = torch.nn.functional.scaled_dot_product_attention(q, k, v, attn_mask=allow, scale=128 ** -0.5)
+        err = np.abs(f32(out)[0] - ref.permute(1, 0, 2).numpy()).max()
+        assert err <= ATTN_ATOL
+
+
+FULL = [(1, [(0, 0), (0, 17), (0, 31)]), (2, [(0, 0), (3, 5), (7, 7)]), (3, [(0, 0), (3, 7)]),
+        (4, [(0, 0), (9, 3), (15, 7)])]
+
+
+@pytest.mark.parametrize("ci,samples", FULL, ids=[CONFIGS[c].name for c, _ in FULL])
+def test_attention_full_size_sampled_heads(ci, samples):
+    """Full-size configs in the launch configuration the bench uses; the oracle
+    checks sampled (sequence, KV head) slices one by one."""
+    cfg = CONFIGS[ci].scaled(L=min(CONFIGS[ci].L, 2), V=0)
+    dcase = make_case(cfg, seed=1000 * ci, device="cuda", with_logits=False)
+    layer = cfg.L - 1
+    out, lse, bits, dense = gpu_attention(dcase, layer)
+    vis = dense.cpu().numpy()[:, 0]
+    G = cfg.Hq // cfg.Hkv
+    case_np = {k: (bf16_bits(v[layer:layer + 1]) if v.dtype == torch.bfloat16 else v.cpu().numpy())
+               for k, v in dcase.items() if isinstance(v, torch.Tensor)}
+    got_out, got_lse = f32(out), f32(lse)
+    assert np.isfinite(got_out).all()
+    for (b, hk) in samples:
+        ref_out, ref_lse = oracle_attention_slice(case_np, 0, b, hk, G, vis, cfg.d ** -0.5)
+        err = np.abs(got_out[b:b + 1, :, hk * G:(hk + 1) * G] - ref_out).max()
+        assert err <= ATTN_ATOL, f"(b={b}, hk={hk}): {err}"
+        assert np.abs(got_lse[b:b + 1, hk * G:(hk + 1) * G] - ref_lse).max() <= 2e-3

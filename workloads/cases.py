@@ -39,10 +39,13 @@ def randn_bf16(shape, std, gen, device, chunk_elems=1 << 26):
 
 
 def _draw_tree(cfg: VerifyConfig, n, rng):
-    D = min(cfg.D, n - 1)
-    if cfg.tree == "uniform" or n < cfg.topk + 1:
-        return random_parent_tree(n, D, rng) if n > 1 else np.array([-1], dtype=np.int32)
-    return topk_expansion_tree(n, D, cfg.topk, rng)
+    if n == 1:
+        return np.array([-1], dtype=np.int32)
+    if n < cfg.N:      # a ragged (smaller) tree: uniform parents, depth bound scaled to its size
+        return random_parent_tree(n, min(cfg.D, max(1, (n - 1) // 2)), rng)
+    if cfg.tree == "uniform":
+        return random_parent_tree(n, min(cfg.D, n - 1), rng)
+    return topk_expansion_tree(n, cfg.D, cfg.topk, rng)
 
 
 def make_case(cfg: VerifyConfig, seed: int, device="cpu", ragged_nodes=False,
