@@ -1,16 +1,849 @@
-// tree_verify_attn entry point.
+// tree_verify_attn: GQA tree attention for sm_100a (Sections 2.3, 2.4, 3.3).
+//
+// Packing.  For one sequence b and KV head hk, the G = Hq/Hkv query heads of
+// every tree node share the same K/V, so (node, group member) pairs are packed
+// into dense MMA rows r = node_local * G + g.  A row tile holds 128 rows =
+// 128/G nodes; a CTA owns MT (1 or 2) row tiles and streams 128-key tiles of
+// the committed prefix, then one tile of the tree's own keys.
+//
+// Pipeline (one CTA per SM, 12 warps):
+//   warp 0      TMA producer: Q tiles once per work item, then K and V tiles
+//               through a 5-slot shared-memory ring (128-byte swizzled boxes).
+//   warp 1      tcgen05.mma issuer: S = Q K^T (both operands from shared
+//               memory) into TMEM, O += P V with P read from TMEM; completion
+//               is signalled to mbarriers with tcgen05.commit.
+//   warps 4-7   softmax warpgroup for row tile 0: one thread per row, online
+//   warps 8-11  softmax with lazy rescale; tile 1 likewise.  The ancestor
+//               bitmask of the row (4 words) is applied only on the tree tile,
+//               the prefix length only on the ragged last prefix tile.
+// TMEM: S0 | S1 | O0 | O1, 128 columns each; P (bf16) overlays its S.
+//
+// Work split.  All key tiles of all (b, hk) units form one linear space that
+// is cut evenly over the CTA groups (a group = the CTAs that hold the row
+// tiles of the same unit and walk the same keys together, so the second reader
+// hits L2).  A unit cut in pieces leaves fp32 partials (O, m, l) in the
+// workspace; the piece that arrives last on the unit's counter merges them.
+// Counters carry a per-call epoch, so the workspace needs no initialisation.
+//
+// Every wait on an mbarrier is bounded: on expiry the CTA raises
+// TV_ST_TIMEOUT for all sequences, all roles leave their loops, outstanding
+// copies are given time to land, TMEM is freed and the kernel returns.
 #include "common.cuh"
 
-extern "C" TV_API int tv_debug_attn_simt(const tv_bf16* q, const tv_bf16* k_cache, const tv_bf16* v_cache,
-                                  const tv_bf16* k_tree, const tv_bf16* v_tree,
-                                  const int32_t* prefix_len, const int32_t* n_nodes,
-                                  const uint32_t* anc_bits,
-                                  int B, int Nmax, int Hq, int Hkv, int d, int Scap, float scale,
-                                  tv_bf16* out, float* lse, tv_stream stream);
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include <atomic>
+#include <chrono>
+
+namespace {
+
+constexpr int kTileN = 128;        // keys per tile
+constexpr int kTileM = 128;        // rows per row tile
+constexpr int kSlots = 5;          // K/V ring slots
+constexpr int kThreads = 384;
+constexpr int kMaxB = 512;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kRescaleThreshold = 8.0f;            // in log2 units
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+
+// ---------------------------------------------------------------- PTX helpers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false if the wait was abandoned (timeout here or abort raised elsewhere).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = globaltimer_ns();
+  uint32_t spins = 0;
+  while (true) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((++spins & 255u) == 0) {
+      if (*abort_flag) return false;
+      if (globaltimer_ns() - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        return false;
+      }
+    }
+  }
+}
+__device__ __forceinline__ void fence_barrier_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async_smem() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
+                                            int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1 (sm_100).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((addr & 0x3FFFFu) >> 4);
+  d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= 1ull << 46;
+  d |= 2ull << 61;
+  return d;
+}
+// Instruction descriptor, kind::f16: bf16 x bf16 -> fp32, M = 128, A K-major.
+__host__ __device__ constexpr uint32_t instr_desc(int n, bool b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | (static_cast<uint32_t>(n >> 3) << 17) |
+         (static_cast<uint32_t>(kTileM >> 4) << 24);
+}
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* v) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* v) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
+        "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(v[16]), "r"(v[17]),
+        "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]),
+        "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* v) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
+        "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+
+// ---------------------------------------------------------------- kernel parameters
+struct AttnParams {
+  const int32_t* prefix_len;
+  const int32_t* n_nodes;
+  const uint32_t* anc_bits;
+  tv_bf16* out;
+  float* lse;
+  int32_t* status;
+  float* part_o;                 // [slots][MT*128][D] fp32
+  float* part_ml;                // [slots][MT*128][2]  (m in log2 units, l)
+  unsigned long long* counters;  // [B*Hkv*NP]
+  unsigned long long epoch;      // 48-bit tag of this call
+  int B, Nmax, Hq, Hkv, Scap, G, NPT, NP, W, groups;
+  uint32_t q_box_bytes;          // bytes of one Q box {64, G, NPT}: 16 KB when G divides 128
+  float scale_log2e;             // scale * log2(e)
+  float scale;
+};
+
+struct Item {
+  int b, hk, j0, j1, len, S, n;
+};
+
+// Shared bookkeeping of the linear tile space: cum[b] = sum of len over b' < b, len_b = ceil(S_b/128) + 1.
+struct Sched {
+  const int* cum;
+  int B, Hkv;
+  long long total;   // Hkv * cum[B]
+  __device__ __forceinline__ long long group_start(int k, int groups) const { return (total * k) / groups; }
+  __device__ __forceinline__ int find_b(long long g) const {
+    int lo = 0, hi = B - 1;   // largest b with Hkv*cum[b] <= g
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) >> 1;
+      if ((long long)Hkv * cum[mid] <= g) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+  }
+};
+
+template <int D, int MT>
+struct SmemLayout {
+  static constexpr int kHalf = 64 * 128 * 2;               // one 64-column, 128-row swizzled box: 16 KB
+  static constexpr int kTileBytes = (D / 64) * kHalf;      // a 128 x D bf16 tile
+  static constexpr int kQ = 0;
+  static constexpr int kRing = MT * kTileBytes;
+  static constexpr int kBars = kRing + kSlots * kTileBytes;
+  // barrier indices (8 bytes each)
+  static constexpr int Q_FULL = 0, Q_EMPTY = 1, KV_FULL = 2, KV_EMPTY = 2 + kSlots, S_FULL = 2 + 2 * kSlots,
+                       P_READY = S_FULL + 2, O_DONE = P_READY + 2, EPI = O_DONE + 2, NBARS = EPI + 1;
+  static constexpr int kMisc = kBars + NBARS * 8;          // tmem ptr, abort flag, last flag
+  static constexpr int kCum = kMisc + 16;
+  static constexpr int kTotal = kCum + (kMaxB + 1) * 4;
+};
+
+// ---------------------------------------------------------------- the kernel
+template <int D, int MT>
+__global__ void __launch_bounds__(kThreads, 1)
+tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kc,
+                 const __grid_constant__ CUtensorMap map_vc, const __grid_constant__ CUtensorMap map_kt,
+                 const __grid_constant__ CUtensorMap map_vt, const AttnParams prm) {
+  using L = SmemLayout<D, MT>;
+  extern __shared__ __align__(1024) uint8_t smem[];
+  const uint32_t sbase = smem_u32(smem);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t bars = sbase + L::kBars;
+  auto bar = [&](int i) { return bars + 8u * i; };
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::kMisc + 4);
+  volatile int* last_flag = reinterpret_cast<volatile int*>(smem + L::kMisc + 8);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + L::kMisc);
+  int* cum = reinterpret_cast<int*>(smem + L::kCum);
+
+  // ---- setup: schedule table, barriers, TMEM
+  if (warp == 0) {
+    int run = 0;
+    for (int base = 0; base < prm.B; base += 32) {
+      const int b = base + lane;
+      int len = 0;
+      if (b < prm.B) {
+        int S = prm.prefix_len[b];
+        S = S < 0 ? 0 : (S > prm.Scap ? prm.Scap : S);
+        len = (S + kTileN - 1) / kTileN + 1;
+      }
+      int inc = len;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += t;
+      }
+      if (b < prm.B) cum[b] = run + inc - len;
+      run += __shfl_sync(0xffffffffu, inc, 31);
+    }
+    if (lane == 0) cum[prm.B] = run;
+  }
+  if (threadIdx.x == 32) {
+    mbar_init(bar(L::Q_FULL), 1);
+    mbar_init(bar(L::Q_EMPTY), 1);
+    for (int s = 0; s < kSlots; ++s) {
+      mbar_init(bar(L::KV_FULL + s), 1);
+      mbar_init(bar(L::KV_EMPTY + s), 1);
+    }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(bar(L::S_FULL + s), 1);
+      mbar_init(bar(L::P_READY + s), 128);
+      mbar_init(bar(L::O_DONE + s), 1);
+    }
+    mbar_init(bar(L::EPI), MT * 128);
+    *abort_flag = ((sbase & 1023u) != 0) ? 1 : 0;   // swizzled tiles need a 1024-byte aligned base
+    *last_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32((const void*)tmem_slot))
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  Sched sch{cum, prm.B, prm.Hkv, (long long)prm.Hkv * cum[prm.B]};
+  const int group = blockIdx.x / prm.NP;
+  const int pair = blockIdx.x % prm.NP;
+  const long long g_begin = sch.group_start(group, prm.groups);
+  const long long g_end = sch.group_start(group + 1, prm.groups);
+
+  // Walks the items of this CTA's range; identical in every role.
+  auto next_item = [&](long long& g, Item& it) -> bool {
+    if (g >= g_end) return false;
+    const int b = sch.find_b(g);
+    const int len = cum[b + 1] - cum[b];
+    const long long local = g - (long long)prm.Hkv * cum[b];
+    it.b = b;
+    it.hk = (int)(local / len);
+    it.j0 = (int)(local % len);
+    const long long room = g_end - g;
+    it.j1 = (int)((long long)(len - it.j0) < room ? len : it.j0 + room);
+    it.len = len;
+    int S = prm.prefix_len[b];
+    it.S = S < 0 ? 0 : (S > prm.Scap ? prm.Scap : S);
+    int n = prm.n_nodes[b];
+    it.n = n < 0 ? 0 : (n > prm.Nmax ? prm.Nmax : n);
+    g += it.j1 - it.j0;
+    return true;
+  };
+
+  constexpr uint32_t kIdescQK = instr_desc(kTileN, false);
+  constexpr uint32_t kIdescPV = instr_desc(D, true);
+  constexpr uint32_t kTmemS0 = 0, kTmemO0 = 256;
+
+  if (warp == 0) {
+    // =========================================================== TMA producer
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+    if (lane == 0 && !*abort_flag) {
+      long long g = g_begin;
+      Item it;
+      uint32_t item_idx = 0, fill = 0;
+      bool ok = true;
+      while (ok && next_item(g, it)) {
+        ok = mbar_wait(bar(L::Q_EMPTY), (item_idx & 1) ^ 1, abort_flag);
+        if (!ok) break;
+        mbar_expect_tx(bar(L::Q_FULL), MT * (D / 64) * prm.q_box_bytes);
+#pragma unroll
+        for (int t = 0; t < MT; ++t)
+#pragma unroll
+          for (int h = 0; h < D / 64; ++h)
+            tma_load_4d(sbase + L::kQ + t * L::kTileBytes + h * L::kHalf, &map_q, bar(L::Q_FULL), h * 64,
+                        it.hk * prm.G, (pair * MT + t) * prm.NPT, it.b);
+        ++item_idx;
+        for (int j = it.j0; j < it.j1 && ok; ++j) {
+          const bool tree = (j == it.len - 1);
+#pragma unroll
+          for (int kv = 0; kv < 2; ++kv) {
+            const uint32_t slot = fill % kSlots, round = fill / kSlots;
+            ok = mbar_wait(bar(L::KV_EMPTY + slot), (round & 1) ^ 1, abort_flag);
+            if (!ok) break;
+            mbar_expect_tx(bar(L::KV_FULL + slot), L::kTileBytes);
+            const uint32_t dst = sbase + L::kRing + slot * L::kTileBytes;
+#pragma unroll
+            for (int h = 0; h < D / 64; ++h) {
+              if (tree)
+                tma_load_4d(dst + h * L::kHalf, kv ? &map_vt : &map_kt, bar(L::KV_FULL + slot), h * 64, it.hk, 0, it.b);
+              else
+                tma_load_3d(dst + h * L::kHalf, kv ? &map_vc : &map_kc, bar(L::KV_FULL + slot), h * 64, j * kTileN,
+                            it.b * prm.Hkv + it.hk);
+            }
+            ++fill;
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // =========================================================== MMA issuer
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+    if (lane == 0 && !*abort_flag) {
+      long long g = g_begin;
+      Item it;
+      uint32_t item_idx = 0, fill = 0, gj = 0;
+      bool ok = true;
+      while (ok && next_item(g, it)) {
+        const int nt = it.j1 - it.j0, nj = nt * MT;
+        ok = mbar_wait(bar(L::Q_FULL), item_idx & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        // fill index of K_j is fill + 2*(j - j0), of V_j one more
+        auto issue_qk = [&](int i) -> bool {      // job i of this item: tile j0 + i/MT, row tile i%MT
+          const int jt = i / MT, t = i % MT;
+          const uint32_t f = fill + 2 * jt, slot = f % kSlots;
+          if (t == 0 || MT == 1)
+            if (!mbar_wait(bar(L::KV_FULL + slot), (f / kSlots) & 1, abort_flag)) return false;
+          tc_fence_after();
+          const uint32_t sb = (gj + i) & 1;
+          const uint32_t qa = sbase + L::kQ + t * L::kTileBytes, ka = sbase + L::kRing + slot * L::kTileBytes;
+#pragma unroll
+          for (int ks = 0; ks < D / 16; ++ks) {
+            const uint32_t off = (ks / 4) * L::kHalf + (ks % 4) * 32;
+            mma_ss(tmem + kTmemS0 + sb * 128, smem_desc(qa + off, 16, 1024), smem_desc(ka + off, 16, 1024), kIdescQK,
+                   ks > 0);
+          }
+          mma_commit(bar(L::S_FULL + sb));
+          if (t == MT - 1) mma_commit(bar(L::KV_EMPTY + slot));
+          if (i == nj - 1) mma_commit(bar(L::Q_EMPTY));
+          return true;
+        };
+        ok = issue_qk(0);
+        if (ok && nj > 1) ok = issue_qk(1);
+        for (int i = 0; i < nj && ok; ++i) {
+          const uint32_t gi = gj + i, sb = gi & 1;
+          const int jt = i / MT, t = i % MT;
+          const uint32_t ob = (MT == 2) ? sb : 0;
+          ok = mbar_wait(bar(L::P_READY + sb), (gi >> 1) & 1, abort_flag);
+          if (!ok) break;
+          const uint32_t f = fill + 2 * jt + 1, slot = f % kSlots;
+          ok = mbar_wait(bar(L::KV_FULL + slot), (f / kSlots) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t va = sbase + L::kRing + slot * L::kTileBytes;
+#pragma unroll
+          for (int ks = 0; ks < kTileN / 16; ++ks)
+            mma_ts(tmem + kTmemO0 + ob * 128, tmem + kTmemS0 + sb * 128 + ks * 8,
+                   smem_desc(va + ks * 2048, L::kHalf, 1024), kIdescPV, (jt > 0 || ks > 0) ? 1u : 0u);
+          mma_commit(bar(L::O_DONE + ob));
+          if (t == MT - 1) mma_commit(bar(L::KV_EMPTY + slot));
+          if (i + 2 < nj) ok = issue_qk(i + 2);
+        }
+        fill += 2 * nt;
+        gj += nj;
+        ++item_idx;
+      }
+    }
+  } else if (warp >= 4) {
+    // =========================================================== softmax / epilogue warpgroups
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+    const int wg = (warp - 4) >> 2;                  // row tile of this warpgroup
+    const int row = ((warp & 3) << 5) | lane;        // TMEM lane = row inside the tile
+    const uint32_t lane_addr = (uint32_t)((warp & 3) << 5) << 16;
+    const bool wg_active = wg < MT;
+    if (wg_active && !*abort_flag) {
+      long long g = g_begin;
+      Item it;
+      uint32_t fill = 0, gj = 0, epi_phase = 0;
+      bool ok = true;
+      // Rendezvous of the softmax warpgroups through an mbarrier, so that it is bounded like every other wait.
+      // All 32 lanes wait together and agree on the outcome, so that the warp-wide TMEM instructions
+      // below are never executed by a part of a warp.
+      auto wwait = [&](uint32_t b_, uint32_t parity) -> bool {
+        return __all_sync(0xffffffffu, mbar_wait(b_, parity, abort_flag));
+      };
+      auto epi_sync = [&]() -> bool {
+        mbar_arrive(bar(L::EPI));
+        const bool r = wwait(bar(L::EPI), epi_phase & 1);
+        ++epi_phase;
+        return r;
+      };
+      while (ok && next_item(g, it)) {
+        const int nt = it.j1 - it.j0, nj = nt * MT;
+        const int node = (pair * MT + wg) * prm.NPT + row / prm.G;
+        const int gm = row % prm.G;
+        const bool row_exists = row < prm.NPT * prm.G && node < prm.Nmax;
+        const bool row_active = row_exists && node < it.n;
+        uint32_t anc[4] = {0u, 0u, 0u, 0u};
+        if (row_active) {
+#pragma unroll
+          for (int w = 0; w < 4; ++w)
+            if (w < prm.W) anc[w] = prm.anc_bits[((size_t)it.b * prm.Nmax + node) * prm.W + w];
+        }
+        float m_used = -INFINITY;      // running reference maximum, in log2 units (score * scale * log2e)
+        float l_sum = 0.f;
+        for (int i = (MT == 2 ? wg : 0); i < nj && ok; i += (MT == 2 ? 2 : 1)) {
+          const uint32_t gi = gj + i, sb = gi & 1;
+          const int jt = i / MT, j = it.j0 + jt;
+          const uint32_t ob = (MT == 2) ? sb : 0;
+          const bool tree = (j == it.len - 1);
+          const int valid_keys = tree ? it.n : min(kTileN, it.S - j * kTileN);
+          // ---- V rows past the valid keys may hold anything (stale cache rows, padded tree slots): zero
+          // them so that 0 * NaN never reaches O.  Idempotent, so both warpgroups may do it.
+          if (valid_keys < kTileN) {
+            const uint32_t f = fill + 2 * jt + 1, slot = f % kSlots;
+            ok = wwait(bar(L::KV_FULL + slot), (f / kSlots) & 1);
+            if (!ok) break;
+            if (row >= valid_keys) {
+              uint8_t* vrow = smem + L::kRing + slot * L::kTileBytes + row * 128;
+#pragma unroll
+              for (int h = 0; h < D / 64; ++h)
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
+                  *reinterpret_cast<uint4*>(vrow + h * L::kHalf + c * 16) = make_uint4(0, 0, 0, 0);
+            }
+            fence_proxy_async_smem();
+          }
+          ok = wwait(bar(L::S_FULL + sb), (gi >> 1) & 1);
+          if (!ok) break;
+          tc_fence_after();
+          uint32_t sreg[128];
+          const uint32_t s_addr = tmem + lane_addr + kTmemS0 + sb * 128;
+#pragma unroll
+          for (int q = 0; q < 4; ++q) tmem_ld32(s_addr + q * 32, sreg + q * 32);
+          tmem_wait_ld();
+          float* s = reinterpret_cast<float*>(sreg);
+          if (valid_keys < kTileN || tree) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              uint32_t word;
+              if (tree) {
+                word = anc[q];
+              } else {
+                const int cnt = valid_keys - 32 * q;
+                word = cnt >= 32 ? 0xffffffffu : (cnt <= 0 ? 0u : ((1u << cnt) - 1u));
+              }
+#pragma unroll
+              for (int c = 0; c < 32; ++c)
+                if (!((word >> c) & 1u)) s[q * 32 + c] = -INFINITY;
+            }
+          }
+          float mx = s[0];
+#pragma unroll
+          for (int c = 1; c < 128; ++c) mx = fmaxf(mx, s[c]);
+          const float mx2 = mx * prm.scale_log2e;
+          // ---- lazy rescale: move the reference maximum only when it would grow by more than the threshold.
+          // The TMEM accesses are warp-wide (.sync.aligned), so the warp rescales as soon as one of its rows
+          // has to; rows that keep their maximum multiply by 1.
+          const bool moves = (mx2 > m_used + kRescaleThreshold || m_used == -INFINITY) && mx2 > -INFINITY;
+          const bool scales = moves && jt > 0 && m_used > -INFINITY;
+          const float alpha = scales ? fast_exp2(m_used - mx2) : 1.f;
+          if (moves) m_used = mx2;
+          l_sum *= alpha;
+          if (__any_sync(0xffffffffu, scales)) {
+            if (MT == 1) {   // with one row tile the previous PV may still be running
+              ok = wwait(bar(L::O_DONE + ob), (gi - 1) & 1);
+              tc_fence_after();
+            }
+            if (ok) {
+              const uint32_t o_addr = tmem + lane_addr + kTmemO0 + ob * 128;
+#pragma unroll
+              for (int q = 0; q < D / 32; ++q) {
+                uint32_t o[32];
+                tmem_ld32(o_addr + q * 32, o);
+                tmem_wait_ld();
+#pragma unroll
+                for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+                tmem_st32(o_addr + q * 32, o);
+              }
+            }
+            if (!ok) break;
+          }
+          // ---- P = exp2(s * c - m), row sum in fp32, P rounded to bf16 into TMEM over S
+          const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
+          float ls = 0.f;
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            uint32_t pk[8];
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+              const float p0 = fast_exp2(fmaf(s[q * 16 + 2 * c], prm.scale_log2e, neg_m));
+              const float p1 = fast_exp2(fmaf(s[q * 16 + 2 * c + 1], prm.scale_log2e, neg_m));
+              ls += p0 + p1;
+              pk[c] = pack_bf16(p0, p1);
+            }
+            // 16 keys = 8 packed columns
+            asm volatile(
+                "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                ::"r"(s_addr + q * 8), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]),
+                  "r"(pk[6]), "r"(pk[7])
+                : "memory");
+          }
+          l_sum += ls;
+          tmem_wait_st();
+          tc_fence_before();
+          mbar_arrive(bar(L::P_READY + sb));
+        }
+        if (!ok) break;
+        // ---- epilogue of the item: wait for the last PV into this O buffer
+        {
+          const int i_last = (MT == 2) ? (nj - 2 + wg) : (nj - 1);
+          const uint32_t gi = gj + i_last;
+          const uint32_t ob = (MT == 2) ? (gi & 1) : 0;
+          const uint32_t done_idx = (MT == 2) ? (gi >> 1) : gi;
+          ok = wwait(bar(L::O_DONE + ob), done_idx & 1);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t o_addr = tmem + lane_addr + kTmemO0 + ob * 128;
+          const bool whole = (it.j0 == 0 && it.j1 == it.len);
+          const int h = it.hk * prm.G + gm;
+          tv_bf16* orow = prm.out + (((size_t)it.b * prm.Nmax + node) * prm.Hq + h) * D;
+          float* lse_p = prm.lse ? prm.lse + ((size_t)it.b * prm.Hq + h) * prm.Nmax + node : nullptr;
+          if (whole) {
+            const float inv = (row_active && l_sum > 0.f) ? 1.f / l_sum : 0.f;
+#pragma unroll
+            for (int q = 0; q < D / 32; ++q) {
+              uint32_t o[32];
+              tmem_ld32(o_addr + q * 32, o);
+              tmem_wait_ld();
+              if (row_exists) {
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                  uint4 v;
+                  v.x = pack_bf16(__uint_as_float(o[8 * c + 0]) * inv, __uint_as_float(o[8 * c + 1]) * inv);
+                  v.y = pack_bf16(__uint_as_float(o[8 * c + 2]) * inv, __uint_as_float(o[8 * c + 3]) * inv);
+                  v.z = pack_bf16(__uint_as_float(o[8 * c + 4]) * inv, __uint_as_float(o[8 * c + 5]) * inv);
+                  v.w = pack_bf16(__uint_as_float(o[8 * c + 6]) * inv, __uint_as_float(o[8 * c + 7]) * inv);
+                  if (!row_active) v = make_uint4(0, 0, 0, 0);
+                  *reinterpret_cast<uint4*>(orow + q * 32 + c * 8) = v;
+                }
+              }
+            }
+            if (row_exists && lse_p)
+              *lse_p = (row_active && l_sum > 0.f) ? (m_used + log2f(l_sum)) / kLog2e : -INFINITY;
+            tc_fence_before();
+          } else {
+            // ---- a piece of a unit: leave (O, m, l) in this CTA's slot, then merge if every piece is in
+            const int slot_id = blockIdx.x * 2 + (it.j0 > 0 ? 0 : 1);
+            float* po = prm.part_o + ((size_t)slot_id * (MT * 128) + wg * 128 + row) * D;
+            float* pml = prm.part_ml + ((size_t)slot_id * (MT * 128) + wg * 128 + row) * 2;
+#pragma unroll
+            for (int q = 0; q < D / 32; ++q) {
+              uint32_t o[32];
+              tmem_ld32(o_addr + q * 32, o);
+              tmem_wait_ld();
+              if (row_active) {
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
+                  *reinterpret_cast<uint4*>(po + q * 32 + c * 4) = make_uint4(o[4 * c], o[4 * c + 1], o[4 * c + 2], o[4 * c + 3]);
+              }
+            }
+            if (row_active) {
+              pml[0] = m_used;
+              pml[1] = l_sum;
+            }
+            tc_fence_before();
+            __threadfence();
+            ok = epi_sync();
+            if (!ok) break;
+            // unit geometry in the linear tile space
+            const long long u0 = (long long)prm.Hkv * cum[it.b] + (long long)it.hk * it.len;
+            int k_first = (int)((u0 * prm.groups) / sch.total);
+            while (k_first + 1 < prm.groups && sch.group_start(k_first + 1, prm.groups) <= u0) ++k_first;
+            while (k_first > 0 && sch.group_start(k_first, prm.groups) > u0) --k_first;
+            const long long u_last = u0 + it.len - 1;
+            int k_last = (int)((u_last * prm.groups) / sch.total);
+            while (k_last + 1 < prm.groups && sch.group_start(k_last + 1, prm.groups) <= u_last) ++k_last;
+            while (k_last > 0 && sch.group_start(k_last, prm.groups) > u_last) --k_last;
+            int n_frag = 0;
+            for (int k = k_first; k <= k_last; ++k)
+              n_frag += sch.group_start(k + 1, prm.groups) > sch.group_start(k, prm.groups) ? 1 : 0;
+            if (threadIdx.x == 128) {
+              unsigned long long* ctr = prm.counters + ((size_t)it.b * prm.Hkv + it.hk) * prm.NP + pair;
+              unsigned long long seen = *reinterpret_cast<volatile unsigned long long*>(ctr), want;
+              int cnt;
+              do {
+                const unsigned long long assumed = seen;
+                cnt = ((assumed >> 16) == prm.epoch) ? (int)(assumed & 0xffffu) : 0;
+                want = (prm.epoch << 16) | (unsigned long long)(cnt + 1);
+                seen = atomicCAS(ctr, assumed, want);
+                if (seen == assumed) break;
+              } while (true);
+              *last_flag = (cnt + 1 == n_frag) ? 1 : 0;
+              __threadfence();
+            }
+            ok = epi_sync();
+            if (!ok) break;
+            if (*last_flag) {
+              if (row_exists) {
+                float mm = -INFINITY;
+                if (row_active) {
+                  for (int k = k_first; k <= k_last; ++k) {
+                    const long long ks = sch.group_start(k, prm.groups);
+                    if (sch.group_start(k + 1, prm.groups) <= ks) continue;
+                    const int sid = (k * prm.NP + pair) * 2 + (ks > u0 ? 0 : 1);
+                    const float* q_ml = prm.part_ml + ((size_t)sid * (MT * 128) + wg * 128 + row) * 2;
+                    mm = fmaxf(mm, __ldcg(q_ml));
+                  }
+                }
+                float lt = 0.f;
+                float acc[D];
+#pragma unroll
+                for (int c = 0; c < D; ++c) acc[c] = 0.f;
+                if (row_active) {
+                  for (int k = k_first; k <= k_last; ++k) {
+                    const long long ks = sch.group_start(k, prm.groups);
+                    if (sch.group_start(k + 1, prm.groups) <= ks) continue;
+                    const int sid = (k * prm.NP + pair) * 2 + (ks > u0 ? 0 : 1);
+                    const float* q_ml = prm.part_ml + ((size_t)sid * (MT * 128) + wg * 128 + row) * 2;
+                    const float* q_o = prm.part_o + ((size_t)sid * (MT * 128) + wg * 128 + row) * D;
+                    const float w = fast_exp2(__ldcg(q_ml) - mm);
+                    lt += w * __ldcg(q_ml + 1);
+#pragma unroll
+                    for (int c = 0; c < D / 4; ++c) {
+                      const float4 v = __ldcg(reinterpret_cast<const float4*>(q_o) + c);
+                      acc[4 * c] = fmaf(w, v.x, acc[4 * c]);
+                      acc[4 * c + 1] = fmaf(w, v.y, acc[4 * c + 1]);
+                      acc[4 * c + 2] = fmaf(w, v.z, acc[4 * c + 2]);
+                      acc[4 * c + 3] = fmaf(w, v.w, acc[4 * c + 3]);
+                    }
+                  }
+                }
+                const float inv = (row_active && lt > 0.f) ? 1.f / lt : 0.f;
+#pragma unroll
+                for (int c = 0; c < D / 8; ++c) {
+                  uint4 v;
+                  v.x = pack_bf16(acc[8 * c + 0] * inv, acc[8 * c + 1] * inv);
+                  v.y = pack_bf16(acc[8 * c + 2] * inv, acc[8 * c + 3] * inv);
+                  v.z = pack_bf16(acc[8 * c + 4] * inv, acc[8 * c + 5] * inv);
+                  v.w = pack_bf16(acc[8 * c + 6] * inv, acc[8 * c + 7] * inv);
+                  *reinterpret_cast<uint4*>(orow + c * 8) = v;
+                }
+                if (lse_p) *lse_p = (row_active && lt > 0.f) ? (mm + log2f(lt)) / kLog2e : -INFINITY;
+              }
+            }
+            ok = epi_sync();   // last_flag may be rewritten by the next item only after everyone read it
+            if (!ok) break;
+          }
+        }
+        fill += 2 * nt;
+        gj += nj;
+      }
+    }
+  } else {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+  }
+
+  // ---- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    // give copies that may still be in flight time to land before the shared memory is released
+    const unsigned long long t0 = globaltimer_ns();
+    while (globaltimer_ns() - t0 < 200000ull) {
+    }
+    if (threadIdx.x == 0)
+      for (int b = 0; b < prm.B; ++b) atomicOr(&prm.status[b], TV_ST_TIMEOUT);
+  }
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+bool encode_map(CUtensorMap* m, const void* base, int rank, const cuuint64_t* dims, const cuuint64_t* strides_bytes,
+                const cuuint32_t* box) {
+  cuuint32_t ones[5] = {1, 1, 1, 1, 1};
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), dims, strides_bytes, box, ones,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct Geometry {
+  int G, NPT, n_row_tiles, MT, NP, sms, groups, grid;
+  size_t counters_off, ml_off, o_off, total;
+};
+
+int sm_count() {
+  static int sms = [] {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
+    return n;
+  }();
+  return sms;
+}
+
+Geometry geometry(int B, int Nmax, int Hq, int Hkv, int d, bool query_device) {
+  Geometry g{};
+  g.G = Hq / Hkv;
+  g.NPT = kTileM / g.G;
+  g.n_row_tiles = (Nmax + g.NPT - 1) / g.NPT;
+  g.MT = g.n_row_tiles > 1 ? 2 : 1;
+  g.NP = (g.n_row_tiles + g.MT - 1) / g.MT;
+  g.sms = query_device ? sm_count() : 148;
+  g.groups = g.sms / g.NP > 0 ? g.sms / g.NP : 1;
+  g.grid = g.groups * g.NP;
+  // workspace: counters, then (m,l) pairs, then partial O, sized for 160 SMs so the size does not depend on the device
+  const size_t max_ctas = 160 > g.grid ? 160 : g.grid;
+  g.counters_off = 0;
+  size_t off = (size_t)B * Hkv * g.NP * sizeof(unsigned long long);
+  off = (off + 255) & ~size_t(255);
+  g.ml_off = off;
+  off += max_ctas * 2 * (size_t)g.MT * 128 * 2 * sizeof(float);
+  off = (off + 255) & ~size_t(255);
+  g.o_off = off;
+  off += max_ctas * 2 * (size_t)g.MT * 128 * d * sizeof(float);
+  g.total = off;
+  return g;
+}
+
+unsigned long long next_epoch() {
+  static std::atomic<unsigned long long> ctr{
+      (unsigned long long)std::chrono::steady_clock::now().time_since_epoch().count() * 2654435761ull};
+  return ctr.fetch_add(1, std::memory_order_relaxed) & 0xffffffffffffull;
+}
+
+template <int D, int MT>
+cudaError_t launch(const Geometry& g, const CUtensorMap* maps, const AttnParams& prm, cudaStream_t s) {
+  using L = SmemLayout<D, MT>;
+  static std::atomic<bool> configured[64];
+  auto kern = tree_attn_kernel<D, MT>;
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev < 0 || dev >= 64 || !configured[dev].load(std::memory_order_acquire)) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64) configured[dev].store(true, std::memory_order_release);
+  }
+  kern<<<g.grid, kThreads, L::kTotal, s>>>(maps[0], maps[1], maps[2], maps[3], maps[4], prm);
+  return cudaGetLastError();
+}
+
+}  // namespace
 
 extern "C" size_t tv_attn_workspace_bytes(int B, int Nmax, int Hq, int Hkv, int d, int Scap) {
-  (void)B; (void)Nmax; (void)Hq; (void)Hkv; (void)d; (void)Scap;
-  return 256;
+  (void)Scap;
+  if (B <= 0 || Nmax <= 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0 || Hq / Hkv > kTileM || d <= 0) return 256;
+  return geometry(B, Nmax, Hq, Hkv, d, false).total;
 }
 
 extern "C" int tree_verify_attn(const tv_bf16* q,
@@ -22,10 +855,63 @@ extern "C" int tree_verify_attn(const tv_bf16* q,
                                 tv_bf16* out, float* lse,
                                 void* workspace, size_t workspace_bytes,
                                 int32_t* status, tv_stream stream) {
-  TV_REQUIRE(status && workspace, "tree_verify_attn: NULL pointer");
-  TV_REQUIRE(Nmax <= 128, "tree_verify_attn: Nmax must be <= 128");
-  if (workspace_bytes < tv_attn_workspace_bytes(B, Nmax, Hq, Hkv, d, Scap))
-    return tv::fail(TV_ERR_WORKSPACE, "tree_verify_attn: workspace too small");
-  return tv_debug_attn_simt(q, k_cache, v_cache, k_tree, v_tree, prefix_len, n_nodes, anc_bits,
-                            B, Nmax, Hq, Hkv, d, Scap, scale, out, lse, stream);
+  TV_REQUIRE(q && k_cache && v_cache && k_tree && v_tree && prefix_len && n_nodes && anc_bits && out && status &&
+                 workspace,
+             "tree_verify_attn: NULL pointer");
+  TV_REQUIRE(B >= 0 && B <= kMaxB, "tree_verify_attn: need 0 <= B <= 512");
+  TV_REQUIRE(Nmax >= 1 && Nmax <= 128, "tree_verify_attn: Nmax must be in 1..128");
+  TV_REQUIRE(d == 64 || d == 128, "tree_verify_attn: d must be 64 or 128");
+  TV_REQUIRE(Hq >= 1 && Hkv >= 1 && Hq % Hkv == 0 && Hq / Hkv <= kTileM, "tree_verify_attn: need Hq %% Hkv == 0 and Hq/Hkv <= 128");
+  TV_REQUIRE(Scap >= 1 && scale > 0.f, "tree_verify_attn: need Scap >= 1 and scale > 0");
+  TV_REQUIRE(tv::aligned16(q) && tv::aligned16(k_cache) && tv::aligned16(v_cache) && tv::aligned16(k_tree) &&
+                 tv::aligned16(v_tree) && tv::aligned16(out),
+             "tree_verify_attn: tensors must be 16-byte aligned");
+  TV_REQUIRE((reinterpret_cast<uintptr_t>(workspace) & 255u) == 0, "tree_verify_attn: workspace must be 256-byte aligned");
+  if (B == 0) return TV_OK;
+  const Geometry g = geometry(B, Nmax, Hq, Hkv, d, true);
+  if (g.grid > 160) return tv::fail(TV_ERR_INVALID_ARG, "tree_verify_attn: device with more than 160 SMs is not supported");
+  if (workspace_bytes < g.total)
+    return tv::fail(TV_ERR_WORKSPACE, "tree_verify_attn: workspace of %zu bytes, need %zu", workspace_bytes, g.total);
+
+  CUtensorMap maps[5];
+  {
+    const cuuint64_t e = 2;
+    cuuint64_t qd[4] = {(cuuint64_t)d, (cuuint64_t)Hq, (cuuint64_t)Nmax, (cuuint64_t)B};
+    cuuint64_t qs[3] = {(cuuint64_t)d * e, (cuuint64_t)Hq * d * e, (cuuint64_t)Nmax * Hq * d * e};
+    cuuint32_t qb[4] = {64, (cuuint32_t)g.G, (cuuint32_t)g.NPT, 1};
+    cuuint64_t cd[3] = {(cuuint64_t)d, (cuuint64_t)Scap, (cuuint64_t)B * Hkv};
+    cuuint64_t cs[2] = {(cuuint64_t)d * e, (cuuint64_t)Scap * d * e};
+    cuuint32_t cb[3] = {64, kTileN, 1};
+    cuuint64_t td[4] = {(cuuint64_t)d, (cuuint64_t)Hkv, (cuuint64_t)Nmax, (cuuint64_t)B};
+    cuuint64_t ts[3] = {(cuuint64_t)d * e, (cuuint64_t)Hkv * d * e, (cuuint64_t)Nmax * Hkv * d * e};
+    cuuint32_t tb[4] = {64, 1, kTileN, 1};
+    const bool ok = encode_map(&maps[0], q, 4, qd, qs, qb) && encode_map(&maps[1], k_cache, 3, cd, cs, cb) &&
+                    encode_map(&maps[2], v_cache, 3, cd, cs, cb) && encode_map(&maps[3], k_tree, 4, td, ts, tb) &&
+                    encode_map(&maps[4], v_tree, 4, td, ts, tb);
+    if (!ok) return tv::fail(TV_ERR_CUDA, "tree_verify_attn: cuTensorMapEncodeTiled failed");
+  }
+  AttnParams prm{};
+  prm.prefix_len = prefix_len;
+  prm.n_nodes = n_nodes;
+  prm.anc_bits = anc_bits;
+  prm.out = out;
+  prm.lse = lse;
+  prm.status = status;
+  char* ws = static_cast<char*>(workspace);
+  prm.counters = reinterpret_cast<unsigned long long*>(ws + g.counters_off);
+  prm.part_ml = reinterpret_cast<float*>(ws + g.ml_off);
+  prm.part_o = reinterpret_cast<float*>(ws + g.o_off);
+  prm.epoch = next_epoch();
+  prm.B = B; prm.Nmax = Nmax; prm.Hq = Hq; prm.Hkv = Hkv; prm.Scap = Scap;
+  prm.G = g.G; prm.NPT = g.NPT; prm.NP = g.NP; prm.W = (Nmax + 31) / 32; prm.groups = g.groups;
+  prm.scale = scale;
+  prm.q_box_bytes = 64u * (uint32_t)g.G * (uint32_t)g.NPT * 2u;
+  prm.scale_log2e = scale * kLog2e;
+  cudaStream_t s = (cudaStream_t)stream;
+  cudaError_t e;
+  if (d == 128) e = g.MT == 2 ? launch<128, 2>(g, maps, prm, s) : launch<128, 1>(g, maps, prm, s);
+  else e = g.MT == 2 ? launch<64, 2>(g, maps, prm, s) : launch<64, 1>(g, maps, prm, s);
+  if (e != cudaSuccess) return tv::fail(TV_ERR_CUDA, "tree_verify_attn: launch failed: %s", cudaGetErrorString(e));
+  tv::count_launches(1);
+  return TV_OK;
 }
