@@ -39,6 +39,9 @@ def _newest_header():
 
 
 def build(force=False, verbose=False):
+    extra = os.environ.get("TV_NVCC_EXTRA", "").split()      # e.g. -DNAME=value for tuning builds
+    if extra:
+        force = True
     os.makedirs(OBJ, exist_ok=True)
     nvcc = _nvcc()
     srcs = sorted(f for f in os.listdir(CSRC) if f.endswith(".cu"))
@@ -50,7 +53,7 @@ def build(force=False, verbose=False):
         obj = os.path.join(OBJ, s[:-3] + ".o")
         objs.append(obj)
         if force or not os.path.exists(obj) or os.path.getmtime(obj) < max(os.path.getmtime(src), hdr_time):
-            cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", src, "-o", obj]
+            cmd = [nvcc] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + ["-c", src, "-o", obj]
             jobs.append(cmd)
 
     def run(cmd):

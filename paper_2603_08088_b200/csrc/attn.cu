@@ -46,6 +46,7 @@ constexpr int kMaxB = 512;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kRescaleThreshold = 8.0f;            // in log2 units
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+constexpr int kTraceCap = 256;     // events per (CTA, role) kept by the optional trace
 
 // ---------------------------------------------------------------- PTX helpers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -130,20 +131,28 @@ __host__ __device__ constexpr uint32_t instr_desc(int n, bool b_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | (static_cast<uint32_t>(n >> 3) << 17) |
          (static_cast<uint32_t>(kTileM >> 4) << 24);
 }
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+// tcgen05.mma, kind::f16, one CTA.  The 64-bit shared-memory descriptors are given as (low, high) words: the
+// high word of every descriptor used here is one constant, so the issuing thread only adds an offset to a
+// low word per MMA.
+__device__ __forceinline__ void mma_ss_lohi(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc,
+                                            uint32_t acc) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc)
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "mov.b64 da, {%1, %3};\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(acc)
       : "memory");
 }
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+__device__ __forceinline__ void mma_ts_lohi(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t hi, uint32_t idesc,
+                                            uint32_t acc) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc)
+      "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(hi), "r"(idesc), "r"(acc)
       : "memory");
 }
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
@@ -187,6 +196,19 @@ __device__ __forceinline__ float fast_exp2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// Optional timeline for tuning: role r of this CTA appends (tag, time since kernel start of CTA 0).
+struct Tracer {
+  unsigned long long* base;
+  int n;
+  __device__ __forceinline__ void init(unsigned long long* trace, int role) {
+    base = trace ? trace + ((size_t)blockIdx.x * 4 + role) * kTraceCap : nullptr;
+    n = 0;
+  }
+  __device__ __forceinline__ void mark(uint32_t tag) {
+    if (base && n < kTraceCap) base[n++] = ((unsigned long long)tag << 48) | (globaltimer_ns() & 0xffffffffffffull);
+  }
+};
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t r;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
@@ -201,12 +223,13 @@ struct AttnParams {
   tv_bf16* out;
   float* lse;
   int32_t* status;
-  float* part_o;                 // [slots][MT*128][D] fp32
-  float* part_ml;                // [slots][MT*128][2]  (m in log2 units, l)
+  float* part_o;                 // [slots][D/4][MT*128][4] fp32, column-group major
+  float* part_ml;                // [slots][2][MT*128]  (m in log2 units, then l)
   unsigned long long* counters;  // [B*Hkv*NP]
   unsigned long long epoch;      // 48-bit tag of this call
   int B, Nmax, Hq, Hkv, Scap, G, NPT, NP, W, groups;
-  uint32_t q_box_bytes;          // bytes of one Q box {64, G, NPT}: 16 KB when G divides 128
+  uint32_t q_box_bytes;
+  unsigned long long* trace;     // optional event trace [cta][role 0..3][kTraceCap] of (tag << 48 | ns), or NULL          // bytes of one Q box {64, G, NPT}: 16 KB when G divides 128
   float scale_log2e;             // scale * log2(e)
   float scale;
 };
@@ -344,15 +367,19 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 
   if (warp == 0) {
     // =========================================================== TMA producer
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
     if (lane == 0 && !*abort_flag) {
       long long g = g_begin;
       Item it;
       uint32_t item_idx = 0, fill = 0;
       bool ok = true;
+      Tracer tr;
+      tr.init(prm.trace, 0);
+      tr.mark(0);
       while (ok && next_item(g, it)) {
         ok = mbar_wait(bar(L::Q_EMPTY), (item_idx & 1) ^ 1, abort_flag);
         if (!ok) break;
+        tr.mark(0x1000u | item_idx);
         mbar_expect_tx(bar(L::Q_FULL), MT * (D / 64) * prm.q_box_bytes);
 #pragma unroll
         for (int t = 0; t < MT; ++t)
@@ -368,6 +395,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             const uint32_t slot = fill % kSlots, round = fill / kSlots;
             ok = mbar_wait(bar(L::KV_EMPTY + slot), (round & 1) ^ 1, abort_flag);
             if (!ok) break;
+            tr.mark(0x2000u | (fill & 0xfffu));
             mbar_expect_tx(bar(L::KV_FULL + slot), L::kTileBytes);
             const uint32_t dst = sbase + L::kRing + slot * L::kTileBytes;
 #pragma unroll
@@ -385,17 +413,26 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     }
   } else if (warp == 1) {
     // =========================================================== MMA issuer
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
     if (lane == 0 && !*abort_flag) {
       long long g = g_begin;
       Item it;
       uint32_t item_idx = 0, fill = 0, gj = 0;
       bool ok = true;
+      Tracer tr;
+      tr.init(prm.trace, 1);
+      tr.mark(0);
+      // descriptor words: low = start address >> 4 | LBO field, high = SBO 1024 B | version 1 | 128-byte swizzle
+      const uint32_t desc_hi = (uint32_t)(smem_desc(0, 0, 1024) >> 32);
+      const uint32_t q_lo = (uint32_t)smem_desc(sbase + L::kQ, 16, 1024);          // K-major: LBO unused
+      const uint32_t k_lo = (uint32_t)smem_desc(sbase + L::kRing, 16, 1024);
+      const uint32_t v_lo = (uint32_t)smem_desc(sbase + L::kRing, L::kHalf, 1024); // MN-major: LBO = next 64 columns
       while (ok && next_item(g, it)) {
         const int nt = it.j1 - it.j0, nj = nt * MT;
         ok = mbar_wait(bar(L::Q_FULL), item_idx & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
+        tr.mark(0x1000u | item_idx);
         // fill index of K_j is fill + 2*(j - j0), of V_j one more
         auto issue_qk = [&](int i) -> bool {      // job i of this item: tile j0 + i/MT, row tile i%MT
           const int jt = i / MT, t = i % MT;
@@ -404,16 +441,17 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             if (!mbar_wait(bar(L::KV_FULL + slot), (f / kSlots) & 1, abort_flag)) return false;
           tc_fence_after();
           const uint32_t sb = (gj + i) & 1;
-          const uint32_t qa = sbase + L::kQ + t * L::kTileBytes, ka = sbase + L::kRing + slot * L::kTileBytes;
+          const uint32_t qa = q_lo + t * (L::kTileBytes >> 4), ka = k_lo + slot * (L::kTileBytes >> 4);
 #pragma unroll
           for (int ks = 0; ks < D / 16; ++ks) {
-            const uint32_t off = (ks / 4) * L::kHalf + (ks % 4) * 32;
-            mma_ss(tmem + kTmemS0 + sb * 128, smem_desc(qa + off, 16, 1024), smem_desc(ka + off, 16, 1024), kIdescQK,
-                   ks > 0);
+            constexpr int kHalf16 = L::kHalf >> 4;
+            const uint32_t off = (ks / 4) * kHalf16 + (ks % 4) * 2;      // 16 columns = 32 bytes inside a swizzled row
+            mma_ss_lohi(tmem + kTmemS0 + sb * 128, qa + off, ka + off, desc_hi, kIdescQK, ks > 0);
           }
           mma_commit(bar(L::S_FULL + sb));
           if (t == MT - 1) mma_commit(bar(L::KV_EMPTY + slot));
           if (i == nj - 1) mma_commit(bar(L::Q_EMPTY));
+          tr.mark(0x2000u | ((gj + i) & 0xfffu));
           return true;
         };
         ok = issue_qk(0);
@@ -422,19 +460,22 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           const uint32_t gi = gj + i, sb = gi & 1;
           const int jt = i / MT, t = i % MT;
           const uint32_t ob = (MT == 2) ? sb : 0;
+          tr.mark(0x3000u | (gi & 0xfffu));
           ok = mbar_wait(bar(L::P_READY + sb), (gi >> 1) & 1, abort_flag);
           if (!ok) break;
           const uint32_t f = fill + 2 * jt + 1, slot = f % kSlots;
           ok = mbar_wait(bar(L::KV_FULL + slot), (f / kSlots) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t va = sbase + L::kRing + slot * L::kTileBytes;
+          tr.mark(0x4000u | (gi & 0xfffu));
+          const uint32_t va = v_lo + slot * (L::kTileBytes >> 4);
 #pragma unroll
-          for (int ks = 0; ks < kTileN / 16; ++ks)
-            mma_ts(tmem + kTmemO0 + ob * 128, tmem + kTmemS0 + sb * 128 + ks * 8,
-                   smem_desc(va + ks * 2048, L::kHalf, 1024), kIdescPV, (jt > 0 || ks > 0) ? 1u : 0u);
+          for (int ks = 0; ks < kTileN / 16; ++ks)        // 16 keys = 16 rows of 128 bytes
+            mma_ts_lohi(tmem + kTmemO0 + ob * 128, tmem + kTmemS0 + sb * 128 + ks * 8, va + ks * 128, desc_hi, kIdescPV,
+                        (jt > 0 || ks > 0) ? 1u : 0u);
           mma_commit(bar(L::O_DONE + ob));
           if (t == MT - 1) mma_commit(bar(L::KV_EMPTY + slot));
+          tr.mark(0x5000u | (gi & 0xfffu));
           if (i + 2 < nj) ok = issue_qk(i + 2);
         }
         fill += 2 * nt;
@@ -444,7 +485,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     }
   } else if (warp >= 4) {
     // =========================================================== softmax / epilogue warpgroups
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
     const int wg = (warp - 4) >> 2;                  // row tile of this warpgroup
     const int row = ((warp & 3) << 5) | lane;        // TMEM lane = row inside the tile
     const uint32_t lane_addr = (uint32_t)((warp & 3) << 5) << 16;
@@ -454,6 +495,9 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       Item it;
       uint32_t fill = 0, gj = 0, epi_phase = 0;
       bool ok = true;
+      Tracer tr;
+      tr.init((threadIdx.x & 127) == 0 ? prm.trace : nullptr, 2 + wg);
+      tr.mark(0);
       // Rendezvous of the softmax warpgroups through an mbarrier, so that it is bounded like every other wait.
       // All 32 lanes wait together and agree on the outcome, so that the warp-wide TMEM instructions
       // below are never executed by a part of a warp.
@@ -502,9 +546,11 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             }
             fence_proxy_async_smem();
           }
+          tr.mark(0x0800u | (gi & 0x7ffu));
           ok = wwait(bar(L::S_FULL + sb), (gi >> 1) & 1);
           if (!ok) break;
           tc_fence_after();
+          tr.mark(0x1000u | (gi & 0xfffu));
           uint32_t sreg[128];
           const uint32_t s_addr = tmem + lane_addr + kTmemS0 + sb * 128;
 #pragma unroll
@@ -539,6 +585,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           if (moves) m_used = mx2;
           l_sum *= alpha;
           if (__any_sync(0xffffffffu, scales)) {
+            tr.mark(0x9000u | (gi & 0xfffu));
             if (MT == 1) {   // with one row tile the previous PV may still be running
               ok = wwait(bar(L::O_DONE + ob), (gi - 1) & 1);
               tc_fence_after();
@@ -581,6 +628,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           tmem_wait_st();
           tc_fence_before();
           mbar_arrive(bar(L::P_READY + sb));
+          tr.mark(0x2000u | (gi & 0xfffu));
         }
         if (!ok) break;
         // ---- epilogue of the item: wait for the last PV into this O buffer
@@ -592,6 +640,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           ok = wwait(bar(L::O_DONE + ob), done_idx & 1);
           if (!ok) break;
           tc_fence_after();
+          tr.mark(0x5000u);
           const uint32_t o_addr = tmem + lane_addr + kTmemO0 + ob * 128;
           const bool whole = (it.j0 == 0 && it.j1 == it.len);
           const int h = it.hk * prm.G + gm;
@@ -621,10 +670,14 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               *lse_p = (row_active && l_sum > 0.f) ? (m_used + log2f(l_sum)) / kLog2e : -INFINITY;
             tc_fence_before();
           } else {
-            // ---- a piece of a unit: leave (O, m, l) in this CTA's slot, then merge if every piece is in
+            // ---- a piece of a unit: leave (O, m, l) in this CTA's slot, then merge if every piece is in.
+            // Partial O is stored column-group major, [slot][D/4][MT*128 rows][4 floats], so that the 32 rows
+            // of a warp write (and later read) 512 contiguous bytes per instruction.
+            constexpr int kRows = MT * 128;
+            const int rr = wg * 128 + row;
             const int slot_id = blockIdx.x * 2 + (it.j0 > 0 ? 0 : 1);
-            float* po = prm.part_o + ((size_t)slot_id * (MT * 128) + wg * 128 + row) * D;
-            float* pml = prm.part_ml + ((size_t)slot_id * (MT * 128) + wg * 128 + row) * 2;
+            float* po = prm.part_o + (size_t)slot_id * (D / 4) * kRows * 4;
+            float* pml = prm.part_ml + (size_t)slot_id * 2 * kRows;
 #pragma unroll
             for (int q = 0; q < D / 32; ++q) {
               uint32_t o[32];
@@ -633,15 +686,17 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               if (row_active) {
 #pragma unroll
                 for (int c = 0; c < 8; ++c)
-                  *reinterpret_cast<uint4*>(po + q * 32 + c * 4) = make_uint4(o[4 * c], o[4 * c + 1], o[4 * c + 2], o[4 * c + 3]);
+                  *reinterpret_cast<uint4*>(po + ((size_t)(q * 8 + c) * kRows + rr) * 4) =
+                      make_uint4(o[4 * c], o[4 * c + 1], o[4 * c + 2], o[4 * c + 3]);
               }
             }
             if (row_active) {
-              pml[0] = m_used;
-              pml[1] = l_sum;
+              pml[rr] = m_used;
+              pml[kRows + rr] = l_sum;
             }
             tc_fence_before();
             __threadfence();
+            tr.mark(0x6000u);
             ok = epi_sync();
             if (!ok) break;
             // unit geometry in the linear tile space
@@ -672,50 +727,77 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             }
             ok = epi_sync();
             if (!ok) break;
+            tr.mark(0x7000u | (*last_flag ? 1u : 0u));
             if (*last_flag) {
               if (row_exists) {
-                float mm = -INFINITY;
+                // pass 1: reference maximum and total weight of the row over all pieces
+                float mm = -INFINITY, lt = 0.f;
                 if (row_active) {
                   for (int k = k_first; k <= k_last; ++k) {
                     const long long ks = sch.group_start(k, prm.groups);
                     if (sch.group_start(k + 1, prm.groups) <= ks) continue;
                     const int sid = (k * prm.NP + pair) * 2 + (ks > u0 ? 0 : 1);
-                    const float* q_ml = prm.part_ml + ((size_t)sid * (MT * 128) + wg * 128 + row) * 2;
-                    mm = fmaxf(mm, __ldcg(q_ml));
+                    mm = fmaxf(mm, __ldcg(prm.part_ml + (size_t)sid * 2 * kRows + rr));
                   }
-                }
-                float lt = 0.f;
-                float acc[D];
-#pragma unroll
-                for (int c = 0; c < D; ++c) acc[c] = 0.f;
-                if (row_active) {
                   for (int k = k_first; k <= k_last; ++k) {
                     const long long ks = sch.group_start(k, prm.groups);
                     if (sch.group_start(k + 1, prm.groups) <= ks) continue;
                     const int sid = (k * prm.NP + pair) * 2 + (ks > u0 ? 0 : 1);
-                    const float* q_ml = prm.part_ml + ((size_t)sid * (MT * 128) + wg * 128 + row) * 2;
-                    const float* q_o = prm.part_o + ((size_t)sid * (MT * 128) + wg * 128 + row) * D;
-                    const float w = fast_exp2(__ldcg(q_ml) - mm);
-                    lt += w * __ldcg(q_ml + 1);
-#pragma unroll
-                    for (int c = 0; c < D / 4; ++c) {
-                      const float4 v = __ldcg(reinterpret_cast<const float4*>(q_o) + c);
-                      acc[4 * c] = fmaf(w, v.x, acc[4 * c]);
-                      acc[4 * c + 1] = fmaf(w, v.y, acc[4 * c + 1]);
-                      acc[4 * c + 2] = fmaf(w, v.z, acc[4 * c + 2]);
-                      acc[4 * c + 3] = fmaf(w, v.w, acc[4 * c + 3]);
-                    }
+                    const float* q_ml = prm.part_ml + (size_t)sid * 2 * kRows;
+                    lt += fast_exp2(__ldcg(q_ml + rr) - mm) * __ldcg(q_ml + kRows + rr);
                   }
                 }
                 const float inv = (row_active && lt > 0.f) ? 1.f / lt : 0.f;
+                // pass 2: 32 output columns at a time, every piece weighted by exp2(m_piece - mm); the loads
+                // of two pieces are issued together to cover the L2 latency
+#pragma unroll 1
+                for (int q = 0; q < D / 32; ++q) {
+                  float acc[32];
 #pragma unroll
-                for (int c = 0; c < D / 8; ++c) {
-                  uint4 v;
-                  v.x = pack_bf16(acc[8 * c + 0] * inv, acc[8 * c + 1] * inv);
-                  v.y = pack_bf16(acc[8 * c + 2] * inv, acc[8 * c + 3] * inv);
-                  v.z = pack_bf16(acc[8 * c + 4] * inv, acc[8 * c + 5] * inv);
-                  v.w = pack_bf16(acc[8 * c + 6] * inv, acc[8 * c + 7] * inv);
-                  *reinterpret_cast<uint4*>(orow + c * 8) = v;
+                  for (int c = 0; c < 32; ++c) acc[c] = 0.f;
+                  if (row_active) {
+                    int k = k_first;
+                    while (k <= k_last) {
+                      int sid[2];
+                      int got = 0;
+                      for (; k <= k_last && got < 2; ++k) {
+                        const long long ks = sch.group_start(k, prm.groups);
+                        if (sch.group_start(k + 1, prm.groups) <= ks) continue;
+                        sid[got++] = (k * prm.NP + pair) * 2 + (ks > u0 ? 0 : 1);
+                      }
+                      if (got == 1) sid[1] = sid[0];
+                      float w[2];
+                      float4 v[2][8];
+#pragma unroll
+                      for (int f = 0; f < 2; ++f) {
+                        w[f] = fast_exp2(__ldcg(prm.part_ml + (size_t)sid[f] * 2 * kRows + rr) - mm);
+                        const float* q_o = prm.part_o + (size_t)sid[f] * (D / 4) * kRows * 4;
+#pragma unroll
+                        for (int c = 0; c < 8; ++c)
+                          v[f][c] = __ldcg(reinterpret_cast<const float4*>(q_o + ((size_t)(q * 8 + c) * kRows + rr) * 4));
+                      }
+                      if (got == 1) w[1] = 0.f;
+                      if (got == 0) w[0] = 0.f;
+#pragma unroll
+                      for (int f = 0; f < 2; ++f)
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                          acc[4 * c] = fmaf(w[f], v[f][c].x, acc[4 * c]);
+                          acc[4 * c + 1] = fmaf(w[f], v[f][c].y, acc[4 * c + 1]);
+                          acc[4 * c + 2] = fmaf(w[f], v[f][c].z, acc[4 * c + 2]);
+                          acc[4 * c + 3] = fmaf(w[f], v[f][c].w, acc[4 * c + 3]);
+                        }
+                    }
+                  }
+#pragma unroll
+                  for (int c = 0; c < 4; ++c) {
+                    uint4 v;
+                    v.x = pack_bf16(acc[8 * c + 0] * inv, acc[8 * c + 1] * inv);
+                    v.y = pack_bf16(acc[8 * c + 2] * inv, acc[8 * c + 3] * inv);
+                    v.z = pack_bf16(acc[8 * c + 4] * inv, acc[8 * c + 5] * inv);
+                    v.w = pack_bf16(acc[8 * c + 6] * inv, acc[8 * c + 7] * inv);
+                    *reinterpret_cast<uint4*>(orow + q * 32 + c * 8) = v;
+                  }
                 }
                 if (lse_p) *lse_p = (row_active && lt > 0.f) ? (mm + log2f(lt)) / kLog2e : -INFINITY;
               }
@@ -724,12 +806,13 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             if (!ok) break;
           }
         }
+        tr.mark(0x8000u);
         fill += 2 * nt;
         gj += nj;
       }
     }
   } else {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
   }
 
   // ---- teardown
@@ -816,6 +899,8 @@ Geometry geometry(int B, int Nmax, int Hq, int Hkv, int d, bool query_device) {
   return g;
 }
 
+std::atomic<unsigned long long*> g_trace{nullptr};
+
 unsigned long long next_epoch() {
   static std::atomic<unsigned long long> ctr{
       (unsigned long long)std::chrono::steady_clock::now().time_since_epoch().count() * 2654435761ull};
@@ -839,6 +924,12 @@ cudaError_t launch(const Geometry& g, const CUtensorMap* maps, const AttnParams&
 }
 
 }  // namespace
+
+// Tuning aid: while a device buffer of 160*4*256 u64 is registered here, every tree_verify_attn launch
+// records a per-CTA, per-role timeline (tag << 48 | globaltimer ns) into it.  NULL switches it off.
+extern "C" TV_API void tv_debug_set_attn_trace(unsigned long long* device_buffer) {
+  g_trace.store(device_buffer, std::memory_order_relaxed);
+}
 
 extern "C" size_t tv_attn_workspace_bytes(int B, int Nmax, int Hq, int Hkv, int d, int Scap) {
   (void)Scap;
@@ -906,6 +997,7 @@ extern "C" int tree_verify_attn(const tv_bf16* q,
   prm.G = g.G; prm.NPT = g.NPT; prm.NP = g.NP; prm.W = (Nmax + 31) / 32; prm.groups = g.groups;
   prm.scale = scale;
   prm.q_box_bytes = 64u * (uint32_t)g.G * (uint32_t)g.NPT * 2u;
+  prm.trace = g_trace.load(std::memory_order_relaxed);
   prm.scale_log2e = scale * kLog2e;
   cudaStream_t s = (cudaStream_t)stream;
   cudaError_t e;
