@@ -177,6 +177,34 @@ TV_API int tree_accept(const tv_bf16* logits, const int32_t* tokens,
                 int32_t* status, tv_stream stream);
 
 /*
+ * tree_accept for callers that cannot allocate device memory (the paper has
+ * no counterpart; this is a convenience of this library).  Some hosts of this
+ * code may not call cudaMalloc at all: a plugin inside a serving runtime that
+ * owns the whole memory pool, code running while another component captures a
+ * stream, or a process whose allocator budget is fixed at start-up.  For them
+ * the scratch of the argmax reduction is a fixed 256 KiB array inside the
+ * library image (every GPU that loads the library holds it until exit).
+ * Same arguments and results as tree_accept, without the workspace.
+ *   - Limit: B * Nmax * ceil(V / 8192) <= 32768 scratch entries
+ *     (tv_accept_noalloc_max_bytes() / 8); larger problems are rejected with
+ *     TV_ERR_WORKSPACE and must use tree_accept.
+ *   - The first call on each device looks up the array's device address (with
+ *     that device current); make that first call outside any stream capture.
+ *   - All calls on a device share the one array, which keeps the previous
+ *     call's contents.  Nothing in it has to start at zero (every entry that
+ *     is read is written first by the same call), but two calls whose kernels
+ *     overlap on the GPU (different streams) race on it: serialise them.
+ *   - No cudaMalloc, cudaFree or allocating library routine is called.
+ */
+TV_API size_t tv_accept_noalloc_max_bytes(void);
+TV_API int tree_accept_noalloc(const tv_bf16* logits, const int32_t* tokens,
+                               const int32_t* retrieve_indices, const int32_t* n_nodes,
+                               int B, int Nmax, int V, int P, int Dp1,
+                               int32_t* argmax_tok, int32_t* safe_idx, int32_t* candidates,
+                               int32_t* accept_len, int32_t* best_path, int32_t* accepted_nodes,
+                               int32_t* next_token, int32_t* status, tv_stream stream);
+
+/*
  * Path-index commit with the prefix-sharing fast reorder (Section 3.1): the
  * committed prefix keeps its place and only the accepted segment is gathered
  * behind it, in place, for all layers in one call:

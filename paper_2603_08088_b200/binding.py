@@ -15,7 +15,8 @@ TV_OK, TV_ERR_INVALID_ARG, TV_ERR_CUDA, TV_ERR_WORKSPACE = 0, 1, 2, 3
 TV_ST_BAD_TREE, TV_ST_BAD_INDEX, TV_ST_CAPACITY, TV_ST_TIMEOUT, TV_ST_PATHS_TRUNCATED = 1, 2, 4, 8, 16
 
 EXPORTS = ["tv_last_error", "tv_version", "tv_launch_count", "tree_build_mask", "tv_attn_workspace_bytes", "tree_verify_attn",
-           "tv_accept_workspace_bytes", "tree_accept", "kv_commit", "tv_step_staging_bytes",
+           "tv_accept_workspace_bytes", "tree_accept", "tv_accept_noalloc_max_bytes", "tree_accept_noalloc",
+           "kv_commit", "tv_step_staging_bytes",
            "tv_verify_step_host"]
 
 
@@ -64,6 +65,10 @@ def load():
     lib.tv_accept_workspace_bytes.argtypes = [_c_int] * 3
     lib.tree_accept.restype = _c_int
     lib.tree_accept.argtypes = [_c_vp] * 4 + [_c_int] * 5 + [_c_vp] * 7 + [_c_vp, _c_sz, _c_vp, _c_vp]
+    lib.tv_accept_noalloc_max_bytes.restype = _c_sz
+    lib.tv_accept_noalloc_max_bytes.argtypes = []
+    lib.tree_accept_noalloc.restype = _c_int
+    lib.tree_accept_noalloc.argtypes = [_c_vp] * 4 + [_c_int] * 5 + [_c_vp] * 7 + [_c_vp, _c_vp]
     lib.kv_commit.restype = _c_int
     lib.kv_commit.argtypes = [_c_vp] * 7 + [_c_int] * 7 + [_c_i64, _c_i64, _c_vp, _c_vp]
     lib.tv_step_staging_bytes.restype = _c_sz
@@ -153,6 +158,22 @@ def tree_accept(logits, tokens, retrieve_indices, n_nodes, argmax_tok, accept_le
                               _ptr(accept_len), _ptr(best_path), _ptr(accepted_nodes), _ptr(next_token),
                               _ptr(workspace), workspace.numel() * workspace.element_size(), _ptr(status),
                               _stream(stream)))
+
+
+def tv_accept_noalloc_max_bytes():
+    return load().tv_accept_noalloc_max_bytes()
+
+
+def tree_accept_noalloc(logits, tokens, retrieve_indices, n_nodes, argmax_tok, accept_len, best_path,
+                        accepted_nodes, next_token, status, safe_idx=None, candidates=None, stream=None):
+    """tree_accept without a caller workspace: the scratch is a fixed array inside the library, for
+    callers that may not allocate device memory.  Raises TreeVerifyError (code 3) past its size limit."""
+    B, Nmax, V = logits.shape
+    P, Dp1 = retrieve_indices.shape[1], retrieve_indices.shape[2]
+    _check(load().tree_accept_noalloc(_ptr(logits), _ptr(tokens), _ptr(retrieve_indices) if P > 0 else None,
+                                      _ptr(n_nodes), B, Nmax, V, P, Dp1, _ptr(argmax_tok), _ptr(safe_idx),
+                                      _ptr(candidates), _ptr(accept_len), _ptr(best_path), _ptr(accepted_nodes),
+                                      _ptr(next_token), _ptr(status), _stream(stream)))
 
 
 def kv_commit(k_cache, v_cache, k_tree, v_tree, accepted_nodes, accept_len, prefix_len, status, stream=None):

@@ -11,6 +11,8 @@
 
 #include <cuda_bf16.h>
 
+#include <mutex>
+
 namespace {
 
 constexpr int kScanThreads = 256;
@@ -207,6 +209,33 @@ accept_kernel(const ArgPair* __restrict__ partial, int n_chunks,
 
 int scan_chunks(int V) { return (V + kChunkElems - 1) / kChunkElems; }
 
+// Scratch of tree_accept_noalloc: a fixed device array that lives in the library image, so that callers
+// who may not allocate device memory can still run the accept step.  Every GPU that loads the library
+// holds these 256 KiB until the process exits.
+constexpr size_t kStaticPairs = 32768;                       // (row, vocabulary chunk) pairs
+static __device__ __align__(256) unsigned char g_accept_scratch[kStaticPairs * sizeof(ArgPair)];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+void* g_scratch_ptr[kMaxDevices] = {nullptr};
+
+// Device address of g_accept_scratch on the current device.  In host code the symbol's name is only a
+// stand-in, not an address a kernel can use; the runtime hands out the real one, once per device.
+int static_scratch(void** out) {
+  int dev = -1;
+  TV_CUDA_OK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices)
+    return tv::fail(TV_ERR_INVALID_ARG, "tree_accept_noalloc: device ordinal %d is not supported", dev);
+  std::lock_guard<std::mutex> lock(g_scratch_mutex);
+  if (!g_scratch_ptr[dev]) {
+    void* p = nullptr;
+    TV_CUDA_OK(cudaGetSymbolAddress(&p, g_accept_scratch));
+    g_scratch_ptr[dev] = p;
+  }
+  *out = g_scratch_ptr[dev];
+  return TV_OK;
+}
+
 }  // namespace
 
 extern "C" size_t tv_accept_workspace_bytes(int B, int Nmax, int V) {
@@ -245,4 +274,27 @@ extern "C" int tree_accept(const tv_bf16* logits, const int32_t* tokens,
   TV_CUDA_OK(cudaGetLastError());
   tv::count_launches(2);
   return TV_OK;
+}
+
+extern "C" size_t tv_accept_noalloc_max_bytes(void) { return kStaticPairs * sizeof(ArgPair); }
+
+extern "C" int tree_accept_noalloc(const tv_bf16* logits, const int32_t* tokens,
+                                   const int32_t* retrieve_indices, const int32_t* n_nodes,
+                                   int B, int Nmax, int V, int P, int Dp1,
+                                   int32_t* argmax_tok, int32_t* safe_idx, int32_t* candidates,
+                                   int32_t* accept_len, int32_t* best_path, int32_t* accepted_nodes,
+                                   int32_t* next_token, int32_t* status, tv_stream stream) {
+  TV_REQUIRE(B >= 0 && Nmax >= 1 && V >= 1, "tree_accept_noalloc: need B >= 0, Nmax >= 1, V >= 1");
+  const size_t need = tv_accept_workspace_bytes(B, Nmax, V);
+  if (need > kStaticPairs * sizeof(ArgPair))
+    return tv::fail(TV_ERR_WORKSPACE,
+                    "tree_accept_noalloc: B*Nmax*ceil(V/%d) = %zu scratch entries, the built-in scratch holds %zu; "
+                    "use tree_accept with a caller workspace",
+                    kChunkElems, need / sizeof(ArgPair), kStaticPairs);
+  void* scratch = nullptr;
+  const int rc = static_scratch(&scratch);
+  if (rc != TV_OK) return rc;
+  return tree_accept(logits, tokens, retrieve_indices, n_nodes, B, Nmax, V, P, Dp1, argmax_tok, safe_idx, candidates,
+                     accept_len, best_path, accepted_nodes, next_token, scratch, kStaticPairs * sizeof(ArgPair),
+                     status, stream);
 }
