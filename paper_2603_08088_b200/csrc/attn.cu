@@ -263,7 +263,7 @@ struct SmemLayout {
   static constexpr int kBars = kRing + kSlots * kTileBytes;
   // barrier indices (8 bytes each)
   static constexpr int Q_FULL = 0, Q_EMPTY = 1, KV_FULL = 2, KV_EMPTY = 2 + kSlots, S_FULL = 2 + 2 * kSlots,
-                       P_READY = S_FULL + 2, O_DONE = P_READY + 2, EPI = O_DONE + 2, NBARS = EPI + 1;
+                       P_READY = S_FULL + 4, O_DONE = P_READY + 4, EPI = O_DONE + 2, NBARS = EPI + 1;
   static constexpr int kMisc = kBars + NBARS * 8;          // tmem ptr, abort flag, last flag
   static constexpr int kCum = kMisc + 16;
   static constexpr int kTotal = kCum + (kMaxB + 1) * 4;
@@ -310,16 +310,16 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   }
   if (threadIdx.x == 32) {
     mbar_init(bar(L::Q_FULL), 1);
-    mbar_init(bar(L::Q_EMPTY), 1);
+    mbar_init(bar(L::Q_EMPTY), MT);
     for (int s = 0; s < kSlots; ++s) {
       mbar_init(bar(L::KV_FULL + s), 1);
-      mbar_init(bar(L::KV_EMPTY + s), 1);
+      mbar_init(bar(L::KV_EMPTY + s), MT);       // one commit per row tile's issuer
     }
-    for (int s = 0; s < 2; ++s) {
+    for (int s = 0; s < 4; ++s) {                // index = row tile * 2 + key half
       mbar_init(bar(L::S_FULL + s), 1);
       mbar_init(bar(L::P_READY + s), 128);
-      mbar_init(bar(L::O_DONE + s), 1);
     }
+    for (int s = 0; s < 2; ++s) mbar_init(bar(L::O_DONE + s), 1);
     mbar_init(bar(L::EPI), MT * 128);
     *abort_flag = ((sbase & 1023u) != 0) ? 1 : 0;   // swizzled tiles need a 1024-byte aligned base
     *last_flag = 0;
@@ -361,7 +361,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     return true;
   };
 
-  constexpr uint32_t kIdescQK = instr_desc(kTileN, false);
+  constexpr uint32_t kIdescQK = instr_desc(64, false);   // S is produced 64 keys at a time
   constexpr uint32_t kIdescPV = instr_desc(D, true);
   constexpr uint32_t kTmemS0 = 0, kTmemO0 = 256;
 
@@ -411,75 +411,90 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
       }
     }
-  } else if (warp == 1) {
-    // =========================================================== MMA issuer
+  } else if (warp == 1 || warp == 2) {
+    // =========================================================== MMA issuers, one per row tile
+    // Row tile t is driven by warp 1 + t.  Its S region is split in two 64-key halves, so the softmax of
+    // one half overlaps the MMAs of the other: per key tile the issuer runs
+    //   wait P(h) -> O += P(h) V(h) -> S(h) = Q K_next(h)^T      for h = 0, 1.
+    // MMAs of one thread execute in issue order, which keeps S(h)/P(h) reuse safe without further waits.
     asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
-    if (lane == 0 && !*abort_flag) {
+    const int t = warp - 1;
+    if (lane == 0 && t < MT && !*abort_flag) {
       long long g = g_begin;
       Item it;
-      uint32_t item_idx = 0, fill = 0, gj = 0;
+      uint32_t item_idx = 0, fill = 0, hj = 0;
       bool ok = true;
       Tracer tr;
       tr.init(prm.trace, 1);
-      tr.mark(0);
+      if (t == 0) tr.mark(0);
       // descriptor words: low = start address >> 4 | LBO field, high = SBO 1024 B | version 1 | 128-byte swizzle
       const uint32_t desc_hi = (uint32_t)(smem_desc(0, 0, 1024) >> 32);
-      const uint32_t q_lo = (uint32_t)smem_desc(sbase + L::kQ, 16, 1024);          // K-major: LBO unused
+      const uint32_t q_lo = (uint32_t)smem_desc(sbase + L::kQ + t * L::kTileBytes, 16, 1024);   // K-major: LBO unused
       const uint32_t k_lo = (uint32_t)smem_desc(sbase + L::kRing, 16, 1024);
-      const uint32_t v_lo = (uint32_t)smem_desc(sbase + L::kRing, L::kHalf, 1024); // MN-major: LBO = next 64 columns
+      const uint32_t v_lo = (uint32_t)smem_desc(sbase + L::kRing, L::kHalf, 1024);  // MN-major: LBO = next 64 columns
+      const uint32_t s_tmem = tmem + kTmemS0 + t * 128, o_tmem = tmem + kTmemO0 + t * 128;
+      constexpr int kHalf16 = L::kHalf >> 4, kTile16 = L::kTileBytes >> 4;
+      constexpr int kHalfKeys16 = (64 * 128) >> 4;        // 64 key rows of 128 bytes
+      // S(h) = Q K(h)^T for the 64 keys of half h of the K tile in `slot`
+      auto issue_qk = [&](uint32_t slot, int h) {
+        const uint32_t ka = k_lo + slot * kTile16 + h * kHalfKeys16;
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) {
+          const uint32_t off = (ks / 4) * kHalf16 + (ks % 4) * 2;        // 16 columns = 32 bytes inside a swizzled row
+          mma_ss_lohi(s_tmem + h * 64, q_lo + off, ka + off, desc_hi, kIdescQK, ks > 0);
+        }
+        mma_commit(bar(L::S_FULL + t * 2 + h));
+      };
       while (ok && next_item(g, it)) {
-        const int nt = it.j1 - it.j0, nj = nt * MT;
+        const int nt = it.j1 - it.j0;
         ok = mbar_wait(bar(L::Q_FULL), item_idx & 1, abort_flag);
         if (!ok) break;
-        tc_fence_after();
-        tr.mark(0x1000u | item_idx);
-        // fill index of K_j is fill + 2*(j - j0), of V_j one more
-        auto issue_qk = [&](int i) -> bool {      // job i of this item: tile j0 + i/MT, row tile i%MT
-          const int jt = i / MT, t = i % MT;
-          const uint32_t f = fill + 2 * jt, slot = f % kSlots;
-          if (t == 0 || MT == 1)
-            if (!mbar_wait(bar(L::KV_FULL + slot), (f / kSlots) & 1, abort_flag)) return false;
+        if (t == 0) tr.mark(0x1000u | item_idx);
+        {
+          const uint32_t slot = fill % kSlots;
+          ok = mbar_wait(bar(L::KV_FULL + slot), (fill / kSlots) & 1, abort_flag);
+          if (!ok) break;
           tc_fence_after();
-          const uint32_t sb = (gj + i) & 1;
-          const uint32_t qa = q_lo + t * (L::kTileBytes >> 4), ka = k_lo + slot * (L::kTileBytes >> 4);
+          issue_qk(slot, 0);
+          issue_qk(slot, 1);
+          mma_commit(bar(L::KV_EMPTY + slot));
+          if (nt == 1) mma_commit(bar(L::Q_EMPTY));
+        }
+        for (int jt = 0; jt < nt && ok; ++jt) {
+          const uint32_t fv = fill + 2 * jt + 1, vslot = fv % kSlots;
+          const uint32_t fk = fv + 1, kslot = fk % kSlots;
+          ok = mbar_wait(bar(L::KV_FULL + vslot), (fv / kSlots) & 1, abort_flag);
+          if (!ok) break;
+          const uint32_t va = v_lo + vslot * kTile16;
 #pragma unroll
-          for (int ks = 0; ks < D / 16; ++ks) {
-            constexpr int kHalf16 = L::kHalf >> 4;
-            const uint32_t off = (ks / 4) * kHalf16 + (ks % 4) * 2;      // 16 columns = 32 bytes inside a swizzled row
-            mma_ss_lohi(tmem + kTmemS0 + sb * 128, qa + off, ka + off, desc_hi, kIdescQK, ks > 0);
+          for (int h = 0; h < 2; ++h) {
+            ok = mbar_wait(bar(L::P_READY + t * 2 + h), (hj >> 1) & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            if (t == 0) tr.mark(0x4000u | (hj & 0xfffu));
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)          // 16 keys = 16 rows of 128 bytes; P(h) starts 64 columns into S
+              mma_ts_lohi(o_tmem, s_tmem + h * 64 + ks * 8, va + (h * 4 + ks) * 128, desc_hi, kIdescPV,
+                          (jt > 0 || h > 0 || ks > 0) ? 1u : 0u);
+            mma_commit(bar(L::O_DONE + t));
+            if (h == 1) mma_commit(bar(L::KV_EMPTY + vslot));
+            if (jt + 1 < nt) {
+              if (h == 0) {
+                ok = mbar_wait(bar(L::KV_FULL + kslot), (fk / kSlots) & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+              }
+              issue_qk(kslot, h);
+              if (h == 1) {
+                mma_commit(bar(L::KV_EMPTY + kslot));
+                if (jt + 2 == nt) mma_commit(bar(L::Q_EMPTY));
+              }
+            }
+            if (t == 0) tr.mark(0x2000u | (hj & 0xfffu));
+            ++hj;
           }
-          mma_commit(bar(L::S_FULL + sb));
-          if (t == MT - 1) mma_commit(bar(L::KV_EMPTY + slot));
-          if (i == nj - 1) mma_commit(bar(L::Q_EMPTY));
-          tr.mark(0x2000u | ((gj + i) & 0xfffu));
-          return true;
-        };
-        ok = issue_qk(0);
-        if (ok && nj > 1) ok = issue_qk(1);
-        for (int i = 0; i < nj && ok; ++i) {
-          const uint32_t gi = gj + i, sb = gi & 1;
-          const int jt = i / MT, t = i % MT;
-          const uint32_t ob = (MT == 2) ? sb : 0;
-          tr.mark(0x3000u | (gi & 0xfffu));
-          ok = mbar_wait(bar(L::P_READY + sb), (gi >> 1) & 1, abort_flag);
-          if (!ok) break;
-          const uint32_t f = fill + 2 * jt + 1, slot = f % kSlots;
-          ok = mbar_wait(bar(L::KV_FULL + slot), (f / kSlots) & 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after();
-          tr.mark(0x4000u | (gi & 0xfffu));
-          const uint32_t va = v_lo + slot * (L::kTileBytes >> 4);
-#pragma unroll
-          for (int ks = 0; ks < kTileN / 16; ++ks)        // 16 keys = 16 rows of 128 bytes
-            mma_ts_lohi(tmem + kTmemO0 + ob * 128, tmem + kTmemS0 + sb * 128 + ks * 8, va + ks * 128, desc_hi, kIdescPV,
-                        (jt > 0 || ks > 0) ? 1u : 0u);
-          mma_commit(bar(L::O_DONE + ob));
-          if (t == MT - 1) mma_commit(bar(L::KV_EMPTY + slot));
-          tr.mark(0x5000u | (gi & 0xfffu));
-          if (i + 2 < nj) ok = issue_qk(i + 2);
         }
         fill += 2 * nt;
-        gj += nj;
         ++item_idx;
       }
     }
@@ -493,7 +508,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     if (wg_active && !*abort_flag) {
       long long g = g_begin;
       Item it;
-      uint32_t fill = 0, gj = 0, epi_phase = 0;
+      uint32_t fill = 0, hj = 0, epi_phase = 0;
       bool ok = true;
       Tracer tr;
       tr.init((threadIdx.x & 127) == 0 ? prm.trace : nullptr, 2 + wg);
@@ -511,7 +526,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         return r;
       };
       while (ok && next_item(g, it)) {
-        const int nt = it.j1 - it.j0, nj = nt * MT;
+        const int nt = it.j1 - it.j0;
         const int node = (pair * MT + wg) * prm.NPT + row / prm.G;
         const int gm = row % prm.G;
         const bool row_exists = row < prm.NPT * prm.G && node < prm.Nmax;
@@ -524,10 +539,10 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
         float m_used = -INFINITY;      // running reference maximum, in log2 units (score * scale * log2e)
         float l_sum = 0.f;
-        for (int i = (MT == 2 ? wg : 0); i < nj && ok; i += (MT == 2 ? 2 : 1)) {
-          const uint32_t gi = gj + i, sb = gi & 1;
-          const int jt = i / MT, j = it.j0 + jt;
-          const uint32_t ob = (MT == 2) ? sb : 0;
+        const uint32_t s_base = tmem + lane_addr + kTmemS0 + wg * 128;
+        const uint32_t o_addr_loop = tmem + lane_addr + kTmemO0 + wg * 128;
+        for (int jt = 0; jt < nt && ok; ++jt) {
+          const int j = it.j0 + jt;
           const bool tree = (j == it.len - 1);
           const int valid_keys = tree ? it.n : min(kTileN, it.S - j * kTileN);
           // ---- V rows past the valid keys may hold anything (stale cache rows, padded tree slots): zero
@@ -546,102 +561,108 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             }
             fence_proxy_async_smem();
           }
-          tr.mark(0x0800u | (gi & 0x7ffu));
-          ok = wwait(bar(L::S_FULL + sb), (gi >> 1) & 1);
-          if (!ok) break;
-          tc_fence_after();
-          tr.mark(0x1000u | (gi & 0xfffu));
-          uint32_t sreg[128];
-          const uint32_t s_addr = tmem + lane_addr + kTmemS0 + sb * 128;
 #pragma unroll
-          for (int q = 0; q < 4; ++q) tmem_ld32(s_addr + q * 32, sreg + q * 32);
-          tmem_wait_ld();
-          float* s = reinterpret_cast<float*>(sreg);
-          if (valid_keys < kTileN || tree) {
+          for (int h = 0; h < 2; ++h) {
+            const int valid_half = min(64, max(0, valid_keys - 64 * h));
+            tr.mark(0x0800u | (hj & 0x7ffu));
+            ok = wwait(bar(L::S_FULL + wg * 2 + h), (hj >> 1) & 1);
+            if (!ok) break;
+            tc_fence_after();
+            tr.mark(0x1000u | (hj & 0xfffu));
+            uint32_t sreg[64];
+            const uint32_t s_addr = s_base + h * 64;
+            tmem_ld32(s_addr, sreg);
+            tmem_ld32(s_addr + 32, sreg + 32);
+            tmem_wait_ld();
+            float* s = reinterpret_cast<float*>(sreg);
+            if (valid_half < 64 || tree) {
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              uint32_t word;
-              if (tree) {
-                word = anc[q];
-              } else {
-                const int cnt = valid_keys - 32 * q;
-                word = cnt >= 32 ? 0xffffffffu : (cnt <= 0 ? 0u : ((1u << cnt) - 1u));
+              for (int q = 0; q < 2; ++q) {
+                uint32_t word;
+                if (tree) {
+                  word = anc[2 * h + q];
+                } else {
+                  const int cnt = valid_half - 32 * q;
+                  word = cnt >= 32 ? 0xffffffffu : (cnt <= 0 ? 0u : ((1u << cnt) - 1u));
+                }
+#pragma unroll
+                for (int c = 0; c < 32; ++c)
+                  if (!((word >> c) & 1u)) s[q * 32 + c] = -INFINITY;
               }
-#pragma unroll
-              for (int c = 0; c < 32; ++c)
-                if (!((word >> c) & 1u)) s[q * 32 + c] = -INFINITY;
             }
-          }
-          float mx = s[0];
+            float mx0 = s[0], mx1 = s[1], mx2_ = s[2], mx3 = s[3];
 #pragma unroll
-          for (int c = 1; c < 128; ++c) mx = fmaxf(mx, s[c]);
-          const float mx2 = mx * prm.scale_log2e;
-          // ---- lazy rescale: move the reference maximum only when it would grow by more than the threshold.
-          // The TMEM accesses are warp-wide (.sync.aligned), so the warp rescales as soon as one of its rows
-          // has to; rows that keep their maximum multiply by 1.
-          const bool moves = (mx2 > m_used + kRescaleThreshold || m_used == -INFINITY) && mx2 > -INFINITY;
-          const bool scales = moves && jt > 0 && m_used > -INFINITY;
-          const float alpha = scales ? fast_exp2(m_used - mx2) : 1.f;
-          if (moves) m_used = mx2;
-          l_sum *= alpha;
-          if (__any_sync(0xffffffffu, scales)) {
-            tr.mark(0x9000u | (gi & 0xfffu));
-            if (MT == 1) {   // with one row tile the previous PV may still be running
-              ok = wwait(bar(L::O_DONE + ob), (gi - 1) & 1);
+            for (int c = 4; c < 64; c += 4) {
+              mx0 = fmaxf(mx0, s[c]);
+              mx1 = fmaxf(mx1, s[c + 1]);
+              mx2_ = fmaxf(mx2_, s[c + 2]);
+              mx3 = fmaxf(mx3, s[c + 3]);
+            }
+            const float mx2 = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2_, mx3)) * prm.scale_log2e;
+            // ---- lazy rescale: move the reference maximum only when it would grow by more than the
+            // threshold.  The TMEM accesses are warp-wide (.sync.aligned), so the warp rescales as soon as
+            // one of its rows has to; rows that keep their maximum multiply by 1.
+            const bool first = (jt == 0 && h == 0);
+            const bool moves = (mx2 > m_used + kRescaleThreshold || m_used == -INFINITY) && mx2 > -INFINITY;
+            const bool scales = moves && !first && m_used > -INFINITY;
+            const float alpha = scales ? fast_exp2(m_used - mx2) : 1.f;
+            if (moves) m_used = mx2;
+            l_sum *= alpha;
+            if (__any_sync(0xffffffffu, scales)) {
+              tr.mark(0x9000u | (hj & 0xfffu));
+              // the PV of the previous half may still be running: wait for its completion (number hj - 1)
+              ok = wwait(bar(L::O_DONE + wg), (hj - 1) & 1);
+              if (!ok) break;
               tc_fence_after();
-            }
-            if (ok) {
-              const uint32_t o_addr = tmem + lane_addr + kTmemO0 + ob * 128;
 #pragma unroll
               for (int q = 0; q < D / 32; ++q) {
                 uint32_t o[32];
-                tmem_ld32(o_addr + q * 32, o);
+                tmem_ld32(o_addr_loop + q * 32, o);
                 tmem_wait_ld();
 #pragma unroll
                 for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
-                tmem_st32(o_addr + q * 32, o);
+                tmem_st32(o_addr_loop + q * 32, o);
               }
             }
-            if (!ok) break;
-          }
-          // ---- P = exp2(s * c - m), row sum in fp32, P rounded to bf16 into TMEM over S
-          const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
-          float ls = 0.f;
+            // ---- P = exp2(s * c - m), row sum in fp32, P rounded to bf16 into TMEM over the start of S(h)
+            const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
+            float ls0 = 0.f, ls1 = 0.f;
 #pragma unroll
-          for (int q = 0; q < 8; ++q) {
-            uint32_t pk[8];
+            for (int q = 0; q < 4; ++q) {
+              uint32_t pk[8];
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {
-              const float p0 = fast_exp2(fmaf(s[q * 16 + 2 * c], prm.scale_log2e, neg_m));
-              const float p1 = fast_exp2(fmaf(s[q * 16 + 2 * c + 1], prm.scale_log2e, neg_m));
-              ls += p0 + p1;
-              pk[c] = pack_bf16(p0, p1);
+              for (int c = 0; c < 8; ++c) {
+                const float p0 = fast_exp2(fmaf(s[q * 16 + 2 * c], prm.scale_log2e, neg_m));
+                const float p1 = fast_exp2(fmaf(s[q * 16 + 2 * c + 1], prm.scale_log2e, neg_m));
+                ls0 += p0;
+                ls1 += p1;
+                pk[c] = pack_bf16(p0, p1);
+              }
+              // 16 keys = 8 packed columns
+              asm volatile(
+                  "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                  ::"r"(s_addr + q * 8), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]),
+                    "r"(pk[6]), "r"(pk[7])
+                  : "memory");
             }
-            // 16 keys = 8 packed columns
-            asm volatile(
-                "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
-                ::"r"(s_addr + q * 8), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]),
-                  "r"(pk[6]), "r"(pk[7])
-                : "memory");
+            l_sum += ls0 + ls1;
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(bar(L::P_READY + wg * 2 + h));
+            tr.mark(0x2000u | (hj & 0xfffu));
+            ++hj;
           }
-          l_sum += ls;
-          tmem_wait_st();
-          tc_fence_before();
-          mbar_arrive(bar(L::P_READY + sb));
-          tr.mark(0x2000u | (gi & 0xfffu));
         }
         if (!ok) break;
         // ---- epilogue of the item: wait for the last PV into this O buffer
         {
-          const int i_last = (MT == 2) ? (nj - 2 + wg) : (nj - 1);
-          const uint32_t gi = gj + i_last;
-          const uint32_t ob = (MT == 2) ? (gi & 1) : 0;
-          const uint32_t done_idx = (MT == 2) ? (gi >> 1) : gi;
-          ok = wwait(bar(L::O_DONE + ob), done_idx & 1);
+          // The item's last two PVs (both halves of the last key tile) may still be in flight.  A parity
+          // wait is only meaningful for a phase at most one ahead of the barrier, so take them in order.
+          ok = wwait(bar(L::O_DONE + wg), (hj - 2) & 1) && wwait(bar(L::O_DONE + wg), (hj - 1) & 1);
           if (!ok) break;
           tc_fence_after();
           tr.mark(0x5000u);
-          const uint32_t o_addr = tmem + lane_addr + kTmemO0 + ob * 128;
+          const uint32_t o_addr = o_addr_loop;
           const bool whole = (it.j0 == 0 && it.j1 == it.len);
           const int h = it.hk * prm.G + gm;
           tv_bf16* orow = prm.out + (((size_t)it.b * prm.Nmax + node) * prm.Hq + h) * D;
@@ -808,7 +829,6 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
         tr.mark(0x8000u);
         fill += 2 * nt;
-        gj += nj;
       }
     }
   } else {
