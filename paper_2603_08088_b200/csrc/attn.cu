@@ -225,7 +225,7 @@ struct AttnParams {
   int32_t* status;
   float* part_o;                 // [slots][D/4][MT*128][4] fp32, column-group major
   float* part_ml;                // [slots][2][MT*128]  (m in log2 units, then l)
-  unsigned long long* counters;  // [B*Hkv*NP]
+  unsigned long long* counters;  // [B*Hkv*NP][2]: tickets claimed, partials ready (epoch-tagged)
   unsigned long long epoch;      // 48-bit tag of this call
   int B, Nmax, Hq, Hkv, Scap, G, NPT, NP, W, groups;
   uint32_t q_box_bytes;
@@ -263,7 +263,8 @@ struct SmemLayout {
   static constexpr int kBars = kRing + kSlots * kTileBytes;
   // barrier indices (8 bytes each)
   static constexpr int Q_FULL = 0, Q_EMPTY = 1, KV_FULL = 2, KV_EMPTY = 2 + kSlots, S_FULL = 2 + 2 * kSlots,
-                       P_READY = S_FULL + 4, O_DONE = P_READY + 4, EPI = O_DONE + 2, NBARS = EPI + 1;
+                       P_READY = S_FULL + 4, O_DONE = P_READY + 4, ITEM_DONE = O_DONE + 2, EPI = ITEM_DONE + 2,
+                       NBARS = EPI + 1;
   static constexpr int kMisc = kBars + NBARS * 8;          // tmem ptr, abort flag, last flag
   static constexpr int kCum = kMisc + 16;
   static constexpr int kTotal = kCum + (kMaxB + 1) * 4;
@@ -319,7 +320,10 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       mbar_init(bar(L::S_FULL + s), 1);
       mbar_init(bar(L::P_READY + s), 128);
     }
-    for (int s = 0; s < 2; ++s) mbar_init(bar(L::O_DONE + s), 1);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(bar(L::O_DONE + s), 1);
+      mbar_init(bar(L::ITEM_DONE + s), 1);
+    }
     mbar_init(bar(L::EPI), MT * 128);
     *abort_flag = ((sbase & 1023u) != 0) ? 1 : 0;   // swizzled tiles need a 1024-byte aligned base
     *last_flag = 0;
@@ -478,6 +482,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                           (jt > 0 || h > 0 || ks > 0) ? 1u : 0u);
             mma_commit(bar(L::O_DONE + t));
             if (h == 1) mma_commit(bar(L::KV_EMPTY + vslot));
+            if (h == 1 && jt + 1 == nt) mma_commit(bar(L::ITEM_DONE + t));   // all MMAs of the item are done
             if (jt + 1 < nt) {
               if (h == 0) {
                 ok = mbar_wait(bar(L::KV_FULL + kslot), (fk / kSlots) & 1, abort_flag);
@@ -508,7 +513,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     if (wg_active && !*abort_flag) {
       long long g = g_begin;
       Item it;
-      uint32_t fill = 0, hj = 0, epi_phase = 0;
+      uint32_t fill = 0, hj = 0, epi_phase = 0, item_cnt = 0;
       bool ok = true;
       Tracer tr;
       tr.init((threadIdx.x & 127) == 0 ? prm.trace : nullptr, 2 + wg);
@@ -574,6 +579,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             tmem_ld32(s_addr, sreg);
             tmem_ld32(s_addr + 32, sreg + 32);
             tmem_wait_ld();
+            tr.mark(0xA000u | (hj & 0xfffu));
             float* s = reinterpret_cast<float*>(sreg);
             if (valid_half < 64 || tree) {
 #pragma unroll
@@ -624,6 +630,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 tmem_st32(o_addr_loop + q * 32, o);
               }
             }
+            tr.mark(0xB000u | (hj & 0xfffu));
             // ---- P = exp2(s * c - m), row sum in fp32, P rounded to bf16 into TMEM over the start of S(h)
             const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
             float ls0 = 0.f, ls1 = 0.f;
@@ -646,6 +653,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                   : "memory");
             }
             l_sum += ls0 + ls1;
+            tr.mark(0xC000u | (hj & 0xfffu));
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bar(L::P_READY + wg * 2 + h));
@@ -656,9 +664,11 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         if (!ok) break;
         // ---- epilogue of the item: wait for the last PV into this O buffer
         {
-          // The item's last two PVs (both halves of the last key tile) may still be in flight.  A parity
-          // wait is only meaningful for a phase at most one ahead of the barrier, so take them in order.
-          ok = wwait(bar(L::O_DONE + wg), (hj - 2) & 1) && wwait(bar(L::O_DONE + wg), (hj - 1) & 1);
+          // Wait for every MMA of the item.  This barrier completes once per item, so its phase is never
+          // more than one away from the one waited for (a parity wait cannot tell phases two apart, which
+          // is why the per-PV barrier O_DONE is not used here: both last PVs may or may not be done yet).
+          ok = wwait(bar(L::ITEM_DONE + wg), item_cnt & 1);
+          ++item_cnt;
           if (!ok) break;
           tc_fence_after();
           tr.mark(0x5000u);
@@ -691,35 +701,15 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               *lse_p = (row_active && l_sum > 0.f) ? (m_used + log2f(l_sum)) / kLog2e : -INFINITY;
             tc_fence_before();
           } else {
-            // ---- a piece of a unit: leave (O, m, l) in this CTA's slot, then merge if every piece is in.
-            // Partial O is stored column-group major, [slot][D/4][MT*128 rows][4 floats], so that the 32 rows
-            // of a warp write (and later read) 512 contiguous bytes per instruction.
+            // ---- a piece of a unit.  The pieces of a unit draw tickets on the unit's "claimed" counter: the
+            // piece with the last ticket becomes the merger and keeps its O in TMEM; every other piece leaves
+            // (O, m, l) in its CTA's slot and then bumps the unit's "ready" counter.  The merger waits (bounded)
+            // until all other pieces are ready - they hold tickets, so they are running their epilogue - and
+            // folds them into its own accumulator.  Both counters carry the call's epoch, so the workspace
+            // needs no initialisation.  Partial O is stored column-group major,
+            // [slot][D/4][MT*128 rows][4 floats]: a warp writes and reads 512 contiguous bytes per instruction.
             constexpr int kRows = MT * 128;
             const int rr = wg * 128 + row;
-            const int slot_id = blockIdx.x * 2 + (it.j0 > 0 ? 0 : 1);
-            float* po = prm.part_o + (size_t)slot_id * (D / 4) * kRows * 4;
-            float* pml = prm.part_ml + (size_t)slot_id * 2 * kRows;
-#pragma unroll
-            for (int q = 0; q < D / 32; ++q) {
-              uint32_t o[32];
-              tmem_ld32(o_addr + q * 32, o);
-              tmem_wait_ld();
-              if (row_active) {
-#pragma unroll
-                for (int c = 0; c < 8; ++c)
-                  *reinterpret_cast<uint4*>(po + ((size_t)(q * 8 + c) * kRows + rr) * 4) =
-                      make_uint4(o[4 * c], o[4 * c + 1], o[4 * c + 2], o[4 * c + 3]);
-              }
-            }
-            if (row_active) {
-              pml[rr] = m_used;
-              pml[kRows + rr] = l_sum;
-            }
-            tc_fence_before();
-            __threadfence();
-            tr.mark(0x6000u);
-            ok = epi_sync();
-            if (!ok) break;
             // unit geometry in the linear tile space
             const long long u0 = (long long)prm.Hkv * cum[it.b] + (long long)it.hk * it.len;
             int k_first = (int)((u0 * prm.groups) / sch.total);
@@ -732,99 +722,209 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             int n_frag = 0;
             for (int k = k_first; k <= k_last; ++k)
               n_frag += sch.group_start(k + 1, prm.groups) > sch.group_start(k, prm.groups) ? 1 : 0;
-            if (threadIdx.x == 128) {
-              unsigned long long* ctr = prm.counters + ((size_t)it.b * prm.Hkv + it.hk) * prm.NP + pair;
-              unsigned long long seen = *reinterpret_cast<volatile unsigned long long*>(ctr), want;
-              int cnt;
-              do {
+            unsigned long long* ctr = prm.counters + (((size_t)it.b * prm.Hkv + it.hk) * prm.NP + pair) * 2;
+            // epoch-tagged increment: returns the count after this arrival
+            auto bump = [&](unsigned long long* c) -> int {
+              unsigned long long seen = *reinterpret_cast<volatile unsigned long long*>(c);
+              while (true) {
                 const unsigned long long assumed = seen;
-                cnt = ((assumed >> 16) == prm.epoch) ? (int)(assumed & 0xffffu) : 0;
-                want = (prm.epoch << 16) | (unsigned long long)(cnt + 1);
-                seen = atomicCAS(ctr, assumed, want);
-                if (seen == assumed) break;
-              } while (true);
-              *last_flag = (cnt + 1 == n_frag) ? 1 : 0;
-              __threadfence();
+                const int cnt = ((assumed >> 16) == prm.epoch) ? (int)(assumed & 0xffffu) : 0;
+                seen = atomicCAS(c, assumed, (prm.epoch << 16) | (unsigned long long)(cnt + 1));
+                if (seen == assumed) return cnt + 1;
+              }
+            };
+            if (threadIdx.x == 128) {
+              const int ticket = bump(ctr);
+              int merger = (ticket == n_frag) ? 1 : 0;
+              if (merger) {
+                // wait until the other n_frag - 1 pieces have published their partials
+                const unsigned long long t0 = globaltimer_ns();
+                while (true) {
+                  const unsigned long long v = *reinterpret_cast<volatile unsigned long long*>(ctr + 1);
+                  const int ready = ((v >> 16) == prm.epoch) ? (int)(v & 0xffffu) : 0;
+                  if (ready >= n_frag - 1) break;
+                  if (*abort_flag || globaltimer_ns() - t0 > kWaitLimitNs) {
+                    *abort_flag = 1;
+                    break;
+                  }
+                }
+                __threadfence();
+              }
+              *last_flag = merger;
             }
             ok = epi_sync();
-            if (!ok) break;
+            if (!ok || *abort_flag) { ok = false; break; }
             tr.mark(0x7000u | (*last_flag ? 1u : 0u));
-            if (*last_flag) {
-              if (row_exists) {
-                // pass 1: reference maximum and total weight of the row over all pieces
-                float mm = -INFINITY, lt = 0.f;
+            const int my_slot = blockIdx.x * 2 + (it.j0 > 0 ? 0 : 1);
+            if (!*last_flag) {
+              float* po = prm.part_o + (size_t)my_slot * (D / 4) * kRows * 4;
+              float* pml = prm.part_ml + (size_t)my_slot * 2 * kRows;
+#pragma unroll
+              for (int q = 0; q < D / 32; ++q) {
+                uint32_t o[32];
+                tmem_ld32(o_addr + q * 32, o);
+                tmem_wait_ld();
+                if (row_active) {
+#pragma unroll
+                  for (int c = 0; c < 8; ++c)
+                    *reinterpret_cast<uint4*>(po + ((size_t)(q * 8 + c) * kRows + rr) * 4) =
+                        make_uint4(o[4 * c], o[4 * c + 1], o[4 * c + 2], o[4 * c + 3]);
+                }
+              }
+              if (row_active) {
+                pml[rr] = m_used;
+                pml[kRows + rr] = l_sum;
+              }
+              tc_fence_before();
+              __threadfence();
+              tr.mark(0x6000u);
+              ok = epi_sync();
+              if (!ok) break;
+              if (threadIdx.x == 128) bump(ctr + 1);
+            } else {
+              // The sums below run over the pieces in their order inside the unit with one fused multiply-add
+              // per piece, whichever piece happens to be the merger: the result does not depend on timing.
+              float mm = m_used, lt = 0.f;
+              int n_other = 0, sid1 = 0, own_pos = 0;
+              for (int k = k_first; k <= k_last; ++k) {
+                const long long ks = sch.group_start(k, prm.groups);
+                if (sch.group_start(k + 1, prm.groups) <= ks) continue;
+                const int sid = (k * prm.NP + pair) * 2 + (ks > u0 ? 0 : 1);
+                if (sid == my_slot) {
+                  own_pos = n_other;         // number of other pieces that come before this one
+                  continue;
+                }
+                sid1 = sid;
+                ++n_other;
+              }
+              if (n_other == 1) {
+                // the usual case, one other piece: fetch its (m, l) and its O with as few dependent round
+                // trips to L2 as possible (everything of a batch is requested before anything is used).
+                // Loads are issued by every thread (row rr always lies inside the slot; rows that are not
+                // active read stale bytes and are masked by selects): no thread-divergent branch may sit
+                // between the warp-wide TMEM instructions below.
+                const float* q_ml = prm.part_ml + (size_t)sid1 * 2 * kRows;
+                const float* q_o = prm.part_o + (size_t)sid1 * (D / 4) * kRows * 4;
+                const float m1 = __ldcg(q_ml + rr);
+                const float l1 = __ldcg(q_ml + kRows + rr);
+                const bool own_first = own_pos == 0;
+                float w_own = 0.f, w1 = 0.f, inv = 0.f;
+#pragma unroll
+                for (int half = 0; half < D / 64; ++half) {
+                  float4 v[16];
+#pragma unroll
+                  for (int c = 0; c < 16; ++c)
+                    v[c] = __ldcg(reinterpret_cast<const float4*>(q_o + ((size_t)(half * 16 + c) * kRows + rr) * 4));
+                  if (half == 0) {
+                    mm = fmaxf(m_used, m1);
+                    w_own = row_active ? fast_exp2(m_used - mm) : 0.f;
+                    w1 = row_active ? fast_exp2(m1 - mm) : 0.f;
+                    lt = own_first ? fmaf(w1, l1, w_own * l_sum) : fmaf(w_own, l_sum, w1 * l1);
+                    inv = (row_active && lt > 0.f) ? 1.f / lt : 0.f;
+                  }
+#pragma unroll
+                  for (int q = 0; q < 2; ++q) {
+                    uint32_t o[32];
+                    tmem_ld32(o_addr + (half * 2 + q) * 32, o);
+                    tmem_wait_ld();
+                    if (row_exists) {
+#pragma unroll
+                      for (int c = 0; c < 4; ++c) {
+                        float r[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                          const float4 vv = v[q * 8 + c * 2 + e / 4];
+                          const float ve = (e % 4 == 0) ? vv.x : (e % 4 == 1) ? vv.y : (e % 4 == 2) ? vv.z : vv.w;
+                          const float oe = __uint_as_float(o[c * 8 + e]);
+                          const float sum = own_first ? fmaf(w1, ve, w_own * oe) : fmaf(w_own, oe, w1 * ve);
+                          r[e] = row_active ? sum * inv : 0.f;
+                        }
+                        uint4 pk;
+                        pk.x = pack_bf16(r[0], r[1]);
+                        pk.y = pack_bf16(r[2], r[3]);
+                        pk.z = pack_bf16(r[4], r[5]);
+                        pk.w = pack_bf16(r[6], r[7]);
+                        *reinterpret_cast<uint4*>(orow + (half * 2 + q) * 32 + c * 8) = pk;
+                      }
+                    }
+                  }
+                }
+              } else {
+                // ---- any number of pieces: pass 1, reference maximum and total weight of the row
                 if (row_active) {
                   for (int k = k_first; k <= k_last; ++k) {
                     const long long ks = sch.group_start(k, prm.groups);
                     if (sch.group_start(k + 1, prm.groups) <= ks) continue;
                     const int sid = (k * prm.NP + pair) * 2 + (ks > u0 ? 0 : 1);
+                    if (sid == my_slot) continue;
                     mm = fmaxf(mm, __ldcg(prm.part_ml + (size_t)sid * 2 * kRows + rr));
                   }
                   for (int k = k_first; k <= k_last; ++k) {
                     const long long ks = sch.group_start(k, prm.groups);
                     if (sch.group_start(k + 1, prm.groups) <= ks) continue;
                     const int sid = (k * prm.NP + pair) * 2 + (ks > u0 ? 0 : 1);
-                    const float* q_ml = prm.part_ml + (size_t)sid * 2 * kRows;
-                    lt += fast_exp2(__ldcg(q_ml + rr) - mm) * __ldcg(q_ml + kRows + rr);
+                    if (sid == my_slot) {
+                      lt = fmaf(fast_exp2(m_used - mm), l_sum, lt);
+                    } else {
+                      const float* q_ml = prm.part_ml + (size_t)sid * 2 * kRows;
+                      lt = fmaf(fast_exp2(__ldcg(q_ml + rr) - mm), __ldcg(q_ml + kRows + rr), lt);
+                    }
                   }
                 }
                 const float inv = (row_active && lt > 0.f) ? 1.f / lt : 0.f;
-                // pass 2: 32 output columns at a time, every piece weighted by exp2(m_piece - mm); the loads
-                // of two pieces are issued together to cover the L2 latency
+                const float w_own = row_active ? fast_exp2(m_used - mm) : 0.f;
+                // ---- pass 2: 32 output columns at a time, pieces in order; the own piece comes from TMEM
 #pragma unroll 1
                 for (int q = 0; q < D / 32; ++q) {
+                  uint32_t o[32];
+                  tmem_ld32(o_addr + q * 32, o);
+                  tmem_wait_ld();
                   float acc[32];
 #pragma unroll
                   for (int c = 0; c < 32; ++c) acc[c] = 0.f;
                   if (row_active) {
-                    int k = k_first;
-                    while (k <= k_last) {
-                      int sid[2];
-                      int got = 0;
-                      for (; k <= k_last && got < 2; ++k) {
-                        const long long ks = sch.group_start(k, prm.groups);
-                        if (sch.group_start(k + 1, prm.groups) <= ks) continue;
-                        sid[got++] = (k * prm.NP + pair) * 2 + (ks > u0 ? 0 : 1);
+                    for (int k = k_first; k <= k_last; ++k) {
+                      const long long ks = sch.group_start(k, prm.groups);
+                      if (sch.group_start(k + 1, prm.groups) <= ks) continue;
+                      const int sid = (k * prm.NP + pair) * 2 + (ks > u0 ? 0 : 1);
+                      if (sid == my_slot) {
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) acc[c] = fmaf(w_own, __uint_as_float(o[c]), acc[c]);
+                        continue;
                       }
-                      if (got == 1) sid[1] = sid[0];
-                      float w[2];
-                      float4 v[2][8];
+                      const float w = fast_exp2(__ldcg(prm.part_ml + (size_t)sid * 2 * kRows + rr) - mm);
+                      const float* q_o = prm.part_o + (size_t)sid * (D / 4) * kRows * 4;
+                      float4 v[8];
 #pragma unroll
-                      for (int f = 0; f < 2; ++f) {
-                        w[f] = fast_exp2(__ldcg(prm.part_ml + (size_t)sid[f] * 2 * kRows + rr) - mm);
-                        const float* q_o = prm.part_o + (size_t)sid[f] * (D / 4) * kRows * 4;
+                      for (int c = 0; c < 8; ++c)
+                        v[c] = __ldcg(reinterpret_cast<const float4*>(q_o + ((size_t)(q * 8 + c) * kRows + rr) * 4));
 #pragma unroll
-                        for (int c = 0; c < 8; ++c)
-                          v[f][c] = __ldcg(reinterpret_cast<const float4*>(q_o + ((size_t)(q * 8 + c) * kRows + rr) * 4));
+                      for (int c = 0; c < 8; ++c) {
+                        acc[4 * c] = fmaf(w, v[c].x, acc[4 * c]);
+                        acc[4 * c + 1] = fmaf(w, v[c].y, acc[4 * c + 1]);
+                        acc[4 * c + 2] = fmaf(w, v[c].z, acc[4 * c + 2]);
+                        acc[4 * c + 3] = fmaf(w, v[c].w, acc[4 * c + 3]);
                       }
-                      if (got == 1) w[1] = 0.f;
-                      if (got == 0) w[0] = 0.f;
-#pragma unroll
-                      for (int f = 0; f < 2; ++f)
-#pragma unroll
-                        for (int c = 0; c < 8; ++c) {
-                          acc[4 * c] = fmaf(w[f], v[f][c].x, acc[4 * c]);
-                          acc[4 * c + 1] = fmaf(w[f], v[f][c].y, acc[4 * c + 1]);
-                          acc[4 * c + 2] = fmaf(w[f], v[f][c].z, acc[4 * c + 2]);
-                          acc[4 * c + 3] = fmaf(w[f], v[f][c].w, acc[4 * c + 3]);
-                        }
                     }
                   }
+                  if (row_exists) {
 #pragma unroll
-                  for (int c = 0; c < 4; ++c) {
-                    uint4 v;
-                    v.x = pack_bf16(acc[8 * c + 0] * inv, acc[8 * c + 1] * inv);
-                    v.y = pack_bf16(acc[8 * c + 2] * inv, acc[8 * c + 3] * inv);
-                    v.z = pack_bf16(acc[8 * c + 4] * inv, acc[8 * c + 5] * inv);
-                    v.w = pack_bf16(acc[8 * c + 6] * inv, acc[8 * c + 7] * inv);
-                    *reinterpret_cast<uint4*>(orow + q * 32 + c * 8) = v;
+                    for (int c = 0; c < 4; ++c) {
+                      uint4 v;
+                      v.x = pack_bf16(acc[8 * c + 0] * inv, acc[8 * c + 1] * inv);
+                      v.y = pack_bf16(acc[8 * c + 2] * inv, acc[8 * c + 3] * inv);
+                      v.z = pack_bf16(acc[8 * c + 4] * inv, acc[8 * c + 5] * inv);
+                      v.w = pack_bf16(acc[8 * c + 6] * inv, acc[8 * c + 7] * inv);
+                      *reinterpret_cast<uint4*>(orow + q * 32 + c * 8) = v;
+                    }
                   }
                 }
-                if (lse_p) *lse_p = (row_active && lt > 0.f) ? (mm + log2f(lt)) / kLog2e : -INFINITY;
               }
+              if (row_exists && lse_p) *lse_p = (row_active && lt > 0.f) ? (mm + log2f(lt)) / kLog2e : -INFINITY;
+              tc_fence_before();
+              ok = epi_sync();   // keeps the two warpgroups' barrier phases in step with the other branch
+              if (!ok) break;
             }
-            ok = epi_sync();   // last_flag may be rewritten by the next item only after everyone read it
-            if (!ok) break;
           }
         }
         tr.mark(0x8000u);
@@ -908,7 +1008,7 @@ Geometry geometry(int B, int Nmax, int Hq, int Hkv, int d, bool query_device) {
   // workspace: counters, then (m,l) pairs, then partial O, sized for 160 SMs so the size does not depend on the device
   const size_t max_ctas = 160 > g.grid ? 160 : g.grid;
   g.counters_off = 0;
-  size_t off = (size_t)B * Hkv * g.NP * sizeof(unsigned long long);
+  size_t off = (size_t)B * Hkv * g.NP * 2 * sizeof(unsigned long long);
   off = (off + 255) & ~size_t(255);
   g.ml_off = off;
   off += max_ctas * 2 * (size_t)g.MT * 128 * 2 * sizeof(float);

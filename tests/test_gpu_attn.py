@@ -186,6 +186,32 @@ def test_chain_tree_is_causal_attention_and_one_node_is_decode():
         assert err <= ATTN_ATOL
 
 
+def test_repeated_launches_are_bit_reproducible_and_never_time_out():
+    """Units cut between CTAs are merged by whichever piece finishes last; the result must not depend on
+    that order, and the bounded waits must never expire (they once did when a wait could lag two barrier
+    phases behind)."""
+    cfg = CONFIGS[4].scaled(L=1, V=0)
+    dcase = make_case(cfg, seed=4001, device="cuda", with_logits=False)
+    B, N = cfg.B, cfg.N
+    bits = torch.zeros(B, N, (N + 31) // 32, dtype=torch.int32, device="cuda")
+    status = torch.zeros(B, dtype=torch.int32, device="cuda")
+    tv.tree_build_mask(dcase["parent"], dcase["n_nodes"], N - 1, 1, bits, status)
+    ws = torch.zeros(tv.tv_attn_workspace_bytes(B, N, cfg.Hq, cfg.Hkv, cfg.d, cfg.Scap), dtype=torch.uint8, device="cuda")
+    first = None
+    for it in range(60):
+        out = torch.zeros(B, N, cfg.Hq, cfg.d, dtype=torch.bfloat16, device="cuda")
+        lse = torch.zeros(B, cfg.Hq, N, dtype=torch.float32, device="cuda")
+        tv.tree_verify_attn(dcase["q"][0], dcase["k_cache"][0], dcase["v_cache"][0], dcase["k_tree"][0],
+                            dcase["v_tree"][0], dcase["prefix_len"], dcase["n_nodes"], bits, cfg.d ** -0.5, out,
+                            ws, status, lse=lse)
+        torch.cuda.synchronize()
+        assert (status == 0).all(), f"launch {it}: status {status.cpu().tolist()}"
+        if first is None:
+            first = (out, lse)
+        else:
+            assert torch.equal(out, first[0]) and torch.equal(lse, first[1]), f"launch {it} differs from launch 0"
+
+
 FULL = [(1, [(0, 0), (0, 17), (0, 31)]), (2, [(0, 0), (3, 5), (7, 7)]), (3, [(0, 0), (3, 7)]),
         (4, [(0, 0), (9, 3), (15, 7)])]
 
