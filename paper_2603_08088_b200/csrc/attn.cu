@@ -45,6 +45,8 @@ constexpr int kThreads = 384;
 constexpr int kMaxB = 512;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kRescaleThreshold = 8.0f;            // in log2 units
+constexpr float kMaxFastP = 256.0f;                  // 2^threshold: largest P the fast path accepts
+constexpr int kPolyPairsOf8 = 3;                     // of every 8 element pairs, how many take 2^x on the FMA pipe
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 constexpr int kTraceCap = 256;     // events per (CTA, role) kept by the optional trace
 
@@ -208,6 +210,27 @@ struct Tracer {
     if (base && n < kTraceCap) base[n++] = ((unsigned long long)tag << 48) | (globaltimer_ns() & 0xffffffffffffull);
   }
 };
+
+// Packed fp32 pair arithmetic (one issue slot for two lanes of work).
+__device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) { return __ffma2_rn(a, b, c); }
+__device__ __forceinline__ float2 fadd2(float2 a, float2 b) { return __fadd2_rn(a, b); }
+// 2^x for a pair on the FMA pipe (the special-function unit is the scarce resource of the softmax):
+// x = n + f with n = round(x), f in [-0.5, 0.5]; 2^f by a cubic (relative error 7.5e-5, far below the
+// bf16 rounding of P), 2^n by an add into the exponent field.  x is clamped to [-125, 16].
+__device__ __forceinline__ float2 exp2_poly2(float2 x) {
+  x.x = fminf(fmaxf(x.x, -125.f), 16.f);
+  x.y = fminf(fmaxf(x.y, -125.f), 16.f);
+  const float2 t = fadd2(x, make_float2(12582912.f, 12582912.f));          // 1.5 * 2^23: low mantissa bits = n
+  const float2 n = fadd2(t, make_float2(-12582912.f, -12582912.f));
+  const float2 f = ffma2(n, make_float2(-1.f, -1.f), x);
+  float2 p = ffma2(f, make_float2(0.0551716685f, 0.0551716685f), make_float2(0.2426111251f, 0.2426111251f));
+  p = ffma2(p, f, make_float2(0.6932609677f, 0.6932609677f));
+  p = ffma2(p, f, make_float2(0.9999280572f, 0.9999280572f));
+  float2 r;
+  r.x = __int_as_float(__float_as_int(p.x) + (__float_as_int(t.x) << 23));
+  r.y = __int_as_float(__float_as_int(p.y) + (__float_as_int(t.y) << 23));
+  return r;
+}
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t r;
@@ -579,7 +602,6 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             tmem_ld32(s_addr, sreg);
             tmem_ld32(s_addr + 32, sreg + 32);
             tmem_wait_ld();
-            tr.mark(0xA000u | (hj & 0xfffu));
             float* s = reinterpret_cast<float*>(sreg);
             if (valid_half < 64 || tree) {
 #pragma unroll
@@ -596,64 +618,95 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                   if (!((word >> c) & 1u)) s[q * 32 + c] = -INFINITY;
               }
             }
-            float mx0 = s[0], mx1 = s[1], mx2_ = s[2], mx3 = s[3];
-#pragma unroll
-            for (int c = 4; c < 64; c += 4) {
-              mx0 = fmaxf(mx0, s[c]);
-              mx1 = fmaxf(mx1, s[c + 1]);
-              mx2_ = fmaxf(mx2_, s[c + 2]);
-              mx3 = fmaxf(mx3, s[c + 3]);
-            }
-            const float mx2 = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2_, mx3)) * prm.scale_log2e;
-            // ---- lazy rescale: move the reference maximum only when it would grow by more than the
-            // threshold.  The TMEM accesses are warp-wide (.sync.aligned), so the warp rescales as soon as
-            // one of its rows has to; rows that keep their maximum multiply by 1.
+            uint32_t pk[32];                 // P of this half, bf16 pairs
             const bool first = (jt == 0 && h == 0);
-            const bool moves = (mx2 > m_used + kRescaleThreshold || m_used == -INFINITY) && mx2 > -INFINITY;
-            const bool scales = moves && !first && m_used > -INFINITY;
-            const float alpha = scales ? fast_exp2(m_used - mx2) : 1.f;
-            if (moves) m_used = mx2;
-            l_sum *= alpha;
-            if (__any_sync(0xffffffffu, scales)) {
-              tr.mark(0x9000u | (hj & 0xfffu));
-              // the PV of the previous half may still be running: wait for its completion (number hj - 1)
-              ok = wwait(bar(L::O_DONE + wg), (hj - 1) & 1);
-              if (!ok) break;
-              tc_fence_after();
+            bool need_slow = true;
+            // ---- fast path (full, unmasked halves after the first): keep the reference maximum, compute
+            // P directly and only check afterwards that nothing overflowed the lazy-rescale range.
+            if (!first && !tree && valid_half == 64) {
+              const float2 c2 = make_float2(prm.scale_log2e, prm.scale_log2e);
+              const float nm = (m_used == -INFINITY) ? 0.f : -m_used;
+              const float2 nm2 = make_float2(nm, nm);
+              float2 sum = make_float2(0.f, 0.f);
 #pragma unroll
-              for (int q = 0; q < D / 32; ++q) {
-                uint32_t o[32];
-                tmem_ld32(o_addr_loop + q * 32, o);
-                tmem_wait_ld();
+              for (int i = 0; i < 32; ++i) {
+                const float2 x = ffma2(make_float2(s[2 * i], s[2 * i + 1]), c2, nm2);
+                float2 pv;
+                if ((i & 7) < kPolyPairsOf8) {
+                  pv = exp2_poly2(x);
+                } else {
+                  pv.x = fast_exp2(x.x);
+                  pv.y = fast_exp2(x.y);
+                }
+                sum = fadd2(sum, pv);
+                pk[i] = pack_bf16(pv.x, pv.y);
+              }
+              // largest P of the row from the packed bf16 pairs (all values are >= 0)
+              __nv_bfloat162 mxp = *reinterpret_cast<__nv_bfloat162*>(&pk[0]);
 #pragma unroll
-                for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
-                tmem_st32(o_addr_loop + q * 32, o);
+              for (int i = 1; i < 32; ++i) mxp = __hmax2_nan(mxp, *reinterpret_cast<__nv_bfloat162*>(&pk[i]));
+              const float pmax = fmaxf(__low2float(mxp), __high2float(mxp));
+              const bool overflow = row_active && !(pmax <= kMaxFastP);      // NaN counts as overflow
+              if (!__any_sync(0xffffffffu, overflow)) {
+                l_sum += sum.x + sum.y;
+                need_slow = false;
               }
             }
-            tr.mark(0xB000u | (hj & 0xfffu));
-            // ---- P = exp2(s * c - m), row sum in fp32, P rounded to bf16 into TMEM over the start of S(h)
-            const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
-            float ls0 = 0.f, ls1 = 0.f;
+            if (need_slow) {
+              float mx0 = s[0], mx1 = s[1], mx2_ = s[2], mx3 = s[3];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              uint32_t pk[8];
+              for (int c = 4; c < 64; c += 4) {
+                mx0 = fmaxf(mx0, s[c]);
+                mx1 = fmaxf(mx1, s[c + 1]);
+                mx2_ = fmaxf(mx2_, s[c + 2]);
+                mx3 = fmaxf(mx3, s[c + 3]);
+              }
+              const float mx2 = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2_, mx3)) * prm.scale_log2e;
+              // ---- lazy rescale: move the reference maximum only when it would grow by more than the
+              // threshold.  The TMEM accesses are warp-wide (.sync.aligned), so the warp rescales as soon as
+              // one of its rows has to; rows that keep their maximum multiply by 1.
+              const bool moves = (mx2 > m_used + kRescaleThreshold || m_used == -INFINITY) && mx2 > -INFINITY;
+              const bool scales = moves && !first && m_used > -INFINITY;
+              const float alpha = scales ? fast_exp2(m_used - mx2) : 1.f;
+              if (moves) m_used = mx2;
+              l_sum *= alpha;
+              if (__any_sync(0xffffffffu, scales)) {
+                tr.mark(0x9000u | (hj & 0xfffu));
+                // the PV of the previous half may still be running: wait for its completion (number hj - 1)
+                ok = wwait(bar(L::O_DONE + wg), (hj - 1) & 1);
+                if (!ok) break;
+                tc_fence_after();
 #pragma unroll
-              for (int c = 0; c < 8; ++c) {
-                const float p0 = fast_exp2(fmaf(s[q * 16 + 2 * c], prm.scale_log2e, neg_m));
-                const float p1 = fast_exp2(fmaf(s[q * 16 + 2 * c + 1], prm.scale_log2e, neg_m));
+                for (int q = 0; q < D / 32; ++q) {
+                  uint32_t o[32];
+                  tmem_ld32(o_addr_loop + q * 32, o);
+                  tmem_wait_ld();
+#pragma unroll
+                  for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+                  tmem_st32(o_addr_loop + q * 32, o);
+                }
+              }
+              // ---- P = exp2(s * c - m), row sum in fp32, P rounded to bf16
+              const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
+              float ls0 = 0.f, ls1 = 0.f;
+#pragma unroll
+              for (int i = 0; i < 32; ++i) {
+                const float p0 = fast_exp2(fmaf(s[2 * i], prm.scale_log2e, neg_m));
+                const float p1 = fast_exp2(fmaf(s[2 * i + 1], prm.scale_log2e, neg_m));
                 ls0 += p0;
                 ls1 += p1;
-                pk[c] = pack_bf16(p0, p1);
+                pk[i] = pack_bf16(p0, p1);
               }
-              // 16 keys = 8 packed columns
+              l_sum += ls0 + ls1;
+            }
+            // ---- P into TMEM over the start of S(h): 16 keys = 8 packed columns per store
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
               asm volatile(
                   "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
-                  ::"r"(s_addr + q * 8), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]),
-                    "r"(pk[6]), "r"(pk[7])
+                  ::"r"(s_addr + q * 8), "r"(pk[q * 8 + 0]), "r"(pk[q * 8 + 1]), "r"(pk[q * 8 + 2]), "r"(pk[q * 8 + 3]),
+                    "r"(pk[q * 8 + 4]), "r"(pk[q * 8 + 5]), "r"(pk[q * 8 + 6]), "r"(pk[q * 8 + 7])
                   : "memory");
-            }
-            l_sum += ls0 + ls1;
-            tr.mark(0xC000u | (hj & 0xfffu));
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bar(L::P_READY + wg * 2 + h));
