@@ -46,8 +46,14 @@ constexpr int kMaxB = 512;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kRescaleThreshold = 8.0f;            // in log2 units
 constexpr float kMaxFastP = 256.0f;                  // 2^threshold: largest P the fast path accepts
-constexpr int kPolyPairsOf8 = 3;                     // of every 8 element pairs, how many take 2^x on the FMA pipe
+// Of every 8 element pairs of the softmax fast path, one takes 2^x on the FMA pipe (measured optimum between
+// the special-function unit and the FMA pipe on the long-context shape).
+#ifndef TV_POLY_SEL
+#define TV_POLY_SEL(i) (((i) & 7) == 3)
+#endif
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+constexpr int kSetupCost = 4;      // virtual tiles charged per unit by the scheduler
+constexpr int kMaxGroups = 160;
 constexpr int kTraceCap = 256;     // events per (CTA, role) kept by the optional trace
 
 // ---------------------------------------------------------------- PTX helpers
@@ -262,11 +268,24 @@ struct Item {
 };
 
 // Shared bookkeeping of the linear tile space: cum[b] = sum of len over b' < b, len_b = ceil(S_b/128) + 1.
+// The schedule works in a "virtual" tile space: every (sequence, KV head) unit is charged kSetupCost
+// virtual tiles in front of its real key tiles, the price of starting a unit (Q load, pipeline refill,
+// epilogue).  Cutting that space evenly gives CTAs that start more units fewer real tiles, and a cut that
+// falls into a unit's setup region snaps to the unit boundary, which saves a split.
 struct Sched {
-  const int* cum;
+  const int* cum;    // cum[b] = sum over b' < b of (len_b' + kSetupCost)
+  const int* gs;     // gs[k] = first virtual tile of CTA group k, gs[groups] = total
   int B, Hkv;
   long long total;   // Hkv * cum[B]
-  __device__ __forceinline__ long long group_start(int k, int groups) const { return (total * k) / groups; }
+  __device__ __forceinline__ long long group_start(int k, int) const { return gs[k]; }
+  __device__ __forceinline__ int find_group(long long pos, int groups) const {
+    int lo = 0, hi = groups - 1;   // largest k with gs[k] <= pos
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) >> 1;
+      if (gs[mid] <= pos) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+  }
   __device__ __forceinline__ int find_b(long long g) const {
     int lo = 0, hi = B - 1;   // largest b with Hkv*cum[b] <= g
     while (lo < hi) {
@@ -290,7 +309,8 @@ struct SmemLayout {
                        NBARS = EPI + 1;
   static constexpr int kMisc = kBars + NBARS * 8;          // tmem ptr, abort flag, last flag
   static constexpr int kCum = kMisc + 16;
-  static constexpr int kTotal = kCum + (kMaxB + 1) * 4;
+  static constexpr int kGs = kCum + (kMaxB + 1) * 4;
+  static constexpr int kTotal = kGs + (kMaxGroups + 1) * 4;
 };
 
 // ---------------------------------------------------------------- the kernel
@@ -309,8 +329,16 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   volatile int* last_flag = reinterpret_cast<volatile int*>(smem + L::kMisc + 8);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + L::kMisc);
   int* cum = reinterpret_cast<int*>(smem + L::kCum);
+  int* gs = reinterpret_cast<int*>(smem + L::kGs);
 
   // ---- setup: schedule table, barriers, TMEM
+  if (threadIdx.x == 64) {     // fetch the five TMA descriptors while the rest of the set-up runs
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_q) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_kc) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_vc) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_kt) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_vt) : "memory");
+  }
   if (warp == 0) {
     int run = 0;
     for (int base = 0; base < prm.B; base += 32) {
@@ -319,7 +347,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       if (b < prm.B) {
         int S = prm.prefix_len[b];
         S = S < 0 ? 0 : (S > prm.Scap ? prm.Scap : S);
-        len = (S + kTileN - 1) / kTileN + 1;
+        len = (S + kTileN - 1) / kTileN + 1 + kSetupCost;
       }
       int inc = len;
 #pragma unroll
@@ -361,8 +389,13 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  {
+    const long long total = (long long)prm.Hkv * cum[prm.B];
+    for (int k = threadIdx.x; k <= prm.groups; k += kThreads) gs[k] = (int)((total * k) / prm.groups);
+  }
+  __syncthreads();
 
-  Sched sch{cum, prm.B, prm.Hkv, (long long)prm.Hkv * cum[prm.B]};
+  Sched sch{cum, gs, prm.B, prm.Hkv, (long long)prm.Hkv * cum[prm.B]};
   const int group = blockIdx.x / prm.NP;
   const int pair = blockIdx.x % prm.NP;
   const long long g_begin = sch.group_start(group, prm.groups);
@@ -370,22 +403,30 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 
   // Walks the items of this CTA's range; identical in every role.
   auto next_item = [&](long long& g, Item& it) -> bool {
-    if (g >= g_end) return false;
-    const int b = sch.find_b(g);
-    const int len = cum[b + 1] - cum[b];
-    const long long local = g - (long long)prm.Hkv * cum[b];
-    it.b = b;
-    it.hk = (int)(local / len);
-    it.j0 = (int)(local % len);
-    const long long room = g_end - g;
-    it.j1 = (int)((long long)(len - it.j0) < room ? len : it.j0 + room);
-    it.len = len;
-    int S = prm.prefix_len[b];
-    it.S = S < 0 ? 0 : (S > prm.Scap ? prm.Scap : S);
-    int n = prm.n_nodes[b];
-    it.n = n < 0 ? 0 : (n > prm.Nmax ? prm.Nmax : n);
-    g += it.j1 - it.j0;
-    return true;
+    while (g < g_end) {
+      const int b = sch.find_b(g);
+      const int lenv = cum[b + 1] - cum[b];                       // setup region + real tiles
+      const long long local = g - (long long)prm.Hkv * cum[b];
+      const int hk = (int)(local / lenv);
+      const int r0 = (int)(local % lenv);
+      const long long room = g_end - g;
+      const int r1 = (long long)(lenv - r0) < room ? lenv : (int)(r0 + room);
+      g += r1 - r0;
+      const int j0 = r0 > kSetupCost ? r0 - kSetupCost : 0;
+      const int j1 = r1 > kSetupCost ? r1 - kSetupCost : 0;
+      if (j1 <= j0) continue;                                     // only setup tiles of this unit fall in the range
+      it.b = b;
+      it.hk = hk;
+      it.j0 = j0;
+      it.j1 = j1;
+      it.len = lenv - kSetupCost;
+      int S = prm.prefix_len[b];
+      it.S = S < 0 ? 0 : (S > prm.Scap ? prm.Scap : S);
+      int n = prm.n_nodes[b];
+      it.n = n < 0 ? 0 : (n > prm.Nmax ? prm.Nmax : n);
+      return true;
+    }
+    return false;
   };
 
   constexpr uint32_t kIdescQK = instr_desc(64, false);   // S is produced 64 keys at a time
@@ -420,6 +461,10 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 #pragma unroll
           for (int kv = 0; kv < 2; ++kv) {
             const uint32_t slot = fill % kSlots, round = fill / kSlots;
+            // At kernel start every CTA asks for its whole ring at once; let Q and the first K/V tile land
+            // before queueing the rest, so that the first MMA can start a few microseconds earlier.
+            if (item_idx == 1 && fill == 2) ok = mbar_wait(bar(L::Q_FULL), 0, abort_flag);
+            if (!ok) break;
             ok = mbar_wait(bar(L::KV_EMPTY + slot), (round & 1) ^ 1, abort_flag);
             if (!ok) break;
             tr.mark(0x2000u | (fill & 0xfffu));
@@ -632,7 +677,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               for (int i = 0; i < 32; ++i) {
                 const float2 x = ffma2(make_float2(s[2 * i], s[2 * i + 1]), c2, nm2);
                 float2 pv;
-                if ((i & 7) < kPolyPairsOf8) {
+                if (TV_POLY_SEL(i)) {
                   pv = exp2_poly2(x);
                 } else {
                   pv.x = fast_exp2(x.x);
@@ -763,18 +808,20 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             // [slot][D/4][MT*128 rows][4 floats]: a warp writes and reads 512 contiguous bytes per instruction.
             constexpr int kRows = MT * 128;
             const int rr = wg * 128 + row;
-            // unit geometry in the linear tile space
-            const long long u0 = (long long)prm.Hkv * cum[it.b] + (long long)it.hk * it.len;
-            int k_first = (int)((u0 * prm.groups) / sch.total);
-            while (k_first + 1 < prm.groups && sch.group_start(k_first + 1, prm.groups) <= u0) ++k_first;
-            while (k_first > 0 && sch.group_start(k_first, prm.groups) > u0) --k_first;
-            const long long u_last = u0 + it.len - 1;
-            int k_last = (int)((u_last * prm.groups) / sch.total);
-            while (k_last + 1 < prm.groups && sch.group_start(k_last + 1, prm.groups) <= u_last) ++k_last;
-            while (k_last > 0 && sch.group_start(k_last, prm.groups) > u_last) --k_last;
+            // unit geometry in the virtual tile space: real tiles occupy [real0, uend)
+            const long long real0 = (long long)prm.Hkv * cum[it.b] + (long long)it.hk * (it.len + kSetupCost) + kSetupCost;
+            const long long uend = real0 + it.len;
+            const int k_first = sch.find_group(real0, prm.groups);
+            const int k_last = sch.find_group(uend - 1, prm.groups);
+            // slot of the piece CTA group k holds of this unit, or -1 if it holds none
+            auto piece_slot = [&](int k) -> int {
+              const long long ks = gs[k], ke = gs[k + 1];
+              const long long lo = ks > real0 ? ks : real0, hi = ke < uend ? ke : uend;
+              if (lo >= hi) return -1;
+              return (k * prm.NP + pair) * 2 + (ks > real0 ? 0 : 1);
+            };
             int n_frag = 0;
-            for (int k = k_first; k <= k_last; ++k)
-              n_frag += sch.group_start(k + 1, prm.groups) > sch.group_start(k, prm.groups) ? 1 : 0;
+            for (int k = k_first; k <= k_last; ++k) n_frag += piece_slot(k) >= 0 ? 1 : 0;
             unsigned long long* ctr = prm.counters + (((size_t)it.b * prm.Hkv + it.hk) * prm.NP + pair) * 2;
             // epoch-tagged increment: returns the count after this arrival
             auto bump = [&](unsigned long long* c) -> int {
@@ -840,9 +887,8 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               float mm = m_used, lt = 0.f;
               int n_other = 0, sid1 = 0, own_pos = 0;
               for (int k = k_first; k <= k_last; ++k) {
-                const long long ks = sch.group_start(k, prm.groups);
-                if (sch.group_start(k + 1, prm.groups) <= ks) continue;
-                const int sid = (k * prm.NP + pair) * 2 + (ks > u0 ? 0 : 1);
+                const int sid = piece_slot(k);
+                if (sid < 0) continue;
                 if (sid == my_slot) {
                   own_pos = n_other;         // number of other pieces that come before this one
                   continue;
@@ -906,16 +952,14 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 // ---- any number of pieces: pass 1, reference maximum and total weight of the row
                 if (row_active) {
                   for (int k = k_first; k <= k_last; ++k) {
-                    const long long ks = sch.group_start(k, prm.groups);
-                    if (sch.group_start(k + 1, prm.groups) <= ks) continue;
-                    const int sid = (k * prm.NP + pair) * 2 + (ks > u0 ? 0 : 1);
+                    const int sid = piece_slot(k);
+                    if (sid < 0) continue;
                     if (sid == my_slot) continue;
                     mm = fmaxf(mm, __ldcg(prm.part_ml + (size_t)sid * 2 * kRows + rr));
                   }
                   for (int k = k_first; k <= k_last; ++k) {
-                    const long long ks = sch.group_start(k, prm.groups);
-                    if (sch.group_start(k + 1, prm.groups) <= ks) continue;
-                    const int sid = (k * prm.NP + pair) * 2 + (ks > u0 ? 0 : 1);
+                    const int sid = piece_slot(k);
+                    if (sid < 0) continue;
                     if (sid == my_slot) {
                       lt = fmaf(fast_exp2(m_used - mm), l_sum, lt);
                     } else {
@@ -937,9 +981,8 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                   for (int c = 0; c < 32; ++c) acc[c] = 0.f;
                   if (row_active) {
                     for (int k = k_first; k <= k_last; ++k) {
-                      const long long ks = sch.group_start(k, prm.groups);
-                      if (sch.group_start(k + 1, prm.groups) <= ks) continue;
-                      const int sid = (k * prm.NP + pair) * 2 + (ks > u0 ? 0 : 1);
+                      const int sid = piece_slot(k);
+                      if (sid < 0) continue;
                       if (sid == my_slot) {
 #pragma unroll
                         for (int c = 0; c < 32; ++c) acc[c] = fmaf(w_own, __uint_as_float(o[c]), acc[c]);
@@ -1133,6 +1176,8 @@ extern "C" int tree_verify_attn(const tv_bf16* q,
   TV_REQUIRE((reinterpret_cast<uintptr_t>(workspace) & 255u) == 0, "tree_verify_attn: workspace must be 256-byte aligned");
   if (B == 0) return TV_OK;
   const Geometry g = geometry(B, Nmax, Hq, Hkv, d, true);
+  TV_REQUIRE((long long)B * Hkv * ((Scap + kTileN - 1) / kTileN + 1 + kSetupCost) < (1ll << 31),
+             "tree_verify_attn: B * Hkv * Scap is too large for the tile scheduler");
   if (g.grid > 160) return tv::fail(TV_ERR_INVALID_ARG, "tree_verify_attn: device with more than 160 SMs is not supported");
   if (workspace_bytes < g.total)
     return tv::fail(TV_ERR_WORKSPACE, "tree_verify_attn: workspace of %zu bytes, need %zu", workspace_bytes, g.total);
