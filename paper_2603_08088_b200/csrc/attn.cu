@@ -54,6 +54,7 @@ constexpr float kMaxFastP = 256.0f;                  // 2^threshold: largest P t
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 constexpr int kSetupCost = 4;      // virtual tiles charged per unit by the scheduler
 constexpr int kMaxGroups = 160;
+constexpr int kMinVirtualTilesPerGroup = 12;   // do not spread a small problem over more CTA groups than this allows
 constexpr int kTraceCap = 256;     // events per (CTA, role) kept by the optional trace
 
 // ---------------------------------------------------------------- PTX helpers
@@ -244,6 +245,18 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return r;
 }
 
+// Epoch-tagged arrival counter: value = (epoch << 16) | count; a value with another epoch counts as zero, so
+// the counters need no initialisation.  `seen` is a value of the counter read earlier.  Returns the count
+// after this arrival.
+__device__ __forceinline__ int bump_counter(unsigned long long* c, unsigned long long seen, unsigned long long epoch) {
+  while (true) {
+    const unsigned long long assumed = seen;
+    const int cnt = ((assumed >> 16) == epoch) ? (int)(assumed & 0xffffu) : 0;
+    seen = atomicCAS(c, assumed, (epoch << 16) | (unsigned long long)(cnt + 1));
+    if (seen == assumed) return cnt + 1;
+  }
+}
+
 // ---------------------------------------------------------------- kernel parameters
 struct AttnParams {
   const int32_t* prefix_len;
@@ -252,7 +265,7 @@ struct AttnParams {
   tv_bf16* out;
   float* lse;
   int32_t* status;
-  float* part_o;                 // [slots][D/4][MT*128][4] fp32, column-group major
+  tv_bf16* part_o;               // [slots][D/8][MT*128][8] bf16 normalised outputs, column-group major
   float* part_ml;                // [slots][2][MT*128]  (m in log2 units, then l)
   unsigned long long* counters;  // [B*Hkv*NP][2]: tickets claimed, partials ready (epoch-tagged)
   unsigned long long epoch;      // 48-bit tag of this call
@@ -389,17 +402,23 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  // Small problems use fewer CTA groups, so that a unit is cut into few pieces (each piece costs a partial
+  // write and a merge) and every group still gets a worthwhile share of tiles.
+  int groups;
   {
     const long long total = (long long)prm.Hkv * cum[prm.B];
-    for (int k = threadIdx.x; k <= prm.groups; k += kThreads) gs[k] = (int)((total * k) / prm.groups);
+    const long long want = total / kMinVirtualTilesPerGroup;
+    groups = want < 1 ? 1 : (want < prm.groups ? (int)want : prm.groups);
+    for (int k = threadIdx.x; k <= prm.groups; k += kThreads)
+      gs[k] = k <= groups ? (int)((total * k) / groups) : (int)total;
   }
   __syncthreads();
 
   Sched sch{cum, gs, prm.B, prm.Hkv, (long long)prm.Hkv * cum[prm.B]};
   const int group = blockIdx.x / prm.NP;
   const int pair = blockIdx.x % prm.NP;
-  const long long g_begin = sch.group_start(group, prm.groups);
-  const long long g_end = sch.group_start(group + 1, prm.groups);
+  const long long g_begin = sch.group_start(group, groups);        // groups past the last used one get an empty range
+  const long long g_end = sch.group_start(group + 1, groups);
 
   // Walks the items of this CTA's range; identical in every role.
   auto next_item = [&](long long& g, Item& it) -> bool {
@@ -612,12 +631,24 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
         float m_used = -INFINITY;      // running reference maximum, in log2 units (score * scale * log2e)
         float l_sum = 0.f;
+        // A piece of a cut unit draws its ticket early (thread 128 only): the counter is read at the start of
+        // the item and the compare-and-swap is issued when the last key tile begins, so that both round trips
+        // are hidden behind the softmax of that tile; the outcome is looked at in the epilogue.
+        const bool piece = !(it.j0 == 0 && it.j1 == it.len);
+        unsigned long long* claim_ctr = prm.counters + (((size_t)it.b * prm.Hkv + it.hk) * prm.NP + pair) * 2;
+        unsigned long long claim_assumed = 0, claim_ret = 1;
+        int claim_cnt = 0;
+        if (piece && threadIdx.x == 128) claim_assumed = *reinterpret_cast<volatile unsigned long long*>(claim_ctr);
         const uint32_t s_base = tmem + lane_addr + kTmemS0 + wg * 128;
         const uint32_t o_addr_loop = tmem + lane_addr + kTmemO0 + wg * 128;
         for (int jt = 0; jt < nt && ok; ++jt) {
           const int j = it.j0 + jt;
           const bool tree = (j == it.len - 1);
           const int valid_keys = tree ? it.n : min(kTileN, it.S - j * kTileN);
+          if (piece && threadIdx.x == 128 && jt == nt - 1) {
+            claim_cnt = ((claim_assumed >> 16) == prm.epoch) ? (int)(claim_assumed & 0xffffu) : 0;
+            claim_ret = atomicCAS(claim_ctr, claim_assumed, (prm.epoch << 16) | (unsigned long long)(claim_cnt + 1));
+          }
           // ---- V rows past the valid keys may hold anything (stale cache rows, padded tree slots): zero
           // them so that 0 * NaN never reaches O.  Idempotent, so both warpgroups may do it.
           if (valid_keys < kTileN) {
@@ -799,20 +830,24 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               *lse_p = (row_active && l_sum > 0.f) ? (m_used + log2f(l_sum)) / kLog2e : -INFINITY;
             tc_fence_before();
           } else {
-            // ---- a piece of a unit.  The pieces of a unit draw tickets on the unit's "claimed" counter: the
-            // piece with the last ticket becomes the merger and keeps its O in TMEM; every other piece leaves
-            // (O, m, l) in its CTA's slot and then bumps the unit's "ready" counter.  The merger waits (bounded)
-            // until all other pieces are ready - they hold tickets, so they are running their epilogue - and
-            // folds them into its own accumulator.  Both counters carry the call's epoch, so the workspace
-            // needs no initialisation.  Partial O is stored column-group major,
-            // [slot][D/4][MT*128 rows][4 floats]: a warp writes and reads 512 contiguous bytes per instruction.
+            // ---- a piece of a unit.  The pieces of a unit draw tickets on the unit's "claimed" counter (the
+            // draw was started while the last key tile was still being processed): the piece with the last
+            // ticket becomes the merger and keeps its O in TMEM; every other piece leaves its normalised
+            // output O/l (bf16) and (m, l) in its CTA's slot and then bumps the unit's "ready" counter.  The
+            // merger waits (bounded) until all other pieces are ready - they hold tickets, so they are in
+            // their epilogue - and combines out = sum_p w_p O_p / sum_p w_p with w_p = l_p 2^(m_p - max m).
+            // Every piece enters the sum as its bf16-rounded normalised output, the merger's own included,
+            // and the sum runs in piece order with one fused multiply-add per piece, so the result does not
+            // depend on which piece merges.  Both counters carry the call's epoch: no initialisation needed.
+            // Partial outputs are stored column-group major, [slot][D/8][MT*128 rows][8 bf16]: a warp writes
+            // and reads 512 contiguous bytes per instruction.
             constexpr int kRows = MT * 128;
             const int rr = wg * 128 + row;
             // unit geometry in the virtual tile space: real tiles occupy [real0, uend)
             const long long real0 = (long long)prm.Hkv * cum[it.b] + (long long)it.hk * (it.len + kSetupCost) + kSetupCost;
             const long long uend = real0 + it.len;
-            const int k_first = sch.find_group(real0, prm.groups);
-            const int k_last = sch.find_group(uend - 1, prm.groups);
+            const int k_first = sch.find_group(real0, groups);
+            const int k_last = sch.find_group(uend - 1, groups);
             // slot of the piece CTA group k holds of this unit, or -1 if it holds none
             auto piece_slot = [&](int k) -> int {
               const long long ks = gs[k], ke = gs[k + 1];
@@ -820,22 +855,29 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               if (lo >= hi) return -1;
               return (k * prm.NP + pair) * 2 + (ks > real0 ? 0 : 1);
             };
-            int n_frag = 0;
-            for (int k = k_first; k <= k_last; ++k) n_frag += piece_slot(k) >= 0 ? 1 : 0;
-            unsigned long long* ctr = prm.counters + (((size_t)it.b * prm.Hkv + it.hk) * prm.NP + pair) * 2;
-            // epoch-tagged increment: returns the count after this arrival
-            auto bump = [&](unsigned long long* c) -> int {
-              unsigned long long seen = *reinterpret_cast<volatile unsigned long long*>(c);
-              while (true) {
-                const unsigned long long assumed = seen;
-                const int cnt = ((assumed >> 16) == prm.epoch) ? (int)(assumed & 0xffffu) : 0;
-                seen = atomicCAS(c, assumed, (prm.epoch << 16) | (unsigned long long)(cnt + 1));
-                if (seen == assumed) return cnt + 1;
+            const int my_slot = blockIdx.x * 2 + (it.j0 > 0 ? 0 : 1);
+            int n_frag = 0, n_other = 0, own_pos = 0, sid_a = 0, sid_b = 0;
+            for (int k = k_first; k <= k_last; ++k) {
+              const int sid = piece_slot(k);
+              if (sid < 0) continue;
+              ++n_frag;
+              if (sid == my_slot) {
+                own_pos = n_other;           // number of other pieces that come before this one
+              } else {
+                if (n_other == 0) sid_a = sid;
+                if (n_other == 1) sid_b = sid;
+                ++n_other;
               }
-            };
+            }
+            unsigned long long* ctr = prm.counters + (((size_t)it.b * prm.Hkv + it.hk) * prm.NP + pair) * 2;
             if (threadIdx.x == 128) {
-              const int ticket = bump(ctr);
-              int merger = (ticket == n_frag) ? 1 : 0;
+              int ticket;
+              if (claim_ret == claim_assumed) {
+                ticket = claim_cnt + 1;                      // the early draw went through
+              } else {
+                ticket = bump_counter(ctr, claim_ret, prm.epoch);
+              }
+              const int merger = (ticket == n_frag) ? 1 : 0;
               if (merger) {
                 // wait until the other n_frag - 1 pieces have published their partials
                 const unsigned long long t0 = globaltimer_ns();
@@ -855,9 +897,9 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             ok = epi_sync();
             if (!ok || *abort_flag) { ok = false; break; }
             tr.mark(0x7000u | (*last_flag ? 1u : 0u));
-            const int my_slot = blockIdx.x * 2 + (it.j0 > 0 ? 0 : 1);
+            const float inv_own = (row_active && l_sum > 0.f) ? 1.f / l_sum : 0.f;
             if (!*last_flag) {
-              float* po = prm.part_o + (size_t)my_slot * (D / 4) * kRows * 4;
+              uint4* po = reinterpret_cast<uint4*>(prm.part_o) + (size_t)my_slot * (D / 8) * kRows;
               float* pml = prm.part_ml + (size_t)my_slot * 2 * kRows;
 #pragma unroll
               for (int q = 0; q < D / 32; ++q) {
@@ -866,9 +908,14 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 tmem_wait_ld();
                 if (row_active) {
 #pragma unroll
-                  for (int c = 0; c < 8; ++c)
-                    *reinterpret_cast<uint4*>(po + ((size_t)(q * 8 + c) * kRows + rr) * 4) =
-                        make_uint4(o[4 * c], o[4 * c + 1], o[4 * c + 2], o[4 * c + 3]);
+                  for (int c = 0; c < 4; ++c) {
+                    uint4 v;
+                    v.x = pack_bf16(__uint_as_float(o[8 * c + 0]) * inv_own, __uint_as_float(o[8 * c + 1]) * inv_own);
+                    v.y = pack_bf16(__uint_as_float(o[8 * c + 2]) * inv_own, __uint_as_float(o[8 * c + 3]) * inv_own);
+                    v.z = pack_bf16(__uint_as_float(o[8 * c + 4]) * inv_own, __uint_as_float(o[8 * c + 5]) * inv_own);
+                    v.w = pack_bf16(__uint_as_float(o[8 * c + 6]) * inv_own, __uint_as_float(o[8 * c + 7]) * inv_own);
+                    po[(size_t)(q * 4 + c) * kRows + rr] = v;
+                  }
                 }
               }
               if (row_active) {
@@ -880,45 +927,46 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               tr.mark(0x6000u);
               ok = epi_sync();
               if (!ok) break;
-              if (threadIdx.x == 128) bump(ctr + 1);
-            } else {
-              // The sums below run over the pieces in their order inside the unit with one fused multiply-add
-              // per piece, whichever piece happens to be the merger: the result does not depend on timing.
-              float mm = m_used, lt = 0.f;
-              int n_other = 0, sid1 = 0, own_pos = 0;
-              for (int k = k_first; k <= k_last; ++k) {
-                const int sid = piece_slot(k);
-                if (sid < 0) continue;
-                if (sid == my_slot) {
-                  own_pos = n_other;         // number of other pieces that come before this one
-                  continue;
-                }
-                sid1 = sid;
-                ++n_other;
+              if (threadIdx.x == 128) {
+                const unsigned long long seen = *reinterpret_cast<volatile unsigned long long*>(ctr + 1);
+                bump_counter(ctr + 1, seen, prm.epoch);
               }
-              if (n_other == 1) {
-                // the usual case, one other piece: fetch its (m, l) and its O with as few dependent round
-                // trips to L2 as possible (everything of a batch is requested before anything is used).
-                // Loads are issued by every thread (row rr always lies inside the slot; rows that are not
-                // active read stale bytes and are masked by selects): no thread-divergent branch may sit
-                // between the warp-wide TMEM instructions below.
-                const float* q_ml = prm.part_ml + (size_t)sid1 * 2 * kRows;
-                const float* q_o = prm.part_o + (size_t)sid1 * (D / 4) * kRows * 4;
-                const float m1 = __ldcg(q_ml + rr);
-                const float l1 = __ldcg(q_ml + kRows + rr);
-                const bool own_first = own_pos == 0;
-                float w_own = 0.f, w1 = 0.f, inv = 0.f;
+            } else {
+              float mm = m_used, lt = 0.f;
+              if (n_other <= 2) {
+                // ---- up to two other pieces (the usual cases): everything of a batch is requested before
+                // anything is used, two dependent round trips to L2 in total.  Loads are issued by every
+                // thread (row rr always lies inside a slot; rows that are not active read stale bytes and
+                // are masked by selects): no thread-divergent branch sits between the warp-wide TMEM ops.
+                if (n_other == 1) sid_b = sid_a;
+                const float* ml_a = prm.part_ml + (size_t)sid_a * 2 * kRows;
+                const float* ml_b = prm.part_ml + (size_t)sid_b * 2 * kRows;
+                const uint4* o_a = reinterpret_cast<const uint4*>(prm.part_o) + (size_t)sid_a * (D / 8) * kRows;
+                const uint4* o_b = reinterpret_cast<const uint4*>(prm.part_o) + (size_t)sid_b * (D / 8) * kRows;
+                const float m_a = __ldcg(ml_a + rr), l_a = __ldcg(ml_a + kRows + rr);
+                const float m_b = (n_other == 2) ? __ldcg(ml_b + rr) : -INFINITY;
+                const float l_b = (n_other == 2) ? __ldcg(ml_b + kRows + rr) : 0.f;
+                float w_o = 0.f, w_a = 0.f, w_b = 0.f, inv = 0.f;
+                // ordered combination of (own, a, b) by the position of the own piece inside the unit
+                auto comb = [&](float vo, float va, float vb) -> float {
+                  if (own_pos == 0) return fmaf(w_b, vb, fmaf(w_a, va, w_o * vo));
+                  if (own_pos == 1) return fmaf(w_b, vb, fmaf(w_o, vo, w_a * va));
+                  return fmaf(w_o, vo, fmaf(w_b, vb, w_a * va));
+                };
 #pragma unroll
                 for (int half = 0; half < D / 64; ++half) {
-                  float4 v[16];
+                  uint4 va[8], vb[8];
 #pragma unroll
-                  for (int c = 0; c < 16; ++c)
-                    v[c] = __ldcg(reinterpret_cast<const float4*>(q_o + ((size_t)(half * 16 + c) * kRows + rr) * 4));
+                  for (int c = 0; c < 8; ++c) {
+                    va[c] = __ldcg(o_a + (size_t)(half * 8 + c) * kRows + rr);
+                    vb[c] = __ldcg(o_b + (size_t)(half * 8 + c) * kRows + rr);
+                  }
                   if (half == 0) {
-                    mm = fmaxf(m_used, m1);
-                    w_own = row_active ? fast_exp2(m_used - mm) : 0.f;
-                    w1 = row_active ? fast_exp2(m1 - mm) : 0.f;
-                    lt = own_first ? fmaf(w1, l1, w_own * l_sum) : fmaf(w_own, l_sum, w1 * l1);
+                    mm = fmaxf(m_used, fmaxf(m_a, m_b));
+                    w_o = row_active ? l_sum * fast_exp2(m_used - mm) : 0.f;
+                    w_a = row_active ? l_a * fast_exp2(m_a - mm) : 0.f;
+                    w_b = (row_active && n_other == 2) ? l_b * fast_exp2(m_b - mm) : 0.f;
+                    lt = comb(1.f, 1.f, 1.f);
                     inv = (row_active && lt > 0.f) ? 1.f / lt : 0.f;
                   }
 #pragma unroll
@@ -929,21 +977,21 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     if (row_exists) {
 #pragma unroll
                       for (int c = 0; c < 4; ++c) {
-                        float r[8];
+                        const uint4 pa = va[q * 4 + c], pb = vb[q * 4 + c];
+                        const uint32_t wa[4] = {pa.x, pa.y, pa.z, pa.w}, wb[4] = {pb.x, pb.y, pb.z, pb.w};
+                        uint32_t pk[4];
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) {
-                          const float4 vv = v[q * 8 + c * 2 + e / 4];
-                          const float ve = (e % 4 == 0) ? vv.x : (e % 4 == 1) ? vv.y : (e % 4 == 2) ? vv.z : vv.w;
-                          const float oe = __uint_as_float(o[c * 8 + e]);
-                          const float sum = own_first ? fmaf(w1, ve, w_own * oe) : fmaf(w_own, oe, w1 * ve);
-                          r[e] = row_active ? sum * inv : 0.f;
+                        for (int e = 0; e < 4; ++e) {
+                          // the own piece enters as its bf16-rounded normalised output, like every other piece
+                          const uint32_t own = pack_bf16(__uint_as_float(o[c * 8 + 2 * e]) * inv_own,
+                                                         __uint_as_float(o[c * 8 + 2 * e + 1]) * inv_own);
+                          const float r0 = comb(__uint_as_float(own << 16), __uint_as_float(wa[e] << 16),
+                                                (n_other == 2) ? __uint_as_float(wb[e] << 16) : 0.f);
+                          const float r1 = comb(__uint_as_float(own & 0xffff0000u), __uint_as_float(wa[e] & 0xffff0000u),
+                                                (n_other == 2) ? __uint_as_float(wb[e] & 0xffff0000u) : 0.f);
+                          pk[e] = row_active ? pack_bf16(r0 * inv, r1 * inv) : 0u;
                         }
-                        uint4 pk;
-                        pk.x = pack_bf16(r[0], r[1]);
-                        pk.y = pack_bf16(r[2], r[3]);
-                        pk.z = pack_bf16(r[4], r[5]);
-                        pk.w = pack_bf16(r[6], r[7]);
-                        *reinterpret_cast<uint4*>(orow + (half * 2 + q) * 32 + c * 8) = pk;
+                        *reinterpret_cast<uint4*>(orow + (half * 2 + q) * 32 + c * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                       }
                     }
                   }
@@ -953,23 +1001,22 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 if (row_active) {
                   for (int k = k_first; k <= k_last; ++k) {
                     const int sid = piece_slot(k);
-                    if (sid < 0) continue;
-                    if (sid == my_slot) continue;
+                    if (sid < 0 || sid == my_slot) continue;
                     mm = fmaxf(mm, __ldcg(prm.part_ml + (size_t)sid * 2 * kRows + rr));
                   }
                   for (int k = k_first; k <= k_last; ++k) {
                     const int sid = piece_slot(k);
                     if (sid < 0) continue;
                     if (sid == my_slot) {
-                      lt = fmaf(fast_exp2(m_used - mm), l_sum, lt);
+                      lt = fmaf(l_sum * fast_exp2(m_used - mm), 1.f, lt);
                     } else {
                       const float* q_ml = prm.part_ml + (size_t)sid * 2 * kRows;
-                      lt = fmaf(fast_exp2(__ldcg(q_ml + rr) - mm), __ldcg(q_ml + kRows + rr), lt);
+                      lt = fmaf(__ldcg(q_ml + kRows + rr) * fast_exp2(__ldcg(q_ml + rr) - mm), 1.f, lt);
                     }
                   }
                 }
                 const float inv = (row_active && lt > 0.f) ? 1.f / lt : 0.f;
-                const float w_own = row_active ? fast_exp2(m_used - mm) : 0.f;
+                const float w_own = row_active ? l_sum * fast_exp2(m_used - mm) : 0.f;
                 // ---- pass 2: 32 output columns at a time, pieces in order; the own piece comes from TMEM
 #pragma unroll 1
                 for (int q = 0; q < D / 32; ++q) {
@@ -985,21 +1032,27 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                       if (sid < 0) continue;
                       if (sid == my_slot) {
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) acc[c] = fmaf(w_own, __uint_as_float(o[c]), acc[c]);
+                        for (int c = 0; c < 16; ++c) {
+                          const uint32_t own = pack_bf16(__uint_as_float(o[2 * c]) * inv_own, __uint_as_float(o[2 * c + 1]) * inv_own);
+                          acc[2 * c] = fmaf(w_own, __uint_as_float(own << 16), acc[2 * c]);
+                          acc[2 * c + 1] = fmaf(w_own, __uint_as_float(own & 0xffff0000u), acc[2 * c + 1]);
+                        }
                         continue;
                       }
-                      const float w = fast_exp2(__ldcg(prm.part_ml + (size_t)sid * 2 * kRows + rr) - mm);
-                      const float* q_o = prm.part_o + (size_t)sid * (D / 4) * kRows * 4;
-                      float4 v[8];
+                      const float* q_ml = prm.part_ml + (size_t)sid * 2 * kRows;
+                      const float w = __ldcg(q_ml + kRows + rr) * fast_exp2(__ldcg(q_ml + rr) - mm);
+                      const uint4* q_o = reinterpret_cast<const uint4*>(prm.part_o) + (size_t)sid * (D / 8) * kRows;
+                      uint4 v[4];
 #pragma unroll
-                      for (int c = 0; c < 8; ++c)
-                        v[c] = __ldcg(reinterpret_cast<const float4*>(q_o + ((size_t)(q * 8 + c) * kRows + rr) * 4));
+                      for (int c = 0; c < 4; ++c) v[c] = __ldcg(q_o + (size_t)(q * 4 + c) * kRows + rr);
 #pragma unroll
-                      for (int c = 0; c < 8; ++c) {
-                        acc[4 * c] = fmaf(w, v[c].x, acc[4 * c]);
-                        acc[4 * c + 1] = fmaf(w, v[c].y, acc[4 * c + 1]);
-                        acc[4 * c + 2] = fmaf(w, v[c].z, acc[4 * c + 2]);
-                        acc[4 * c + 3] = fmaf(w, v[c].w, acc[4 * c + 3]);
+                      for (int c = 0; c < 4; ++c) {
+                        const uint32_t wv[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                          acc[8 * c + 2 * e] = fmaf(w, __uint_as_float(wv[e] << 16), acc[8 * c + 2 * e]);
+                          acc[8 * c + 2 * e + 1] = fmaf(w, __uint_as_float(wv[e] & 0xffff0000u), acc[8 * c + 2 * e + 1]);
+                        }
                       }
                     }
                   }
@@ -1110,7 +1163,7 @@ Geometry geometry(int B, int Nmax, int Hq, int Hkv, int d, bool query_device) {
   off += max_ctas * 2 * (size_t)g.MT * 128 * 2 * sizeof(float);
   off = (off + 255) & ~size_t(255);
   g.o_off = off;
-  off += max_ctas * 2 * (size_t)g.MT * 128 * d * sizeof(float);
+  off += max_ctas * 2 * (size_t)g.MT * 128 * d * sizeof(tv_bf16);
   g.total = off;
   return g;
 }
@@ -1209,7 +1262,7 @@ extern "C" int tree_verify_attn(const tv_bf16* q,
   char* ws = static_cast<char*>(workspace);
   prm.counters = reinterpret_cast<unsigned long long*>(ws + g.counters_off);
   prm.part_ml = reinterpret_cast<float*>(ws + g.ml_off);
-  prm.part_o = reinterpret_cast<float*>(ws + g.o_off);
+  prm.part_o = reinterpret_cast<tv_bf16*>(ws + g.o_off);
   prm.epoch = next_epoch();
   prm.B = B; prm.Nmax = Nmax; prm.Hq = Hq; prm.Hkv = Hkv; prm.Scap = Scap;
   prm.G = g.G; prm.NPT = g.NPT; prm.NP = g.NP; prm.W = (Nmax + 31) / 32; prm.groups = g.groups;
