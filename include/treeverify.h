@@ -125,8 +125,9 @@ TV_API size_t tv_attn_workspace_bytes(int B, int Nmax, int Hq, int Hkv, int d, i
  *                                      tv_attn_workspace_bytes(...) bytes
  *   status[B]                      in/out: TV_ST_TIMEOUT is ORed in if a
  *                                      bounded wait expired (outputs invalid)
- * Limits: d in {64,128}; Nmax <= 128; Hq % Hkv == 0; all tensors 16-byte
- * aligned; 0 <= prefix_len[b] <= Scap.
+ * Limits: d in {64,128}; Nmax <= 256 (the node budgets of the paper's sweep);
+ * Hq % Hkv == 0, Hq / Hkv <= 128; B <= 512; all tensors 16-byte aligned;
+ * 0 <= prefix_len[b] <= Scap; scale > 0.
  */
 TV_API int tree_verify_attn(const tv_bf16* q,
                      const tv_bf16* k_cache, const tv_bf16* v_cache,

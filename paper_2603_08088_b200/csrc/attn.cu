@@ -270,6 +270,7 @@ struct AttnParams {
   unsigned long long* counters;  // [B*Hkv*NP][2]: tickets claimed, partials ready (epoch-tagged)
   unsigned long long epoch;      // 48-bit tag of this call
   int B, Nmax, Hq, Hkv, Scap, G, NPT, NP, W, groups;
+  int TT;                        // key tiles of the tree's own K/V: ceil(Nmax / 128), 1 or 2
   uint32_t q_box_bytes;
   unsigned long long* trace;     // optional event trace [cta][role 0..3][kTraceCap] of (tag << 48 | ns), or NULL          // bytes of one Q box {64, G, NPT}: 16 KB when G divides 128
   float scale_log2e;             // scale * log2(e)
@@ -360,7 +361,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       if (b < prm.B) {
         int S = prm.prefix_len[b];
         S = S < 0 ? 0 : (S > prm.Scap ? prm.Scap : S);
-        len = (S + kTileN - 1) / kTileN + 1 + kSetupCost;
+        len = (S + kTileN - 1) / kTileN + prm.TT + kSetupCost;
       }
       int inc = len;
 #pragma unroll
@@ -476,7 +477,8 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                         it.hk * prm.G, (pair * MT + t) * prm.NPT, it.b);
         ++item_idx;
         for (int j = it.j0; j < it.j1 && ok; ++j) {
-          const bool tree = (j == it.len - 1);
+          const int tt = j - (it.len - prm.TT);      // >= 0: index of the tree key tile
+          const bool tree = tt >= 0;
 #pragma unroll
           for (int kv = 0; kv < 2; ++kv) {
             const uint32_t slot = fill % kSlots, round = fill / kSlots;
@@ -492,7 +494,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 #pragma unroll
             for (int h = 0; h < D / 64; ++h) {
               if (tree)
-                tma_load_4d(dst + h * L::kHalf, kv ? &map_vt : &map_kt, bar(L::KV_FULL + slot), h * 64, it.hk, 0, it.b);
+                tma_load_4d(dst + h * L::kHalf, kv ? &map_vt : &map_kt, bar(L::KV_FULL + slot), h * 64, it.hk, tt * kTileN, it.b);
               else
                 tma_load_3d(dst + h * L::kHalf, kv ? &map_vc : &map_kc, bar(L::KV_FULL + slot), h * 64, j * kTileN,
                             it.b * prm.Hkv + it.hk);
@@ -623,10 +625,10 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const int gm = row % prm.G;
         const bool row_exists = row < prm.NPT * prm.G && node < prm.Nmax;
         const bool row_active = row_exists && node < it.n;
-        uint32_t anc[4] = {0u, 0u, 0u, 0u};
+        uint32_t anc[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
         if (row_active) {
 #pragma unroll
-          for (int w = 0; w < 4; ++w)
+          for (int w = 0; w < 8; ++w)
             if (w < prm.W) anc[w] = prm.anc_bits[((size_t)it.b * prm.Nmax + node) * prm.W + w];
         }
         float m_used = -INFINITY;      // running reference maximum, in log2 units (score * scale * log2e)
@@ -643,8 +645,9 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const uint32_t o_addr_loop = tmem + lane_addr + kTmemO0 + wg * 128;
         for (int jt = 0; jt < nt && ok; ++jt) {
           const int j = it.j0 + jt;
-          const bool tree = (j == it.len - 1);
-          const int valid_keys = tree ? it.n : min(kTileN, it.S - j * kTileN);
+          const int tt = j - (it.len - prm.TT);      // >= 0: index of the tree key tile
+          const bool tree = tt >= 0;
+          const int valid_keys = tree ? max(0, min(kTileN, it.n - tt * kTileN)) : min(kTileN, it.S - j * kTileN);
           if (piece && threadIdx.x == 128 && jt == nt - 1) {
             claim_cnt = ((claim_assumed >> 16) == prm.epoch) ? (int)(claim_assumed & 0xffffu) : 0;
             claim_ret = atomicCAS(claim_ctr, claim_assumed, (prm.epoch << 16) | (unsigned long long)(claim_cnt + 1));
@@ -684,7 +687,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               for (int q = 0; q < 2; ++q) {
                 uint32_t word;
                 if (tree) {
-                  word = anc[2 * h + q];
+                  word = (tt > 0) ? anc[4 + 2 * h + q] : anc[2 * h + q];
                 } else {
                   const int cnt = valid_half - 32 * q;
                   word = cnt >= 32 ? 0xffffffffu : (cnt <= 0 ? 0u : ((1u << cnt) - 1u));
@@ -1217,7 +1220,7 @@ extern "C" int tree_verify_attn(const tv_bf16* q,
                  workspace,
              "tree_verify_attn: NULL pointer");
   TV_REQUIRE(B >= 0 && B <= kMaxB, "tree_verify_attn: need 0 <= B <= 512");
-  TV_REQUIRE(Nmax >= 1 && Nmax <= 128, "tree_verify_attn: Nmax must be in 1..128");
+  TV_REQUIRE(Nmax >= 1 && Nmax <= 256, "tree_verify_attn: Nmax must be in 1..256");
   TV_REQUIRE(d == 64 || d == 128, "tree_verify_attn: d must be 64 or 128");
   TV_REQUIRE(Hq >= 1 && Hkv >= 1 && Hq % Hkv == 0 && Hq / Hkv <= kTileM, "tree_verify_attn: need Hq %% Hkv == 0 and Hq/Hkv <= 128");
   TV_REQUIRE(Scap >= 1 && scale > 0.f, "tree_verify_attn: need Scap >= 1 and scale > 0");
@@ -1227,7 +1230,7 @@ extern "C" int tree_verify_attn(const tv_bf16* q,
   TV_REQUIRE((reinterpret_cast<uintptr_t>(workspace) & 255u) == 0, "tree_verify_attn: workspace must be 256-byte aligned");
   if (B == 0) return TV_OK;
   const Geometry g = geometry(B, Nmax, Hq, Hkv, d, true);
-  TV_REQUIRE((long long)B * Hkv * ((Scap + kTileN - 1) / kTileN + 1 + kSetupCost) < (1ll << 31),
+  TV_REQUIRE((long long)B * Hkv * ((Scap + kTileN - 1) / kTileN + 2 + kSetupCost) < (1ll << 31),
              "tree_verify_attn: B * Hkv * Scap is too large for the tile scheduler");
   if (g.grid > 160) return tv::fail(TV_ERR_INVALID_ARG, "tree_verify_attn: device with more than 160 SMs is not supported");
   if (workspace_bytes < g.total)
@@ -1264,6 +1267,7 @@ extern "C" int tree_verify_attn(const tv_bf16* q,
   prm.epoch = next_epoch();
   prm.B = B; prm.Nmax = Nmax; prm.Hq = Hq; prm.Hkv = Hkv; prm.Scap = Scap;
   prm.G = g.G; prm.NPT = g.NPT; prm.NP = g.NP; prm.W = (Nmax + 31) / 32; prm.groups = g.groups;
+  prm.TT = (Nmax + kTileN - 1) / kTileN;
   prm.scale = scale;
   prm.q_box_bytes = 64u * (uint32_t)g.G * (uint32_t)g.NPT * 2u;
   prm.trace = g_trace.load(std::memory_order_relaxed);

@@ -49,9 +49,9 @@ def test_null_and_bad_dims_are_rejected_without_a_launch(lib):
     assert rc == 1
     rc = lib.tree_accept(one, one, one, one, 1, 8, 100, 2, 3, one, None, None, one, one, one, one, one, 0, one, None)
     assert rc == 3     # workspace too small
-    rc = lib.tree_verify_attn(one, one, one, one, one, one, one, one, 1, 200, 4, 2, 64, 64, 1.0, one, None,
+    rc = lib.tree_verify_attn(one, one, one, one, one, one, one, one, 1, 300, 4, 2, 64, 64, 1.0, one, None,
                               one, 1 << 30, one, None)
-    assert rc == 1     # Nmax > 128
+    assert rc == 1     # Nmax > 256
 
 
 def test_missing_library_fails_loudly(monkeypatch):

@@ -88,6 +88,28 @@ def test_attention_parity_small(name, ci, over, simt):
             assert np.isneginf(f32(lse)[b, :, n[b]:]).all()
 
 
+BUDGETS = [(16, 10), (32, 10), (64, 4), (64, 16), (128, 10), (200, 12), (256, 10), (256, 16)]
+
+
+@pytest.mark.parametrize("N,D", BUDGETS, ids=[f"M{n}_D{d}" for n, d in BUDGETS])
+def test_budget_sweep_shapes(N, D):
+    """Node budgets and depth bounds of the paper's sweep (Table 2: M in 16..256, Dmax in 4..16);
+    more than 128 nodes means two tree key tiles and eight mask words per row."""
+    cfg = CONFIGS[2].scaled(B=3, Hq=8, Hkv=2, S_lo=100, S_hi=420, Scap=512, N=N, D=D, tree="spine", V=0)
+    case = make_case(cfg, seed=7000 + N + D, ragged_nodes=True, with_logits=False)
+    n = case["n_nodes"].numpy()
+    nan = torch.tensor(float("nan"), dtype=torch.bfloat16)
+    for b in range(cfg.B):
+        case["k_tree"][:, b, n[b]:] = nan
+        case["v_tree"][:, b, n[b]:] = nan
+    dcase = to_device(case)
+    out, lse, bits, dense = gpu_attention(dcase)
+    ref_out, ref_lse = oracle_attention(case_to_numpy(case), dense.cpu().numpy())
+    assert_attention_close(out, lse, ref_out, ref_lse, f"M={N} D={D}")
+    out2, lse2, _, _ = gpu_attention(dcase, simt=True)
+    assert_attention_close(out2, lse2, ref_out, ref_lse, f"simt M={N} D={D}")
+
+
 def _tree_case(parent, S, Hq, Hkv, d, Scap, seed, std=1.0):
     N = len(parent)
     cfg = CONFIGS[0].scaled(B=1, Hq=Hq, Hkv=Hkv, d=d, S_lo=S, S_hi=S, Scap=Scap, N=N, D=min(3, N - 1), std=std, V=0)

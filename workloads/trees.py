@@ -75,6 +75,25 @@ def topk_expansion_tree(N, D, topk, rng):
             return parent
 
 
+def spine_tree(N, D, rng):
+    """A tree that reaches depth D for any budget N > D: nodes 1..D form a chain from the root, every later
+    node picks a uniform parent among the nodes of depth < D (deep, narrow budgets of the paper's sweep)."""
+    assert N >= D + 1
+    parent = np.full(N, -1, dtype=np.int32)
+    dep = np.zeros(N, dtype=np.int64)
+    for i in range(1, N):
+        if i <= D:
+            p = i - 1
+        else:
+            while True:
+                p = int(rng.integers(0, i))
+                if dep[p] < D:
+                    break
+        parent[i] = p
+        dep[i] = dep[p] + 1
+    return parent
+
+
 def chain_tree(N):
     """0 <- 1 <- 2 ... : the linear speculative proposal of Section 2.2."""
     return np.arange(-1, N - 1, dtype=np.int32)
