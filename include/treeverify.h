@@ -178,6 +178,22 @@ TV_API int tree_accept(const tv_bf16* logits, const int32_t* tokens,
                 int32_t* status, tv_stream stream);
 
 /*
+ * Node verification scores (Section 3.3, "Mapping teacher outputs to node
+ * verification scores"): the teacher's logit of every node's proposed token,
+ * taken from the logits row of the node's parent slot (that row predicts the
+ * node's token): scores[b,k] = logits[b, parent~[b,k], tokens[b,k]], the input
+ * of a score-based (non-greedy) acceptance rule.  An in-range gather over the
+ * vocabulary, guarded by valid: the sentinel parent is remapped to 0, the root
+ * and padded slots give 0, a token outside [0,V) gives -inf and raises
+ * TV_ST_BAD_INDEX (its index is remapped to 0 before the gather).
+ *   logits[B,Nmax,V] bf16, tokens[B,Nmax], parent[B,Nmax], n_nodes[B]  in
+ *   scores[B,Nmax] fp32  out;  status[B]  in/out
+ */
+TV_API int tree_node_scores(const tv_bf16* logits, const int32_t* tokens, const int32_t* parent,
+                            const int32_t* n_nodes, int B, int Nmax, int V, float* scores,
+                            int32_t* status, tv_stream stream);
+
+/*
  * tree_accept for callers that cannot allocate device memory (the paper has
  * no counterpart; this is a convenience of this library).  Some hosts of this
  * code may not call cudaMalloc at all: a plugin inside a serving runtime that

@@ -254,6 +254,34 @@ def argmax_rows(logits_bits, n_nodes):
     return am
 
 
+def node_scores(logits_bits, tokens, parent, n_nodes):
+    """Teacher score of every node's proposed token (Section 3.3, "Mapping teacher outputs to node
+    verification scores"): the logits that predict node k's token are those computed at its parent's
+    slot, so score[b,k] = logits[b, parent~[k], tokens[b,k]] with the dummy-root remap of Section 3.2.
+    An in-range gather over the vocabulary guarded by valid: the root (already part of the prefix) and
+    padded slots give 0; a token outside [0,V) is remapped to 0 before the gather, scores -inf and
+    raises BAD_INDEX.  Returns scores[B,Nmax] (float32 values of the bf16 logits) and status[B]."""
+    B, Nmax, V = logits_bits.shape
+    scores = np.zeros((B, Nmax), dtype=np.float32)
+    status = np.zeros(B, dtype=np.int32)
+    for b in range(B):
+        n = int(n_nodes[b])
+        for k in range(1, min(n, Nmax)):
+            p = int(parent[b, k])
+            sp = p if 0 <= p < n else 0
+            t = int(tokens[b, k])
+            ok = 0 <= t < V
+            st = t if ok else 0
+            assert 0 <= sp < Nmax and 0 <= st < V          # every dereferenced index is in range
+            val = np.float32(decode_bf16(logits_bits[b, sp, st]))
+            if ok:
+                scores[b, k] = val
+            else:
+                scores[b, k] = -np.inf
+                status[b] |= ST_BAD_INDEX
+    return scores, status
+
+
 def greedy_accept(retrieve, tokens, n_nodes, am):
     """Longest accepted prefix over all candidate rows (Section 2.3: accepted
     nodes form a single root-to-leaf path prefix; greedy rule, Section 5).

@@ -15,7 +15,7 @@ TV_OK, TV_ERR_INVALID_ARG, TV_ERR_CUDA, TV_ERR_WORKSPACE = 0, 1, 2, 3
 TV_ST_BAD_TREE, TV_ST_BAD_INDEX, TV_ST_CAPACITY, TV_ST_TIMEOUT, TV_ST_PATHS_TRUNCATED = 1, 2, 4, 8, 16
 
 EXPORTS = ["tv_last_error", "tv_version", "tv_launch_count", "tree_build_mask", "tv_attn_workspace_bytes", "tree_verify_attn",
-           "tv_accept_workspace_bytes", "tree_accept", "tv_accept_noalloc_max_bytes", "tree_accept_noalloc",
+           "tv_accept_workspace_bytes", "tree_accept", "tree_node_scores", "tv_accept_noalloc_max_bytes", "tree_accept_noalloc",
            "kv_commit", "tv_step_staging_bytes",
            "tv_verify_step_host"]
 
@@ -65,6 +65,8 @@ def load():
     lib.tv_accept_workspace_bytes.argtypes = [_c_int] * 3
     lib.tree_accept.restype = _c_int
     lib.tree_accept.argtypes = [_c_vp] * 4 + [_c_int] * 5 + [_c_vp] * 7 + [_c_vp, _c_sz, _c_vp, _c_vp]
+    lib.tree_node_scores.restype = _c_int
+    lib.tree_node_scores.argtypes = [_c_vp] * 4 + [_c_int] * 3 + [_c_vp, _c_vp, _c_vp]
     lib.tv_accept_noalloc_max_bytes.restype = _c_sz
     lib.tv_accept_noalloc_max_bytes.argtypes = []
     lib.tree_accept_noalloc.restype = _c_int
@@ -158,6 +160,12 @@ def tree_accept(logits, tokens, retrieve_indices, n_nodes, argmax_tok, accept_le
                               _ptr(accept_len), _ptr(best_path), _ptr(accepted_nodes), _ptr(next_token),
                               _ptr(workspace), workspace.numel() * workspace.element_size(), _ptr(status),
                               _stream(stream)))
+
+
+def tree_node_scores(logits, tokens, parent, n_nodes, scores, status, stream=None):
+    B, Nmax, V = logits.shape
+    _check(load().tree_node_scores(_ptr(logits), _ptr(tokens), _ptr(parent), _ptr(n_nodes), B, Nmax, V,
+                                   _ptr(scores), _ptr(status), _stream(stream)))
 
 
 def tv_accept_noalloc_max_bytes():

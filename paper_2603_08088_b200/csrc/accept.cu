@@ -207,6 +207,29 @@ accept_kernel(const ArgPair* __restrict__ partial, int n_chunks,
   }
 }
 
+// One thread per (sequence, node): score of the node's proposed token in the logits of its parent's slot.
+__global__ void node_scores_kernel(const tv_bf16* __restrict__ logits, const int32_t* __restrict__ tokens,
+                                   const int32_t* __restrict__ parent, const int32_t* __restrict__ n_nodes,
+                                   int B, int Nmax, int V, float* __restrict__ scores, int32_t* __restrict__ status) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= B * Nmax) return;
+  const int b = idx / Nmax, k = idx - b * Nmax;
+  int n = n_nodes[b];
+  n = n < 0 ? 0 : (n > Nmax ? Nmax : n);
+  float val = 0.f;
+  if (k >= 1 && k < n) {
+    const int p = parent[idx];
+    const int sp = (p >= 0 && p < n) ? p : 0;          // dummy-root remap before the gather
+    const int t = tokens[idx];
+    const bool ok = t >= 0 && t < V;
+    const int st = ok ? t : 0;                          // in-range vocabulary index
+    const float g = bf16_bits_to_float(logits[((size_t)b * Nmax + sp) * V + st]);
+    val = ok ? g : -INFINITY;
+    if (!ok) atomicOr(&status[b], TV_ST_BAD_INDEX);
+  }
+  scores[idx] = val;
+}
+
 int scan_chunks(int V) { return (V + kChunkElems - 1) / kChunkElems; }
 
 // Scratch of tree_accept_noalloc: a fixed device array that lives in the library image, so that callers
@@ -297,4 +320,18 @@ extern "C" int tree_accept_noalloc(const tv_bf16* logits, const int32_t* tokens,
   return tree_accept(logits, tokens, retrieve_indices, n_nodes, B, Nmax, V, P, Dp1, argmax_tok, safe_idx, candidates,
                      accept_len, best_path, accepted_nodes, next_token, scratch, kStaticPairs * sizeof(ArgPair),
                      status, stream);
+}
+
+extern "C" int tree_node_scores(const tv_bf16* logits, const int32_t* tokens, const int32_t* parent,
+                                const int32_t* n_nodes, int B, int Nmax, int V, float* scores,
+                                int32_t* status, tv_stream stream) {
+  TV_REQUIRE(logits && tokens && parent && n_nodes && scores && status, "tree_node_scores: NULL pointer");
+  TV_REQUIRE(B >= 0 && Nmax >= 1 && V >= 1, "tree_node_scores: need B >= 0, Nmax >= 1, V >= 1");
+  if (B == 0) return TV_OK;
+  const int total = B * Nmax;
+  node_scores_kernel<<<(total + 127) / 128, 128, 0, (cudaStream_t)stream>>>(logits, tokens, parent, n_nodes, B, Nmax, V,
+                                                                             scores, status);
+  TV_CUDA_OK(cudaGetLastError());
+  tv::count_launches(1);
+  return TV_OK;
 }

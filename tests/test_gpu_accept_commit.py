@@ -155,3 +155,27 @@ def test_commit_bytes_exact(d, Hkv):
                                     nodes_bad, A_bad, S_bad)
     assert np.array_equal(kc, rk) and np.array_equal(vc, rv) and np.array_equal(S2, rS) and np.array_equal(st, rst)
     assert st.tolist() == [orc.ST_CAPACITY, 0, orc.ST_BAD_INDEX, orc.ST_BAD_INDEX, orc.ST_CAPACITY]
+
+
+def test_node_scores_parity():
+    """tree_node_scores against the oracle: bit-exact fp32 values of the gathered bf16 logits."""
+    cfg = CONFIGS[4].scaled(S_lo=1, S_hi=8, Scap=32, L=1, B=6, V=153600)
+    case = make_case(cfg, seed=77, ragged_nodes=True, with_cache=False)
+    tokens = case["tokens"].clone()
+    n = case["n_nodes"].numpy()
+    bad = [b for b in range(cfg.B) if n[b] >= 2][:2]
+    assert len(bad) == 2
+    tokens[bad[0], int(n[bad[0]]) - 1] = cfg.V          # out of range: -inf and BAD_INDEX
+    tokens[bad[1], 1] = -7
+    tokens[bad[1], int(n[bad[1]]):] = -1                # padded slots are never looked at
+    dev = "cuda"
+    scores = torch.full((cfg.B, cfg.N), 5.0, dtype=torch.float32, device=dev)
+    status = torch.zeros(cfg.B, dtype=torch.int32, device=dev)
+    tv.tree_node_scores(case["logits"].to(dev), tokens.to(dev), case["parent"].to(dev), case["n_nodes"].to(dev),
+                        scores, status)
+    torch.cuda.synchronize()
+    ref, ref_st = orc.node_scores(bf16_bits(case["logits"]), tokens.numpy(), case["parent"].numpy(),
+                                  case["n_nodes"].numpy())
+    assert np.array_equal(scores.cpu().numpy(), ref)
+    assert np.array_equal(status.cpu().numpy(), ref_st)
+    assert ref_st[bad[0]] == orc.ST_BAD_INDEX and np.isneginf(ref[bad[1], 1]) and (ref[:, 0] == 0).all()

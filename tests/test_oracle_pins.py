@@ -484,3 +484,36 @@ def test_commit_equivalence_with_sequential_decoding():
     nodes_c = np.arange(5, dtype=np.int32)[None]
     kc3, _, _, _ = orc.kv_commit(kc[None], vc[None], kt[None], vt[None], nodes_c, np.array([3]), S)
     assert (kc3[0, 0, :, 7:11] == kt[0, 0:4].transpose(1, 0, 2)).all()
+
+
+def test_node_scores_gather_and_link_to_greedy_acceptance():
+    """score[k] = logits[parent(k), token(k)]: checked against numpy fancy indexing, and against the
+    acceptance rule - a node is accepted by the greedy rule exactly when its score equals the row
+    maximum at its parent and its token is the lowest maximiser."""
+    rng = np.random.default_rng(21)
+    B, N, V = 2, 12, 300
+    parent = np.stack([random_parent_tree(N, 4, rng), random_parent_tree(N, 3, rng)])
+    n = np.array([N, 9])
+    bits = _bf16(rng.standard_normal((B, N, V)).astype(np.float32))
+    tokens = rng.integers(0, V, size=(B, N)).astype(np.int32)
+    am = orc.argmax_rows(bits, n)
+    for b in range(B):                        # make some nodes match the teacher
+        for k in (1, 3, 5):
+            tokens[b, k] = am[b, max(parent[b, k], 0)]
+    scores, st = orc.node_scores(bits, tokens, parent, n)
+    assert (st == 0).all()
+    wide = (bits.astype(np.uint32) << 16).view(np.float32)
+    for b in range(B):
+        sp = np.maximum(parent[b], 0)
+        want = wide[b, sp, tokens[b]]
+        want[0] = 0
+        want[n[b]:] = 0
+        assert np.array_equal(scores[b], want)
+        for k in range(1, n[b]):
+            is_top = scores[b, k] == wide[b, sp[k]].max()
+            assert (tokens[b, k] == am[b, sp[k]]) == (is_top and tokens[b, k] == np.flatnonzero(wide[b, sp[k]] == wide[b, sp[k]].max())[0])
+    bad = tokens.copy()
+    bad[1, 2] = V
+    bad[0, 4] = -3
+    s2, st2 = orc.node_scores(bits, bad, parent, n)
+    assert st2.tolist() == [orc.ST_BAD_INDEX] * 2 and np.isneginf(s2[1, 2]) and np.isneginf(s2[0, 4])
