@@ -9,20 +9,29 @@
 // Pipeline (one CTA per SM, 12 warps):
 //   warp 0      TMA producer: Q tiles once per work item, then K and V tiles
 //               through a 5-slot shared-memory ring (128-byte swizzled boxes).
-//   warp 1      tcgen05.mma issuer: S = Q K^T (both operands from shared
-//               memory) into TMEM, O += P V with P read from TMEM; completion
-//               is signalled to mbarriers with tcgen05.commit.
+//   warp 1      tcgen05.mma issuer (one thread): S = Q K^T for a whole 128-key
+//               tile (N = 128; 64-key MMAs re-read Q from shared memory twice as
+//               often and run at 2/3 of the rate), O += P V with P read from
+//               TMEM; completion goes to mbarriers with tcgen05.commit.  With
+//               two row tiles it serves them in turn, so the softmax of one row
+//               tile runs while the tensor pipe works for the other.
 //   warps 4-7   softmax warpgroup for row tile 0: one thread per row, online
 //   warps 8-11  softmax with lazy rescale; tile 1 likewise.  The ancestor
-//               bitmask of the row (4 words) is applied only on the tree tile,
-//               the prefix length only on the ragged last prefix tile.
-// TMEM: S0 | S1 | O0 | O1, 128 columns each; P (bf16) overlays its S.
+//               bitmask of the row is applied only on the tree tile(s), the
+//               prefix length only on the ragged last prefix tile.
+// TMEM: S0 | S1 | O0 | O1, 128 columns each; P (bf16) overlays the first 64
+// columns of its S.  With one row tile the two S buffers alternate by key tile.
+//
+// Code size matters here: instruction fetches compete with the K/V stream for
+// L2 and HBM, and code that runs once per work item (set-up, epilogue, merge)
+// is fetched cold every time.  Cold paths are therefore written as loops, not
+// unrolled, and the timeline marks are compiled out unless -DTV_TRACE is given.
 //
 // Work split.  All key tiles of all (b, hk) units form one linear space that
 // is cut evenly over the CTA groups (a group = the CTAs that hold the row
 // tiles of the same unit and walk the same keys together, so the second reader
-// hits L2).  A unit cut in pieces leaves fp32 partials (O, m, l) in the
-// workspace; the piece that arrives last on the unit's counter merges them.
+// hits L2).  A unit cut in pieces leaves partials (normalised O in bf16, m, l) in the
+// workspace; the piece that draws the last ticket on the unit's counter merges them.
 // Counters carry a per-call epoch, so the workspace needs no initialisation.
 //
 // Every wait on an mbarrier is bounded: on expiry the CTA raises
@@ -214,10 +223,21 @@ struct Tracer {
     n = 0;
   }
   __device__ __forceinline__ void mark(uint32_t tag) {
+#ifndef TV_TRACE
+    (void)tag;        // compiled out: even switched off, the marks cost several per cent of the kernel's time
+    return;
+#endif
     if (base && n < kTraceCap) base[n++] = ((unsigned long long)tag << 48) | (globaltimer_ns() & 0xffffffffffffull);
   }
 };
 
+#ifdef TV_PROF
+#define TV_PROF_T(var) do { var = clock(); } while (0)
+#define TV_PROF_USE(x) asm volatile("{.reg .b32 t; mov.b32 t, %0;}" ::"r"(x))
+#else
+#define TV_PROF_T(var) do { } while (0)
+#define TV_PROF_USE(x) do { } while (0)
+#endif
 // Packed fp32 pair arithmetic (one issue slot for two lanes of work).
 __device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) { return __ffma2_rn(a, b, c); }
 __device__ __forceinline__ float2 fadd2(float2 a, float2 b) { return __fadd2_rn(a, b); }
@@ -319,7 +339,7 @@ struct SmemLayout {
   static constexpr int kBars = kRing + kSlots * kTileBytes;
   // barrier indices (8 bytes each)
   static constexpr int Q_FULL = 0, Q_EMPTY = 1, KV_FULL = 2, KV_EMPTY = 2 + kSlots, S_FULL = 2 + 2 * kSlots,
-                       P_READY = S_FULL + 4, O_DONE = P_READY + 4, ITEM_DONE = O_DONE + 2, EPI = ITEM_DONE + 2,
+                       P_READY = S_FULL + 2, O_DONE = P_READY + 2, ITEM_DONE = O_DONE + 2, EPI = ITEM_DONE + 2,
                        NBARS = EPI + 1;
   static constexpr int kMisc = kBars + NBARS * 8;          // tmem ptr, abort flag, last flag
   static constexpr int kCum = kMisc + 16;
@@ -376,12 +396,12 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   }
   if (threadIdx.x == 32) {
     mbar_init(bar(L::Q_FULL), 1);
-    mbar_init(bar(L::Q_EMPTY), MT);
+    mbar_init(bar(L::Q_EMPTY), 1);
     for (int s = 0; s < kSlots; ++s) {
       mbar_init(bar(L::KV_FULL + s), 1);
-      mbar_init(bar(L::KV_EMPTY + s), MT);       // one commit per row tile's issuer
+      mbar_init(bar(L::KV_EMPTY + s), 1);
     }
-    for (int s = 0; s < 4; ++s) {                // index = row tile * 2 + key half
+    for (int s = 0; s < 2; ++s) {                // index = S buffer
       mbar_init(bar(L::S_FULL + s), 1);
       mbar_init(bar(L::P_READY + s), 128);
     }
@@ -449,7 +469,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     return false;
   };
 
-  constexpr uint32_t kIdescQK = instr_desc(64, false);   // S is produced 64 keys at a time
+  constexpr uint32_t kIdescQK = instr_desc(kTileN, false);
   constexpr uint32_t kIdescPV = instr_desc(D, true);
   constexpr uint32_t kTmemS0 = 0, kTmemO0 = 256;
 
@@ -504,89 +524,110 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
       }
     }
-  } else if (warp == 1 || warp == 2) {
-    // =========================================================== MMA issuers, one per row tile
-    // Row tile t is driven by warp 1 + t.  Its S region is split in two 64-key halves, so the softmax of
-    // one half overlaps the MMAs of the other: per key tile the issuer runs
-    //   wait P(h) -> O += P(h) V(h) -> S(h) = Q K_next(h)^T      for h = 0, 1.
-    // MMAs of one thread execute in issue order, which keeps S(h)/P(h) reuse safe without further waits.
+  } else if (warp == 1) {
+    // =========================================================== MMA issuer
+    // One thread issues every MMA of the CTA.  S of a key tile is a full 128-key tile (N = 128: with 64-key
+    // MMAs the Q operand is re-read from shared memory twice as often and the pipe runs at 2/3 of its rate).
+    // P overlays the first 64 columns of its S buffer, so S of the next key tile can only be computed after
+    // the PV that reads P; the tensor pipe runs MMAs in issue order, which gives that for free.
+    //   two row tiles (buffer = row tile):  wait P_t -> O_t += P_t V -> S_t = Q_t K_next^T, t = 0, 1 in turn, so
+    //     that the softmax of one row tile runs while the pipe works for the other one;
+    //   one row tile (buffers alternate by key tile):  S_next = Q K_next^T -> wait P -> O += P V.
     asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
-    const int t = warp - 1;
-    if (lane == 0 && t < MT && !*abort_flag) {
+    if (lane == 0 && !*abort_flag) {
       long long g = g_begin;
       Item it;
-      uint32_t item_idx = 0, fill = 0, hj = 0;
+      uint32_t item_idx = 0, fill = 0, tj = 0;
       bool ok = true;
       Tracer tr;
       tr.init(prm.trace, 1);
-      if (t == 0) tr.mark(0);
+      tr.mark(0);
       // descriptor words: low = start address >> 4 | LBO field, high = SBO 1024 B | version 1 | 128-byte swizzle
       const uint32_t desc_hi = (uint32_t)(smem_desc(0, 0, 1024) >> 32);
-      const uint32_t q_lo = (uint32_t)smem_desc(sbase + L::kQ + t * L::kTileBytes, 16, 1024);   // K-major: LBO unused
+      const uint32_t q_lo = (uint32_t)smem_desc(sbase + L::kQ, 16, 1024);   // K-major: LBO unused
       const uint32_t k_lo = (uint32_t)smem_desc(sbase + L::kRing, 16, 1024);
       const uint32_t v_lo = (uint32_t)smem_desc(sbase + L::kRing, L::kHalf, 1024);  // MN-major: LBO = next 64 columns
-      const uint32_t s_tmem = tmem + kTmemS0 + t * 128, o_tmem = tmem + kTmemO0 + t * 128;
       constexpr int kHalf16 = L::kHalf >> 4, kTile16 = L::kTileBytes >> 4;
-      constexpr int kHalfKeys16 = (64 * 128) >> 4;        // 64 key rows of 128 bytes
-      // S(h) = Q K(h)^T for the 64 keys of half h of the K tile in `slot`
-      auto issue_qk = [&](uint32_t slot, int h) {
-        const uint32_t ka = k_lo + slot * kTile16 + h * kHalfKeys16;
+      // S(buf) = Q_t K^T for the 128 keys of the K tile in `slot`
+      auto issue_qk = [&](int t, int buf, uint32_t slot) {
+        const uint32_t qa = q_lo + t * kTile16, ka = k_lo + slot * kTile16;
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks) {
           const uint32_t off = (ks / 4) * kHalf16 + (ks % 4) * 2;        // 16 columns = 32 bytes inside a swizzled row
-          mma_ss_lohi(s_tmem + h * 64, q_lo + off, ka + off, desc_hi, kIdescQK, ks > 0);
+          mma_ss_lohi(tmem + kTmemS0 + buf * 128, qa + off, ka + off, desc_hi, kIdescQK, ks > 0);
         }
-        mma_commit(bar(L::S_FULL + t * 2 + h));
+        mma_commit(bar(L::S_FULL + buf));
+      };
+      // O_t += P(buf) V for the 128 keys of the V tile in `slot`
+      auto issue_pv = [&](int t, int buf, uint32_t slot, bool first_tile) {
+        const uint32_t va = v_lo + slot * kTile16;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks)            // 16 keys = 16 rows of 128 bytes = 8 packed P columns
+          mma_ts_lohi(tmem + kTmemO0 + t * 128, tmem + kTmemS0 + buf * 128 + ks * 8, va + ks * 128, desc_hi, kIdescPV,
+                      (!first_tile || ks > 0) ? 1u : 0u);
+        mma_commit(bar(L::O_DONE + t));
       };
       while (ok && next_item(g, it)) {
         const int nt = it.j1 - it.j0;
         ok = mbar_wait(bar(L::Q_FULL), item_idx & 1, abort_flag);
         if (!ok) break;
-        if (t == 0) tr.mark(0x1000u | item_idx);
+        tr.mark(0x1000u | item_idx);
         {
           const uint32_t slot = fill % kSlots;
           ok = mbar_wait(bar(L::KV_FULL + slot), (fill / kSlots) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
-          issue_qk(slot, 0);
-          issue_qk(slot, 1);
+          if (MT == 2) {
+            issue_qk(0, 0, slot);
+            issue_qk(1, 1, slot);
+          } else {
+            issue_qk(0, tj & 1, slot);
+          }
           mma_commit(bar(L::KV_EMPTY + slot));
           if (nt == 1) mma_commit(bar(L::Q_EMPTY));
         }
-        for (int jt = 0; jt < nt && ok; ++jt) {
+        for (int jt = 0; jt < nt && ok; ++jt, ++tj) {
           const uint32_t fv = fill + 2 * jt + 1, vslot = fv % kSlots;
           const uint32_t fk = fv + 1, kslot = fk % kSlots;
-          ok = mbar_wait(bar(L::KV_FULL + vslot), (fv / kSlots) & 1, abort_flag);
-          if (!ok) break;
-          const uint32_t va = v_lo + vslot * kTile16;
+          const bool more = jt + 1 < nt;
+          if (MT == 2) {
 #pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            ok = mbar_wait(bar(L::P_READY + t * 2 + h), (hj >> 1) & 1, abort_flag);
+            for (int t = 0; t < 2; ++t) {
+              ok = mbar_wait(bar(L::P_READY + t), tj & 1, abort_flag);
+              if (!ok) break;
+              if (t == 0) {
+                ok = mbar_wait(bar(L::KV_FULL + vslot), (fv / kSlots) & 1, abort_flag);
+                if (ok && more) ok = mbar_wait(bar(L::KV_FULL + kslot), (fk / kSlots) & 1, abort_flag);
+                if (!ok) break;
+              }
+              tc_fence_after();
+              tr.mark(0x4000u | ((2 * tj + t) & 0xfffu));
+              issue_pv(t, t, vslot, jt == 0);
+              if (!more) mma_commit(bar(L::ITEM_DONE + t));      // all MMAs of the item's row tile are done
+              if (more) issue_qk(t, t, kslot);
+              tr.mark(0x2000u | ((2 * tj + t) & 0xfffu));
+            }
+            if (!ok) break;
+          } else {
+            const int buf = tj & 1;
+            if (more) {
+              ok = mbar_wait(bar(L::KV_FULL + kslot), (fk / kSlots) & 1, abort_flag);
+              if (!ok) break;
+              tc_fence_after();
+              issue_qk(0, buf ^ 1, kslot);
+            }
+            ok = mbar_wait(bar(L::P_READY + buf), (tj >> 1) & 1, abort_flag);
+            if (ok) ok = mbar_wait(bar(L::KV_FULL + vslot), (fv / kSlots) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
-            if (t == 0) tr.mark(0x4000u | (hj & 0xfffu));
-#pragma unroll
-            for (int ks = 0; ks < 4; ++ks)          // 16 keys = 16 rows of 128 bytes; P(h) starts 64 columns into S
-              mma_ts_lohi(o_tmem, s_tmem + h * 64 + ks * 8, va + (h * 4 + ks) * 128, desc_hi, kIdescPV,
-                          (jt > 0 || h > 0 || ks > 0) ? 1u : 0u);
-            mma_commit(bar(L::O_DONE + t));
-            if (h == 1) mma_commit(bar(L::KV_EMPTY + vslot));
-            if (h == 1 && jt + 1 == nt) mma_commit(bar(L::ITEM_DONE + t));   // all MMAs of the item are done
-            if (jt + 1 < nt) {
-              if (h == 0) {
-                ok = mbar_wait(bar(L::KV_FULL + kslot), (fk / kSlots) & 1, abort_flag);
-                if (!ok) break;
-                tc_fence_after();
-              }
-              issue_qk(kslot, h);
-              if (h == 1) {
-                mma_commit(bar(L::KV_EMPTY + kslot));
-                if (jt + 2 == nt) mma_commit(bar(L::Q_EMPTY));
-              }
-            }
-            if (t == 0) tr.mark(0x2000u | (hj & 0xfffu));
-            ++hj;
+            tr.mark(0x4000u | (tj & 0xfffu));
+            issue_pv(0, buf, vslot, jt == 0);
+            if (!more) mma_commit(bar(L::ITEM_DONE));
+            tr.mark(0x2000u | (tj & 0xfffu));
           }
+          mma_commit(bar(L::KV_EMPTY + vslot));
+          if (more) mma_commit(bar(L::KV_EMPTY + kslot));
+          if (jt + 2 == nt) mma_commit(bar(L::Q_EMPTY));
         }
         fill += 2 * nt;
         ++item_idx;
@@ -602,11 +643,16 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     if (wg_active && !*abort_flag) {
       long long g = g_begin;
       Item it;
-      uint32_t fill = 0, hj = 0, epi_phase = 0, item_cnt = 0;
+      uint32_t fill = 0, tj = 0, epi_phase = 0, item_cnt = 0;   // tj: key tiles handled so far (all items)
       bool ok = true;
       Tracer tr;
       tr.init((threadIdx.x & 127) == 0 ? prm.trace : nullptr, 2 + wg);
       tr.mark(0);
+#ifdef TV_PROF
+      unsigned int prof[6] = {0u, 0u, 0u, 0u, 0u, 0u}, pc0 = 0, pc1 = 0, pc2 = 0, pend = 0;
+      const long long prof_c0 = clock64();
+      const unsigned long long prof_g0 = globaltimer_ns();   // cycles: wait S, ld, compute, hand-over; tiles
+#endif
       // Rendezvous of the softmax warpgroups through an mbarrier, so that it is bounded like every other wait.
       // All 32 lanes wait together and agree on the outcome, so that the warp-wide TMEM instructions
       // below are never executed by a part of a warp.
@@ -641,9 +687,8 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         unsigned long long claim_assumed = 0, claim_ret = 1;
         int claim_cnt = 0;
         if (piece && threadIdx.x == 128) claim_assumed = *reinterpret_cast<volatile unsigned long long*>(claim_ctr);
-        const uint32_t s_base = tmem + lane_addr + kTmemS0 + wg * 128;
         const uint32_t o_addr_loop = tmem + lane_addr + kTmemO0 + wg * 128;
-        for (int jt = 0; jt < nt && ok; ++jt) {
+        for (int jt = 0; jt < nt && ok; ++jt, ++tj) {
           const int j = it.j0 + jt;
           const int tt = j - (it.len - prm.TT);      // >= 0: index of the tree key tile
           const bool tree = tt >= 0;
@@ -668,41 +713,63 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             }
             fence_proxy_async_smem();
           }
+          // S buffer of this key tile: the row tile's own one, or alternating by key tile when the CTA has one
+          // row tile; its barriers complete once per use of the buffer.
+          const int buf = (MT == 2) ? wg : (int)(tj & 1u);
+          const uint32_t use_par = (MT == 2) ? (tj & 1u) : ((tj >> 1) & 1u);
+          const uint32_t s_base = tmem + lane_addr + kTmemS0 + buf * 128;
+          tr.mark(0x0800u | (tj & 0x7ffu));
+          TV_PROF_T(pc0);
+#ifdef TV_PROF
+          if (jt > 0) prof[5] += pc0 - pend;
+#endif
+          ok = wwait(bar(L::S_FULL + buf), use_par);
+          if (!ok) break;
+          tc_fence_after();
+          TV_PROF_T(pc1);
+#ifdef TV_PROF
+          prof[0] += pc1 - pc0;
+#endif
+          tr.mark(0x1000u | (tj & 0xfffu));
 #pragma unroll
           for (int h = 0; h < 2; ++h) {
             const int valid_half = min(64, max(0, valid_keys - 64 * h));
-            tr.mark(0x0800u | (hj & 0x7ffu));
-            ok = wwait(bar(L::S_FULL + wg * 2 + h), (hj >> 1) & 1);
-            if (!ok) break;
-            tc_fence_after();
-            tr.mark(0x1000u | (hj & 0xfffu));
             uint32_t sreg[64];
             const uint32_t s_addr = s_base + h * 64;
+            TV_PROF_T(pc0);
             tmem_ld32(s_addr, sreg);
             tmem_ld32(s_addr + 32, sreg + 32);
             tmem_wait_ld();
+            TV_PROF_USE(sreg[31]);
+            TV_PROF_USE(sreg[63]);
+            TV_PROF_T(pc1);
             float* s = reinterpret_cast<float*>(sreg);
-            if (valid_half < 64 || tree) {
+            const bool masked = tree || valid_half < 64;
+            if (masked) {
+              // two 32-bit words of this chunk: ancestor bits on a tree tile, a length mask on the ragged tile
+              uint32_t w0, w1;
+              if (tree) {
+                const uint32_t a0 = tt > 0 ? anc[4] : anc[0], a1 = tt > 0 ? anc[5] : anc[1];
+                const uint32_t a2 = tt > 0 ? anc[6] : anc[2], a3 = tt > 0 ? anc[7] : anc[3];
+                w0 = h ? a2 : a0;
+                w1 = h ? a3 : a1;
+              } else {
+                w0 = valid_half >= 32 ? 0xffffffffu : ((1u << valid_half) - 1u);
+                w1 = valid_half >= 64 ? 0xffffffffu : (valid_half <= 32 ? 0u : ((1u << (valid_half - 32)) - 1u));
+              }
 #pragma unroll
-              for (int q = 0; q < 2; ++q) {
-                uint32_t word;
-                if (tree) {
-                  word = (tt > 0) ? anc[4 + 2 * h + q] : anc[2 * h + q];
-                } else {
-                  const int cnt = valid_half - 32 * q;
-                  word = cnt >= 32 ? 0xffffffffu : (cnt <= 0 ? 0u : ((1u << cnt) - 1u));
-                }
-#pragma unroll
-                for (int c = 0; c < 32; ++c)
-                  if (!((word >> c) & 1u)) s[q * 32 + c] = -INFINITY;
+              for (int c = 0; c < 32; ++c) {
+                if (!((w0 >> c) & 1u)) s[c] = -INFINITY;
+                if (!((w1 >> c) & 1u)) s[32 + c] = -INFINITY;
               }
             }
-            uint32_t pk[32];                 // P of this half, bf16 pairs
+            uint32_t pk[32];                 // P of this chunk, bf16 pairs
             const bool first = (jt == 0 && h == 0);
-            bool need_slow = true;
-            // ---- fast path (full, unmasked halves after the first): keep the reference maximum, compute
-            // P directly and only check afterwards that nothing overflowed the lazy-rescale range.
-            if (!first && !tree && valid_half == 64) {
+            // Full, unmasked chunks after the first keep the reference maximum, compute P directly and only
+            // check afterwards (from the row sum) that nothing left the lazy-rescale range.  Every other
+            // chunk, and a chunk that fails the check, takes the true maximum first.
+            bool with_max = first || masked;
+            if (!with_max) {
               const float2 c2 = make_float2(prm.scale_log2e, prm.scale_log2e);
               const float nm = (m_used == -INFINITY) ? 0.f : -m_used;
               const float2 nm2 = make_float2(nm, nm);
@@ -711,6 +778,11 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               for (int i = 0; i < 32; ++i) {
                 const float2 x = ffma2(make_float2(s[2 * i], s[2 * i + 1]), c2, nm2);
                 float2 pv;
+#ifdef TV_EXP_SKIP_EXP
+                if (true) {
+                  pv = x;
+                } else
+#endif
                 if (TV_POLY_SEL(i)) {
                   pv = exp2_poly2(x);
                 } else {
@@ -726,10 +798,11 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               const bool overflow = row_active && !(fsum <= kMaxFastSum);
               if (!__any_sync(0xffffffffu, overflow)) {
                 l_sum += fsum;
-                need_slow = false;
+              } else {
+                with_max = true;
               }
             }
-            if (need_slow) {
+            if (with_max) {
               float mx0 = s[0], mx1 = s[1], mx2_ = s[2], mx3 = s[3];
 #pragma unroll
               for (int c = 4; c < 64; c += 4) {
@@ -748,12 +821,12 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               if (moves) m_used = mx2;
               l_sum *= alpha;
               if (__any_sync(0xffffffffu, scales)) {
-                tr.mark(0x9000u | (hj & 0xfffu));
-                // the PV of the previous half may still be running: wait for its completion (number hj - 1)
-                ok = wwait(bar(L::O_DONE + wg), (hj - 1) & 1);
+                tr.mark(0x9000u | (tj & 0xfffu));
+                // the PV of the previous key tile may still be running: wait for its completion (number tj - 1)
+                ok = wwait(bar(L::O_DONE + wg), (tj - 1) & 1);
                 if (!ok) break;
                 tc_fence_after();
-#pragma unroll
+#pragma unroll 1
                 for (int q = 0; q < D / 32; ++q) {
                   uint32_t o[32];
                   tmem_ld32(o_addr_loop + q * 32, o);
@@ -763,7 +836,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                   tmem_st32(o_addr_loop + q * 32, o);
                 }
               }
-              // ---- P = exp2(s * c - m), row sum in fp32, P rounded to bf16
+              // ---- P = exp2(s * c - m), row sum in fp32, P rounded to bf16 (masked scores give exactly 0)
               const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
               float ls0 = 0.f, ls1 = 0.f;
 #pragma unroll
@@ -776,20 +849,36 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               }
               l_sum += ls0 + ls1;
             }
-            // ---- P into TMEM over the start of S(h): 16 keys = 8 packed columns per store
+            if (!ok) break;
+            TV_PROF_USE(pk[31]);
+            TV_PROF_USE(pk[15]);
+            TV_PROF_USE(__float_as_uint(l_sum));
+            TV_PROF_T(pc2);
+#ifdef TV_PROF
+            prof[1] += pc1 - pc0;
+            prof[2] += pc2 - pc1;
+#endif
+            // ---- P over the start of the S buffer (columns already read): 16 keys = 8 packed columns per store
 #pragma unroll
             for (int q = 0; q < 4; ++q)
               asm volatile(
                   "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
-                  ::"r"(s_addr + q * 8), "r"(pk[q * 8 + 0]), "r"(pk[q * 8 + 1]), "r"(pk[q * 8 + 2]), "r"(pk[q * 8 + 3]),
+                  ::"r"(s_base + h * 32 + q * 8), "r"(pk[q * 8 + 0]), "r"(pk[q * 8 + 1]), "r"(pk[q * 8 + 2]), "r"(pk[q * 8 + 3]),
                     "r"(pk[q * 8 + 4]), "r"(pk[q * 8 + 5]), "r"(pk[q * 8 + 6]), "r"(pk[q * 8 + 7])
                   : "memory");
-            tmem_wait_st();
-            tc_fence_before();
-            mbar_arrive(bar(L::P_READY + wg * 2 + h));
-            tr.mark(0x2000u | (hj & 0xfffu));
-            ++hj;
           }
+          if (!ok) break;
+          TV_PROF_T(pc0);
+          tmem_wait_st();
+          tc_fence_before();
+          mbar_arrive(bar(L::P_READY + buf));
+          TV_PROF_T(pc1);
+#ifdef TV_PROF
+          prof[3] += pc1 - pc0;
+          prof[4] += 1;
+          pend = pc1;
+#endif
+          tr.mark(0x2000u | (tj & 0xfffu));
         }
         if (!ok) break;
         // ---- epilogue of the item: wait for the last PV into this O buffer
@@ -807,14 +896,15 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           const int h = it.hk * prm.G + gm;
           tv_bf16* orow = prm.out + (((size_t)it.b * prm.Nmax + node) * prm.Hq + h) * D;
           float* lse_p = prm.lse ? prm.lse + ((size_t)it.b * prm.Hq + h) * prm.Nmax + node : nullptr;
-          if (whole) {
-            const float inv = (row_active && l_sum > 0.f) ? 1.f / l_sum : 0.f;
-#pragma unroll
+          // Normalised bf16 output of this row, 32 columns at a time (one copy of the loop for every use: the
+          // epilogue is cold code, fetched while the other CTAs still stream K/V).
+          auto store_rows = [&](uint4* dst, size_t stride_u4, float inv, bool do_store, bool zero) {
+#pragma unroll 1
             for (int q = 0; q < D / 32; ++q) {
               uint32_t o[32];
               tmem_ld32(o_addr + q * 32, o);
               tmem_wait_ld();
-              if (row_exists) {
+              if (do_store) {
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                   uint4 v;
@@ -822,11 +912,15 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                   v.y = pack_bf16(__uint_as_float(o[8 * c + 2]) * inv, __uint_as_float(o[8 * c + 3]) * inv);
                   v.z = pack_bf16(__uint_as_float(o[8 * c + 4]) * inv, __uint_as_float(o[8 * c + 5]) * inv);
                   v.w = pack_bf16(__uint_as_float(o[8 * c + 6]) * inv, __uint_as_float(o[8 * c + 7]) * inv);
-                  if (!row_active) v = make_uint4(0, 0, 0, 0);
-                  *reinterpret_cast<uint4*>(orow + q * 32 + c * 8) = v;
+                  if (zero) v = make_uint4(0, 0, 0, 0);       // rows of padded nodes: O may hold anything
+                  dst[(size_t)(q * 4 + c) * stride_u4] = v;
                 }
               }
             }
+          };
+          if (whole) {
+            const float inv = (row_active && l_sum > 0.f) ? 1.f / l_sum : 0.f;
+            store_rows(reinterpret_cast<uint4*>(orow), 1, inv, row_exists, !row_active);
             if (row_exists && lse_p)
               *lse_p = (row_active && l_sum > 0.f) ? (m_used + log2f(l_sum)) / kLog2e : -INFINITY;
             tc_fence_before();
@@ -902,23 +996,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             if (!*last_flag) {
               uint4* po = reinterpret_cast<uint4*>(prm.part_o) + (size_t)my_slot * (D / 8) * kRows;
               float* pml = prm.part_ml + (size_t)my_slot * 2 * kRows;
-#pragma unroll
-              for (int q = 0; q < D / 32; ++q) {
-                uint32_t o[32];
-                tmem_ld32(o_addr + q * 32, o);
-                tmem_wait_ld();
-                if (row_active) {
-#pragma unroll
-                  for (int c = 0; c < 4; ++c) {
-                    uint4 v;
-                    v.x = pack_bf16(__uint_as_float(o[8 * c + 0]) * inv_own, __uint_as_float(o[8 * c + 1]) * inv_own);
-                    v.y = pack_bf16(__uint_as_float(o[8 * c + 2]) * inv_own, __uint_as_float(o[8 * c + 3]) * inv_own);
-                    v.z = pack_bf16(__uint_as_float(o[8 * c + 4]) * inv_own, __uint_as_float(o[8 * c + 5]) * inv_own);
-                    v.w = pack_bf16(__uint_as_float(o[8 * c + 6]) * inv_own, __uint_as_float(o[8 * c + 7]) * inv_own);
-                    po[(size_t)(q * 4 + c) * kRows + rr] = v;
-                  }
-                }
-              }
+              store_rows(po + rr, kRows, inv_own, row_active, false);
               if (row_active) {
                 pml[rr] = m_used;
                 pml[kRows + rr] = l_sum;
@@ -933,140 +1011,79 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 bump_counter(ctr + 1, seen, prm.epoch);
               }
             } else {
+              // ---- pass 1: reference maximum and total weight of the row, pieces in order.  Loads are issued
+              // by every thread (row rr always lies inside a slot; rows that are not active read stale bytes
+              // and are masked by selects): no thread-divergent branch sits between the warp-wide TMEM ops.
               float mm = m_used, lt = 0.f;
-              if (n_other <= 2) {
-                // ---- up to two other pieces (the usual cases): everything of a batch is requested before
-                // anything is used, two dependent round trips to L2 in total.  Loads are issued by every
-                // thread (row rr always lies inside a slot; rows that are not active read stale bytes and
-                // are masked by selects): no thread-divergent branch sits between the warp-wide TMEM ops.
-                if (n_other == 1) sid_b = sid_a;
-                const float* ml_a = prm.part_ml + (size_t)sid_a * 2 * kRows;
-                const float* ml_b = prm.part_ml + (size_t)sid_b * 2 * kRows;
-                const uint4* o_a = reinterpret_cast<const uint4*>(prm.part_o) + (size_t)sid_a * (D / 8) * kRows;
-                const uint4* o_b = reinterpret_cast<const uint4*>(prm.part_o) + (size_t)sid_b * (D / 8) * kRows;
-                const float m_a = __ldcg(ml_a + rr), l_a = __ldcg(ml_a + kRows + rr);
-                const float m_b = (n_other == 2) ? __ldcg(ml_b + rr) : -INFINITY;
-                const float l_b = (n_other == 2) ? __ldcg(ml_b + kRows + rr) : 0.f;
-                float w_o = 0.f, w_a = 0.f, w_b = 0.f, inv = 0.f;
-                // ordered combination of (own, a, b) by the position of the own piece inside the unit
-                auto comb = [&](float vo, float va, float vb) -> float {
-                  if (own_pos == 0) return fmaf(w_b, vb, fmaf(w_a, va, w_o * vo));
-                  if (own_pos == 1) return fmaf(w_b, vb, fmaf(w_o, vo, w_a * va));
-                  return fmaf(w_o, vo, fmaf(w_b, vb, w_a * va));
-                };
+              for (int k = k_first; k <= k_last; ++k) {
+                const int sid = piece_slot(k);
+                if (sid < 0 || sid == my_slot) continue;
+                mm = fmaxf(mm, __ldcg(prm.part_ml + (size_t)sid * 2 * kRows + rr));
+              }
+              for (int k = k_first; k <= k_last; ++k) {
+                const int sid = piece_slot(k);
+                if (sid < 0) continue;
+                if (sid == my_slot) {
+                  lt = fmaf(l_sum * fast_exp2(m_used - mm), 1.f, lt);
+                } else {
+                  const float* q_ml = prm.part_ml + (size_t)sid * 2 * kRows;
+                  lt = fmaf(__ldcg(q_ml + kRows + rr) * fast_exp2(__ldcg(q_ml + rr) - mm), 1.f, lt);
+                }
+              }
+              if (!row_active) lt = 0.f;
+              const float inv = (row_active && lt > 0.f) ? 1.f / lt : 0.f;
+              const float w_own = l_sum * fast_exp2(m_used - mm);
+              // ---- pass 2: 64 output columns at a time, pieces in order (one fused multiply-add per piece and
+              // element); the own piece comes from TMEM and enters as its bf16-rounded normalised output
+#pragma unroll 1
+              for (int hq = 0; hq < D / 64; ++hq) {
+                float acc[64];
 #pragma unroll
-                for (int half = 0; half < D / 64; ++half) {
-                  uint4 va[8], vb[8];
+                for (int c = 0; c < 64; ++c) acc[c] = 0.f;
+                for (int k = k_first; k <= k_last; ++k) {
+                  const int sid = piece_slot(k);
+                  if (sid < 0) continue;
+                  if (sid == my_slot) {
+#pragma unroll
+                    for (int q = 0; q < 2; ++q) {
+                      uint32_t o[32];
+                      tmem_ld32(o_addr + (hq * 2 + q) * 32, o);
+                      tmem_wait_ld();
+#pragma unroll
+                      for (int c = 0; c < 16; ++c) {
+                        const uint32_t own = pack_bf16(__uint_as_float(o[2 * c]) * inv_own, __uint_as_float(o[2 * c + 1]) * inv_own);
+                        acc[q * 32 + 2 * c] = fmaf(w_own, __uint_as_float(own << 16), acc[q * 32 + 2 * c]);
+                        acc[q * 32 + 2 * c + 1] = fmaf(w_own, __uint_as_float(own & 0xffff0000u), acc[q * 32 + 2 * c + 1]);
+                      }
+                    }
+                    continue;
+                  }
+                  const float* q_ml = prm.part_ml + (size_t)sid * 2 * kRows;
+                  const uint4* q_o = reinterpret_cast<const uint4*>(prm.part_o) + (size_t)sid * (D / 8) * kRows;
+                  uint4 v[8];
+#pragma unroll
+                  for (int c = 0; c < 8; ++c) v[c] = __ldcg(q_o + (size_t)(hq * 8 + c) * kRows + rr);
+                  const float w = __ldcg(q_ml + kRows + rr) * fast_exp2(__ldcg(q_ml + rr) - mm);
 #pragma unroll
                   for (int c = 0; c < 8; ++c) {
-                    va[c] = __ldcg(o_a + (size_t)(half * 8 + c) * kRows + rr);
-                    vb[c] = __ldcg(o_b + (size_t)(half * 8 + c) * kRows + rr);
-                  }
-                  if (half == 0) {
-                    mm = fmaxf(m_used, fmaxf(m_a, m_b));
-                    w_o = row_active ? l_sum * fast_exp2(m_used - mm) : 0.f;
-                    w_a = row_active ? l_a * fast_exp2(m_a - mm) : 0.f;
-                    w_b = (row_active && n_other == 2) ? l_b * fast_exp2(m_b - mm) : 0.f;
-                    lt = comb(1.f, 1.f, 1.f);
-                    inv = (row_active && lt > 0.f) ? 1.f / lt : 0.f;
-                  }
+                    const uint32_t wv[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
 #pragma unroll
-                  for (int q = 0; q < 2; ++q) {
-                    uint32_t o[32];
-                    tmem_ld32(o_addr + (half * 2 + q) * 32, o);
-                    tmem_wait_ld();
-                    if (row_exists) {
-#pragma unroll
-                      for (int c = 0; c < 4; ++c) {
-                        const uint4 pa = va[q * 4 + c], pb = vb[q * 4 + c];
-                        const uint32_t wa[4] = {pa.x, pa.y, pa.z, pa.w}, wb[4] = {pb.x, pb.y, pb.z, pb.w};
-                        uint32_t pk[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                          // the own piece enters as its bf16-rounded normalised output, like every other piece
-                          const uint32_t own = pack_bf16(__uint_as_float(o[c * 8 + 2 * e]) * inv_own,
-                                                         __uint_as_float(o[c * 8 + 2 * e + 1]) * inv_own);
-                          const float r0 = comb(__uint_as_float(own << 16), __uint_as_float(wa[e] << 16),
-                                                (n_other == 2) ? __uint_as_float(wb[e] << 16) : 0.f);
-                          const float r1 = comb(__uint_as_float(own & 0xffff0000u), __uint_as_float(wa[e] & 0xffff0000u),
-                                                (n_other == 2) ? __uint_as_float(wb[e] & 0xffff0000u) : 0.f);
-                          pk[e] = row_active ? pack_bf16(r0 * inv, r1 * inv) : 0u;
-                        }
-                        *reinterpret_cast<uint4*>(orow + (half * 2 + q) * 32 + c * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                      }
+                    for (int e = 0; e < 4; ++e) {
+                      acc[8 * c + 2 * e] = fmaf(w, __uint_as_float(wv[e] << 16), acc[8 * c + 2 * e]);
+                      acc[8 * c + 2 * e + 1] = fmaf(w, __uint_as_float(wv[e] & 0xffff0000u), acc[8 * c + 2 * e + 1]);
                     }
                   }
                 }
-              } else {
-                // ---- any number of pieces: pass 1, reference maximum and total weight of the row
-                if (row_active) {
-                  for (int k = k_first; k <= k_last; ++k) {
-                    const int sid = piece_slot(k);
-                    if (sid < 0 || sid == my_slot) continue;
-                    mm = fmaxf(mm, __ldcg(prm.part_ml + (size_t)sid * 2 * kRows + rr));
-                  }
-                  for (int k = k_first; k <= k_last; ++k) {
-                    const int sid = piece_slot(k);
-                    if (sid < 0) continue;
-                    if (sid == my_slot) {
-                      lt = fmaf(l_sum * fast_exp2(m_used - mm), 1.f, lt);
-                    } else {
-                      const float* q_ml = prm.part_ml + (size_t)sid * 2 * kRows;
-                      lt = fmaf(__ldcg(q_ml + kRows + rr) * fast_exp2(__ldcg(q_ml + rr) - mm), 1.f, lt);
-                    }
-                  }
-                }
-                const float inv = (row_active && lt > 0.f) ? 1.f / lt : 0.f;
-                const float w_own = row_active ? l_sum * fast_exp2(m_used - mm) : 0.f;
-                // ---- pass 2: 32 output columns at a time, pieces in order; the own piece comes from TMEM
-#pragma unroll 1
-                for (int q = 0; q < D / 32; ++q) {
-                  uint32_t o[32];
-                  tmem_ld32(o_addr + q * 32, o);
-                  tmem_wait_ld();
-                  float acc[32];
+                if (row_exists) {
 #pragma unroll
-                  for (int c = 0; c < 32; ++c) acc[c] = 0.f;
-                  if (row_active) {
-                    for (int k = k_first; k <= k_last; ++k) {
-                      const int sid = piece_slot(k);
-                      if (sid < 0) continue;
-                      if (sid == my_slot) {
-#pragma unroll
-                        for (int c = 0; c < 16; ++c) {
-                          const uint32_t own = pack_bf16(__uint_as_float(o[2 * c]) * inv_own, __uint_as_float(o[2 * c + 1]) * inv_own);
-                          acc[2 * c] = fmaf(w_own, __uint_as_float(own << 16), acc[2 * c]);
-                          acc[2 * c + 1] = fmaf(w_own, __uint_as_float(own & 0xffff0000u), acc[2 * c + 1]);
-                        }
-                        continue;
-                      }
-                      const float* q_ml = prm.part_ml + (size_t)sid * 2 * kRows;
-                      const float w = __ldcg(q_ml + kRows + rr) * fast_exp2(__ldcg(q_ml + rr) - mm);
-                      const uint4* q_o = reinterpret_cast<const uint4*>(prm.part_o) + (size_t)sid * (D / 8) * kRows;
-                      uint4 v[4];
-#pragma unroll
-                      for (int c = 0; c < 4; ++c) v[c] = __ldcg(q_o + (size_t)(q * 4 + c) * kRows + rr);
-#pragma unroll
-                      for (int c = 0; c < 4; ++c) {
-                        const uint32_t wv[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                          acc[8 * c + 2 * e] = fmaf(w, __uint_as_float(wv[e] << 16), acc[8 * c + 2 * e]);
-                          acc[8 * c + 2 * e + 1] = fmaf(w, __uint_as_float(wv[e] & 0xffff0000u), acc[8 * c + 2 * e + 1]);
-                        }
-                      }
-                    }
-                  }
-                  if (row_exists) {
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                      uint4 v;
-                      v.x = pack_bf16(acc[8 * c + 0] * inv, acc[8 * c + 1] * inv);
-                      v.y = pack_bf16(acc[8 * c + 2] * inv, acc[8 * c + 3] * inv);
-                      v.z = pack_bf16(acc[8 * c + 4] * inv, acc[8 * c + 5] * inv);
-                      v.w = pack_bf16(acc[8 * c + 6] * inv, acc[8 * c + 7] * inv);
-                      *reinterpret_cast<uint4*>(orow + q * 32 + c * 8) = v;
-                    }
+                  for (int c = 0; c < 8; ++c) {
+                    uint4 v;
+                    v.x = pack_bf16(acc[8 * c + 0] * inv, acc[8 * c + 1] * inv);
+                    v.y = pack_bf16(acc[8 * c + 2] * inv, acc[8 * c + 3] * inv);
+                    v.z = pack_bf16(acc[8 * c + 4] * inv, acc[8 * c + 5] * inv);
+                    v.w = pack_bf16(acc[8 * c + 6] * inv, acc[8 * c + 7] * inv);
+                    if (!row_active) v = make_uint4(0, 0, 0, 0);
+                    *reinterpret_cast<uint4*>(orow + hq * 64 + c * 8) = v;
                   }
                 }
               }
@@ -1080,6 +1097,14 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         tr.mark(0x8000u);
         fill += 2 * nt;
       }
+#ifdef TV_PROF
+      if (tr.base)
+      {
+        for (int i = 0; i < 6; ++i) tr.base[kTraceCap - 8 + i] = prof[i];
+        tr.base[kTraceCap - 2] = clock64() - prof_c0;
+        tr.base[kTraceCap - 1] = globaltimer_ns() - prof_g0;
+      }
+#endif
     }
   } else {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
@@ -1195,8 +1220,9 @@ cudaError_t launch(const Geometry& g, const CUtensorMap* maps, const AttnParams&
 
 }  // namespace
 
-// Tuning aid: while a device buffer of 160*4*256 u64 is registered here, every tree_verify_attn launch
-// records a per-CTA, per-role timeline (tag << 48 | globaltimer ns) into it.  NULL switches it off.
+// Tuning aid, live only in a library built with -DTV_TRACE: while a device buffer of 160*4*256 u64 is
+// registered here, every tree_verify_attn launch records a per-CTA, per-role timeline (tag << 48 |
+// globaltimer ns) into it.  NULL switches it off.
 extern "C" TV_API void tv_debug_set_attn_trace(unsigned long long* device_buffer) {
   g_trace.store(device_buffer, std::memory_order_relaxed);
 }
