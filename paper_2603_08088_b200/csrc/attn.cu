@@ -120,10 +120,13 @@ __device__ __forceinline__ void fence_proxy_async_smem() {
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
+// Tiled TMA loads.  The 3D one carries an L2 eviction-priority hint: the committed K/V prefix is read once per
+// launch, and letting it leave L2 first keeps Q, the partials and the kernel's own code resident.
+__device__ __forceinline__ void tma_load_3d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
+                                                 uint64_t policy) {
   asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5}], [%2], %6;"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "l"(policy)
       : "memory");
 }
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
@@ -310,9 +313,9 @@ struct Sched {
   const int* cum;    // cum[b] = sum over b' < b of (len_b' + kSetupCost)
   const int* gs;     // gs[k] = first virtual tile of CTA group k, gs[groups] = total
   int B, Hkv;
-  long long total;   // Hkv * cum[B]
-  __device__ __forceinline__ long long group_start(int k, int) const { return gs[k]; }
-  __device__ __forceinline__ int find_group(long long pos, int groups) const {
+  int total;         // Hkv * cum[B]; the host refuses problems whose tile count does not fit 31 bits
+  __device__ __forceinline__ int group_start(int k, int) const { return gs[k]; }
+  __device__ __forceinline__ int find_group(int pos, int groups) const {
     int lo = 0, hi = groups - 1;   // largest k with gs[k] <= pos
     while (lo < hi) {
       const int mid = (lo + hi + 1) >> 1;
@@ -320,11 +323,11 @@ struct Sched {
     }
     return lo;
   }
-  __device__ __forceinline__ int find_b(long long g) const {
+  __device__ __forceinline__ int find_b(int g) const {
     int lo = 0, hi = B - 1;   // largest b with Hkv*cum[b] <= g
     while (lo < hi) {
       const int mid = (lo + hi + 1) >> 1;
-      if ((long long)Hkv * cum[mid] <= g) lo = mid; else hi = mid - 1;
+      if (Hkv * cum[mid] <= g) lo = mid; else hi = mid - 1;
     }
     return lo;
   }
@@ -375,6 +378,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   }
   if (warp == 0) {
     int run = 0;
+#pragma unroll 1
     for (int base = 0; base < prm.B; base += 32) {
       const int b = base + lane;
       int len = 0;
@@ -397,6 +401,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   if (threadIdx.x == 32) {
     mbar_init(bar(L::Q_FULL), 1);
     mbar_init(bar(L::Q_EMPTY), 1);
+#pragma unroll 1
     for (int s = 0; s < kSlots; ++s) {
       mbar_init(bar(L::KV_FULL + s), 1);
       mbar_init(bar(L::KV_EMPTY + s), 1);
@@ -427,30 +432,33 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   // write and a merge) and every group still gets a worthwhile share of tiles.
   int groups;
   {
-    const long long total = (long long)prm.Hkv * cum[prm.B];
-    const long long want = total / kMinVirtualTilesPerGroup;
-    groups = want < 1 ? 1 : (want < prm.groups ? (int)want : prm.groups);
+    const unsigned total = (unsigned)(prm.Hkv * cum[prm.B]);
+    const unsigned want = total / (unsigned)kMinVirtualTilesPerGroup;
+    groups = want < 1u ? 1 : (want < (unsigned)prm.groups ? (int)want : prm.groups);
+    // gs[k] = floor(total * k / groups) in 32-bit arithmetic: total = q * groups + r
+    const unsigned q = total / (unsigned)groups, r = total % (unsigned)groups;
+#pragma unroll 1
     for (int k = threadIdx.x; k <= prm.groups; k += kThreads)
-      gs[k] = k <= groups ? (int)((total * k) / groups) : (int)total;
+      gs[k] = k <= groups ? (int)(k * q + (k * r) / (unsigned)groups) : (int)total;
   }
   __syncthreads();
 
-  Sched sch{cum, gs, prm.B, prm.Hkv, (long long)prm.Hkv * cum[prm.B]};
+  Sched sch{cum, gs, prm.B, prm.Hkv, prm.Hkv * cum[prm.B]};
   const int group = blockIdx.x / prm.NP;
   const int pair = blockIdx.x % prm.NP;
-  const long long g_begin = sch.group_start(group, groups);        // groups past the last used one get an empty range
-  const long long g_end = sch.group_start(group + 1, groups);
+  const int g_begin = sch.group_start(group, groups);        // groups past the last used one get an empty range
+  const int g_end = sch.group_start(group + 1, groups);
 
   // Walks the items of this CTA's range; identical in every role.
-  auto next_item = [&](long long& g, Item& it) -> bool {
+  auto next_item = [&](int& g, Item& it) -> bool {
     while (g < g_end) {
       const int b = sch.find_b(g);
       const int lenv = cum[b + 1] - cum[b];                       // setup region + real tiles
-      const long long local = g - (long long)prm.Hkv * cum[b];
-      const int hk = (int)(local / lenv);
-      const int r0 = (int)(local % lenv);
-      const long long room = g_end - g;
-      const int r1 = (long long)(lenv - r0) < room ? lenv : (int)(r0 + room);
+      const unsigned local = (unsigned)(g - prm.Hkv * cum[b]);
+      const int hk = (int)(local / (unsigned)lenv);
+      const int r0 = (int)(local - (unsigned)hk * (unsigned)lenv);
+      const int room = g_end - g;
+      const int r1 = (lenv - r0) < room ? lenv : r0 + room;
       g += r1 - r0;
       const int j0 = r0 > kSetupCost ? r0 - kSetupCost : 0;
       const int j1 = r1 > kSetupCost ? r1 - kSetupCost : 0;
@@ -477,13 +485,15 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     // =========================================================== TMA producer
     asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
     if (lane == 0 && !*abort_flag) {
-      long long g = g_begin;
+      int g = g_begin;
       Item it;
       uint32_t item_idx = 0, fill = 0;
       bool ok = true;
       Tracer tr;
       tr.init(prm.trace, 0);
       tr.mark(0);
+      uint64_t kv_policy;      // the committed prefix is streamed once: first in line for eviction from L2
+      asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(kv_policy));
       while (ok && next_item(g, it)) {
         ok = mbar_wait(bar(L::Q_EMPTY), (item_idx & 1) ^ 1, abort_flag);
         if (!ok) break;
@@ -516,8 +526,8 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               if (tree)
                 tma_load_4d(dst + h * L::kHalf, kv ? &map_vt : &map_kt, bar(L::KV_FULL + slot), h * 64, it.hk, tt * kTileN, it.b);
               else
-                tma_load_3d(dst + h * L::kHalf, kv ? &map_vc : &map_kc, bar(L::KV_FULL + slot), h * 64, j * kTileN,
-                            it.b * prm.Hkv + it.hk);
+                tma_load_3d_hint(dst + h * L::kHalf, kv ? &map_vc : &map_kc, bar(L::KV_FULL + slot), h * 64, j * kTileN,
+                                 it.b * prm.Hkv + it.hk, kv_policy);
             }
             ++fill;
           }
@@ -535,7 +545,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     //   one row tile (buffers alternate by key tile):  S_next = Q K_next^T -> wait P -> O += P V.
     asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
     if (lane == 0 && !*abort_flag) {
-      long long g = g_begin;
+      int g = g_begin;
       Item it;
       uint32_t item_idx = 0, fill = 0, tj = 0;
       bool ok = true;
@@ -641,7 +651,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const uint32_t lane_addr = (uint32_t)((warp & 3) << 5) << 16;
     const bool wg_active = wg < MT;
     if (wg_active && !*abort_flag) {
-      long long g = g_begin;
+      int g = g_begin;
       Item it;
       uint32_t fill = 0, tj = 0, epi_phase = 0, item_cnt = 0;   // tj: key tiles handled so far (all items)
       bool ok = true;
@@ -939,30 +949,24 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             constexpr int kRows = MT * 128;
             const int rr = wg * 128 + row;
             // unit geometry in the virtual tile space: real tiles occupy [real0, uend)
-            const long long real0 = (long long)prm.Hkv * cum[it.b] + (long long)it.hk * (it.len + kSetupCost) + kSetupCost;
-            const long long uend = real0 + it.len;
+            const int real0 = prm.Hkv * cum[it.b] + it.hk * (it.len + kSetupCost) + kSetupCost;
+            const int uend = real0 + it.len;
             const int k_first = sch.find_group(real0, groups);
             const int k_last = sch.find_group(uend - 1, groups);
             // slot of the piece CTA group k holds of this unit, or -1 if it holds none
             auto piece_slot = [&](int k) -> int {
-              const long long ks = gs[k], ke = gs[k + 1];
-              const long long lo = ks > real0 ? ks : real0, hi = ke < uend ? ke : uend;
+              const int ks = gs[k], ke = gs[k + 1];
+              const int lo = ks > real0 ? ks : real0, hi = ke < uend ? ke : uend;
               if (lo >= hi) return -1;
               return (k * prm.NP + pair) * 2 + (ks > real0 ? 0 : 1);
             };
             const int my_slot = blockIdx.x * 2 + (it.j0 > 0 ? 0 : 1);
-            int n_frag = 0, n_other = 0, own_pos = 0, sid_a = 0, sid_b = 0;
+            int n_frag = 0;
+#pragma unroll 1
             for (int k = k_first; k <= k_last; ++k) {
               const int sid = piece_slot(k);
               if (sid < 0) continue;
               ++n_frag;
-              if (sid == my_slot) {
-                own_pos = n_other;           // number of other pieces that come before this one
-              } else {
-                if (n_other == 0) sid_a = sid;
-                if (n_other == 1) sid_b = sid;
-                ++n_other;
-              }
             }
             unsigned long long* ctr = prm.counters + (((size_t)it.b * prm.Hkv + it.hk) * prm.NP + pair) * 2;
             if (threadIdx.x == 128) {
@@ -1015,11 +1019,13 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               // by every thread (row rr always lies inside a slot; rows that are not active read stale bytes
               // and are masked by selects): no thread-divergent branch sits between the warp-wide TMEM ops.
               float mm = m_used, lt = 0.f;
+#pragma unroll 1
               for (int k = k_first; k <= k_last; ++k) {
                 const int sid = piece_slot(k);
                 if (sid < 0 || sid == my_slot) continue;
                 mm = fmaxf(mm, __ldcg(prm.part_ml + (size_t)sid * 2 * kRows + rr));
               }
+#pragma unroll 1
               for (int k = k_first; k <= k_last; ++k) {
                 const int sid = piece_slot(k);
                 if (sid < 0) continue;
@@ -1040,6 +1046,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 float acc[64];
 #pragma unroll
                 for (int c = 0; c < 64; ++c) acc[c] = 0.f;
+#pragma unroll 1
                 for (int k = k_first; k <= k_last; ++k) {
                   const int sid = piece_slot(k);
                   if (sid < 0) continue;
@@ -1119,6 +1126,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     while (globaltimer_ns() - t0 < 200000ull) {
     }
     if (threadIdx.x == 0)
+#pragma unroll 1
       for (int b = 0; b < prm.B; ++b) atomicOr(&prm.status[b], TV_ST_TIMEOUT);
   }
   __syncthreads();
