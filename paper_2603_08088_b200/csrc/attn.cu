@@ -659,7 +659,10 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       tr.init((threadIdx.x & 127) == 0 ? prm.trace : nullptr, 2 + wg);
       tr.mark(0);
 #ifdef TV_PROF
-      unsigned int prof[6] = {0u, 0u, 0u, 0u, 0u, 0u}, pc0 = 0, pc1 = 0, pc2 = 0, pend = 0;
+      unsigned int prof[12] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u}, pc0 = 0, pc1 = 0, pc2 = 0, pend = 0;
+      // 0 wait S, 1 ld, 2 compute, 3 hand-over, 4 tiles, 5 between tiles, 6 start -> first S, 7 wait ITEM_DONE,
+      // 8 epilogue (whole or piece), 9 items, 10 first tile of an item: from item start to its S
+      const unsigned int prof_start = clock();
       const long long prof_c0 = clock64();
       const unsigned long long prof_g0 = globaltimer_ns();   // cycles: wait S, ld, compute, hand-over; tiles
 #endif
@@ -676,6 +679,9 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         return r;
       };
       while (ok && next_item(g, it)) {
+#ifdef TV_PROF
+        const unsigned int pitem = clock();
+#endif
         const int nt = it.j1 - it.j0;
         const int node = (pair * MT + wg) * prm.NPT + row / prm.G;
         const int gm = row % prm.G;
@@ -739,6 +745,8 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           TV_PROF_T(pc1);
 #ifdef TV_PROF
           prof[0] += pc1 - pc0;
+          if (tj == 0) prof[6] = pc1 - prof_start;
+          if (jt == 0) prof[10] += pc1 - pitem;
 #endif
           tr.mark(0x1000u | (tj & 0xfffu));
 #pragma unroll
@@ -896,10 +904,15 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           // Wait for every MMA of the item.  This barrier completes once per item, so its phase is never
           // more than one away from the one waited for (a parity wait cannot tell phases two apart, which
           // is why the per-PV barrier O_DONE is not used here: both last PVs may or may not be done yet).
+          TV_PROF_T(pc0);
           ok = wwait(bar(L::ITEM_DONE + wg), item_cnt & 1);
           ++item_cnt;
           if (!ok) break;
           tc_fence_after();
+          TV_PROF_T(pc1);
+#ifdef TV_PROF
+          prof[7] += pc1 - pc0;
+#endif
           tr.mark(0x5000u);
           const uint32_t o_addr = o_addr_loop;
           const bool whole = (it.j0 == 0 && it.j1 == it.len);
@@ -1102,12 +1115,16 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           }
         }
         tr.mark(0x8000u);
+#ifdef TV_PROF
+        prof[8] += clock() - pc1;
+        prof[9] += 1;
+#endif
         fill += 2 * nt;
       }
 #ifdef TV_PROF
       if (tr.base)
       {
-        for (int i = 0; i < 6; ++i) tr.base[kTraceCap - 8 + i] = prof[i];
+        for (int i = 0; i < 12; ++i) tr.base[kTraceCap - 16 + i] = prof[i];
         tr.base[kTraceCap - 2] = clock64() - prof_c0;
         tr.base[kTraceCap - 1] = globaltimer_ns() - prof_g0;
       }
