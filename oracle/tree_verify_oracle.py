@@ -206,6 +206,38 @@ def tree_attention(q_bits, k_cache_bits, v_cache_bits, k_tree_bits, v_tree_bits,
     return out, lse
 
 
+def merge_partials(o_parts, lse_parts):
+    """Attention over a key set split in R disjoint ranges, from the per-range results (the context split
+    that longer-context, multi-device serving needs; Section 6, "Limitations and future work"; the
+    attention itself is Section 2.4).  For one query row, range r gives O_r = softmax over its own keys
+    times V and lse_r = log of the sum of exp(score) over its keys; over the union the softmax weights are
+    exp(score) / sum_r exp(lse_r), so  O = sum_r exp(lse_r) O_r / sum_r exp(lse_r)  and
+    lse = log sum_r exp(lse_r)  (evaluated with the maximum subtracted).  A range without visible keys has
+    lse_r = -inf and weight 0; a row without any key gives zeros and -inf.
+    o_parts[R,B,Nmax,Hq,d], lse_parts[R,B,Hq,Nmax] -> out[B,Nmax,Hq,d] f64, lse[B,Hq,Nmax] f64."""
+    o_parts = np.asarray(o_parts, dtype=np.float64)
+    lse_parts = np.asarray(lse_parts, dtype=np.float64)
+    R, B, Nmax, Hq, d = o_parts.shape
+    out = np.zeros((B, Nmax, Hq, d), dtype=np.float64)
+    lse = np.full((B, Hq, Nmax), -np.inf, dtype=np.float64)
+    for b in range(B):
+        for h in range(Hq):
+            for i in range(Nmax):
+                l = lse_parts[:, b, h, i]
+                m = l.max()
+                if m == -np.inf:
+                    continue
+                w = np.exp(l - m)                      # exp(-inf) = 0 for empty ranges
+                tot = w.sum()
+                acc = np.zeros(d, dtype=np.float64)
+                for r in range(R):
+                    if w[r] > 0.0:                     # an empty range may carry anything in O_r
+                        acc += w[r] * o_parts[r, b, i, h, :]
+                out[b, i, h, :] = acc / tot
+                lse[b, h, i] = m + np.log(tot)
+    return out, lse
+
+
 # ---------------------------------------------------------------------------
 # Sections 2.5, 3.2: accelerator-safe path gather
 # ---------------------------------------------------------------------------

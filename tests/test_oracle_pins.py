@@ -517,3 +517,56 @@ def test_node_scores_gather_and_link_to_greedy_acceptance():
     bad[0, 4] = -3
     s2, st2 = orc.node_scores(bits, bad, parent, n)
     assert st2.tolist() == [orc.ST_BAD_INDEX] * 2 and np.isneginf(s2[1, 2]) and np.isneginf(s2[0, 4])
+
+
+def test_merge_partials_equals_attention_over_the_union_of_key_ranges():
+    """Pin for merge_partials: splitting the committed prefix in R ranges, attending to each range
+    separately (tree keys with the last range only) and merging must give the attention over all
+    keys - an identity of the softmax, so the two oracle results agree to rounding."""
+    rng = np.random.default_rng(11)
+    B, Hq, Hkv, d, N, Scap = 2, 4, 2, 8, 6, 40
+    f = lambda *s: _bf16(rng.standard_normal(s).astype(np.float32))
+    q, kc, vc = f(B, N, Hq, d), f(B, Hkv, Scap, d), f(B, Hkv, Scap, d)
+    kt, vt = f(B, N, Hkv, d), f(B, N, Hkv, d)
+    S = np.array([37, 5])
+    n = np.array([6, 4])
+    parent = np.array([[-1, 0, 0, 1, 1, 2], [-1, 0, 1, 2, 0, 0]])
+    vis = orc.build_mask(parent, n, 5, 1, emit_paths=False)["dense"][:, 0]
+    full, full_lse = orc.tree_attention(q, kc, vc, kt, vt, S, n, vis, 0.3)
+    for R in (1, 2, 3, 5):
+        o_parts, l_parts = [], []
+        for r in range(R):
+            lo, hi = (S * r) // R, (S * (r + 1)) // R          # key range of "rank" r per sequence
+            kc_r, vc_r = np.zeros_like(kc), np.zeros_like(vc)
+            for b in range(B):
+                kc_r[b, :, :hi[b] - lo[b]] = kc[b, :, lo[b]:hi[b]]
+                vc_r[b, :, :hi[b] - lo[b]] = vc[b, :, lo[b]:hi[b]]
+            vis_r = vis if r == R - 1 else np.zeros_like(vis)   # tree keys belong to the last range
+            o, l = orc.tree_attention(q, kc_r, vc_r, kt, vt, hi - lo, n, vis_r, 0.3)
+            o_parts.append(o)
+            l_parts.append(l)
+        out, lse = orc.merge_partials(np.stack(o_parts), np.stack(l_parts))
+        assert np.allclose(out, full, rtol=0, atol=1e-12)
+        assert np.array_equal(np.isneginf(lse), np.isneginf(full_lse))
+        fin = np.isfinite(full_lse)
+        assert np.allclose(lse[fin], full_lse[fin], rtol=0, atol=1e-12)
+    # with R = 5 the short sequence (S = 5 -> ranges of 1 key) and padded rows exercise small and empty ranges
+
+
+def test_merge_partials_closed_forms():
+    """R = 1 is the identity; equal lse gives the plain average; an empty range (lse = -inf) is ignored even
+    if its O holds NaN; all ranges empty gives zeros and -inf."""
+    o = np.zeros((3, 1, 2, 1, 4))
+    o[0, 0, 0, 0] = [1, 2, 3, 4]
+    o[1, 0, 0, 0] = [3, 2, 1, 0]
+    o[2] = np.nan
+    l = np.full((3, 1, 1, 2), -np.inf)
+    l[0, 0, 0, 0] = l[1, 0, 0, 0] = 0.7
+    out, lse = orc.merge_partials(o, l)
+    assert np.allclose(out[0, 0, 0], [2, 2, 2, 2]) and np.isclose(lse[0, 0, 0], 0.7 + np.log(2.0))
+    assert (out[0, 1, 0] == 0).all() and lse[0, 0, 1] == -np.inf
+    one, one_l = orc.merge_partials(o[:1], l[:1])
+    assert np.array_equal(one[0, 0, 0], o[0, 0, 0, 0]) and one_l[0, 0, 0] == 0.7
+    l[1, 0, 0, 0] = 0.7 + np.log(3.0)                      # weights 1 : 3
+    out, lse = orc.merge_partials(o, l)
+    assert np.allclose(out[0, 0, 0], (np.array([1, 2, 3, 4]) + 3 * np.array([3, 2, 1, 0])) / 4)
