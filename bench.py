@@ -322,11 +322,57 @@ def run_ours(args, cfg):
                      "tensor_tflops": attn_flops(cfg, S_host) / (attn_ms * 1e-3) / 1e12},
         "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e,
     }
+    if args.context_split > 1:
+        case["prefix_len"].copy_(prefix0)
+        line["context_split"] = context_split_member(cfg, case, buf, args.context_split, dev)
     if args.cpu_baseline:
         sec, desc, threads = oracle_sample_seconds(cfg, args.seed)
         line["cpu_baseline"] = {"value": 1.0 / sec, "unit": UNIT, "cores": threads, "kind": "oracle",
                                 "sample": desc, "est_seconds_per_step": sec}
     print(json.dumps(line))
+
+
+def context_split_member(cfg, case, buf, R, dev):
+    """What one member of an R-way context split of this workload does per layer, timed on this GPU: attention
+    over its 1/R of every prefix (it owns the tree keys, the worst case) and the merge of R gathered partials.
+    The all-gather itself needs R GPUs and is not timed here; its payload is reported."""
+    import paper_2603_08088_b200 as tv
+    from paper_2603_08088_b200 import dist as tvd
+    B, N, Hq, d = cfg.B, cfg.N, cfg.Hq, cfg.d
+    lo, hi = tvd.split_prefix(case["prefix_len"], R - 1, R)
+    local_len = (hi - lo).to(torch.int32)
+    out = torch.empty(B, N, Hq, d, dtype=torch.bfloat16, device=dev)
+    lse = torch.empty(B, Hq, N, dtype=torch.float32, device=dev)
+    o_parts = torch.randn(R, B, N, Hq, d, device=dev).to(torch.bfloat16)
+    l_parts = torch.randn(R, B, Hq, N, device=dev)
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def attn():
+        tv.tree_verify_attn(case["q"][0], case["k_cache"][0], case["v_cache"][0], case["k_tree"][0], case["v_tree"][0],
+                            local_len, case["n_nodes"], buf.anc_bits, d ** -0.5, out, buf.attn_ws, buf.status, lse=lse)
+
+    def merge():
+        tv.tree_merge_partials(o_parts, l_parts, out, lse)
+
+    res = {}
+    for name, fn in (("attn", attn), ("merge", merge)):
+        for _ in range(3):
+            fn()
+        a, b = ev(), ev()
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(20):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        res[name] = a.elapsed_time(b) / 20 * 1e3
+    gather_bytes = (R - 1) * (B * N * Hq * d * 2 + B * Hq * N * 4)
+    merge_bytes = R * (B * N * Hq * d * 2 + B * Hq * N * 4) + B * N * Hq * d * 2 + B * Hq * N * 4
+    return {"members": R, "member_attn_us": res["attn"], "merge_us": res["merge"],
+            "merge_gbs": merge_bytes / (res["merge"] * 1e-6) / 1e9,
+            "allgather_bytes_received_per_member": gather_bytes,
+            "note": "one member timed on one GPU (back-to-back launches, inputs re-read from L2 where they fit); "
+                    "the all-gather is not timed"}
 
 
 def main():
@@ -338,6 +384,8 @@ def main():
     ap.add_argument("--workload", default="full_step_32l", choices=[c.name for c in CONFIGS])
     ap.add_argument("--seed", type=int, default=4000)
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    ap.add_argument("--context-split", type=int, default=1,
+                    help="also time one member of an R-way context split of the workload (extra key in the JSON line)")
     args = ap.parse_args()
     cfg = get_config(args.workload)
     if args.impl == "reference":

@@ -194,6 +194,25 @@ TV_API int tree_node_scores(const tv_bf16* logits, const int32_t* tokens, const 
                             int32_t* status, tv_stream stream);
 
 /*
+ * Attention over a key set that was split in R disjoint ranges (Section 6,
+ * "Limitations and future work": longer-context workloads and multi-device
+ * serving; the attention is Section 2.4).  Each member of a context-split group
+ * runs tree_verify_attn over its own range of the committed prefix (the tree's
+ * keys belong to exactly one member; the others pass all-zero anc_bits) and
+ * keeps out and lse; after the partials of all members have been gathered into
+ * local memory, this call combines them per query row:
+ *   out = sum_r w_r O_r / sum_r w_r,  w_r = exp(lse_r - max_r lse_r),
+ *   lse = max_r lse_r + log sum_r w_r.
+ * A range without visible keys has lse_r = -inf and weight 0 (its O_r is not
+ * read); a row without any key gives zeros and -inf.
+ *   o_parts[R,B,Nmax,Hq,d] bf16, lse_parts[R,B,Hq,Nmax] fp32 (natural log)  in, device, local memory
+ *   out[B,Nmax,Hq,d] bf16  out;  lse[B,Hq,Nmax] fp32  out, may be NULL
+ * d must be a multiple of 8, o_parts and out 16-byte aligned.
+ */
+TV_API int tree_merge_partials(const tv_bf16* o_parts, const float* lse_parts, int R, int B, int Nmax, int Hq, int d,
+                               tv_bf16* out, float* lse, tv_stream stream);
+
+/*
  * tree_accept for callers that cannot allocate device memory (the paper has
  * no counterpart; this is a convenience of this library).  Some hosts of this
  * code may not call cudaMalloc at all: a plugin inside a serving runtime that

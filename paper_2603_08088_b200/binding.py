@@ -15,7 +15,7 @@ TV_OK, TV_ERR_INVALID_ARG, TV_ERR_CUDA, TV_ERR_WORKSPACE = 0, 1, 2, 3
 TV_ST_BAD_TREE, TV_ST_BAD_INDEX, TV_ST_CAPACITY, TV_ST_TIMEOUT, TV_ST_PATHS_TRUNCATED = 1, 2, 4, 8, 16
 
 EXPORTS = ["tv_last_error", "tv_version", "tv_launch_count", "tree_build_mask", "tv_attn_workspace_bytes", "tree_verify_attn",
-           "tv_accept_workspace_bytes", "tree_accept", "tree_node_scores", "tv_accept_noalloc_max_bytes", "tree_accept_noalloc",
+           "tv_accept_workspace_bytes", "tree_accept", "tree_node_scores", "tree_merge_partials", "tv_accept_noalloc_max_bytes", "tree_accept_noalloc",
            "kv_commit", "tv_step_staging_bytes",
            "tv_verify_step_host"]
 
@@ -67,6 +67,8 @@ def load():
     lib.tree_accept.argtypes = [_c_vp] * 4 + [_c_int] * 5 + [_c_vp] * 7 + [_c_vp, _c_sz, _c_vp, _c_vp]
     lib.tree_node_scores.restype = _c_int
     lib.tree_node_scores.argtypes = [_c_vp] * 4 + [_c_int] * 3 + [_c_vp, _c_vp, _c_vp]
+    lib.tree_merge_partials.restype = _c_int
+    lib.tree_merge_partials.argtypes = [_c_vp, _c_vp] + [_c_int] * 5 + [_c_vp, _c_vp, _c_vp]
     lib.tv_accept_noalloc_max_bytes.restype = _c_sz
     lib.tv_accept_noalloc_max_bytes.argtypes = []
     lib.tree_accept_noalloc.restype = _c_int
@@ -166,6 +168,12 @@ def tree_node_scores(logits, tokens, parent, n_nodes, scores, status, stream=Non
     B, Nmax, V = logits.shape
     _check(load().tree_node_scores(_ptr(logits), _ptr(tokens), _ptr(parent), _ptr(n_nodes), B, Nmax, V,
                                    _ptr(scores), _ptr(status), _stream(stream)))
+
+
+def tree_merge_partials(o_parts, lse_parts, out, lse=None, stream=None):
+    R, B, Nmax, Hq, d = o_parts.shape
+    _check(load().tree_merge_partials(_ptr(o_parts), _ptr(lse_parts), R, B, Nmax, Hq, d, _ptr(out),
+                                      _ptr(lse) if lse is not None else None, _stream(stream)))
 
 
 def tv_accept_noalloc_max_bytes():
