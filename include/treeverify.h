@@ -122,12 +122,20 @@ TV_API size_t tv_attn_workspace_bytes(int B, int Nmax, int Hq, int Hkv, int d, i
  *   lse[B,Hq,Nmax]                 out or NULL, fp32 log-sum-exp of the
  *                                      scaled scores; -inf for padded rows
  *   workspace                      device scratch, 256-byte aligned, at least
- *                                      tv_attn_workspace_bytes(...) bytes
+ *                                      tv_attn_workspace_bytes(...) bytes; needs
+ *                                      no initialisation; calls that share one
+ *                                      must be issued in one stream
  *   status[B]                      in/out: TV_ST_TIMEOUT is ORed in if a
  *                                      bounded wait expired (outputs invalid)
  * Limits: d in {64,128}; Nmax <= 256 (the node budgets of the paper's sweep);
  * Hq % Hkv == 0, Hq / Hkv <= 128; B <= 512; all tensors 16-byte aligned;
  * 0 <= prefix_len[b] <= Scap; scale > 0.
+ * Stream order: the kernel is launched with programmatic stream serialisation.
+ * Behind another tree_verify_attn launch (the layers of one step) it starts
+ * while that one drains and requests its first committed-prefix tiles at once;
+ * q, the tree's K/V, anc_bits, out, lse and the workspace are only touched
+ * after every earlier kernel of the stream has finished.  Behind any other
+ * kernel it starts when that kernel has finished, as usual.
  */
 TV_API int tree_verify_attn(const tv_bf16* q,
                      const tv_bf16* k_cache, const tv_bf16* v_cache,

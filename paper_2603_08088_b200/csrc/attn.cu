@@ -44,6 +44,8 @@
 
 #include <atomic>
 #include <chrono>
+#include <mutex>
+#include <unordered_map>
 
 namespace {
 
@@ -117,6 +119,11 @@ __device__ __forceinline__ void fence_barrier_init() {
 __device__ __forceinline__ void fence_proxy_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
+// Programmatic dependent launch.  gdc_wait: every kernel launched before this one in the stream has finished and
+// its writes are visible.  gdc_launch_dependents: the next kernel in the stream may be scheduled once every CTA of
+// this grid has got here or has exited.
+__device__ __forceinline__ void gdc_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void gdc_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -494,10 +501,18 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       tr.mark(0);
       uint64_t kv_policy;      // the committed prefix is streamed once: first in line for eviction from L2
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(kv_policy));
-      while (ok && next_item(g, it)) {
-        ok = mbar_wait(bar(L::Q_EMPTY), (item_idx & 1) ^ 1, abort_flag);
-        if (!ok) break;
-        tr.mark(0x1000u | item_idx);
+      // Overlap with the kernel in front (programmatic dependent launch): the committed prefix, prefix_len and
+      // n_nodes are not written by a tree_verify_attn call, the one kernel that lets this one start early, so
+      // the first prefix tiles are requested at once; Q and the tree's K/V - what a preceding kernel may still
+      // be producing - wait for that kernel to finish.  Only then may the next kernel be scheduled, so that at
+      // most two launches are in flight and the two halves of the workspace suffice.
+      bool synced = false;
+      auto sync_with_predecessor = [&]() {
+        gdc_wait();
+        gdc_launch_dependents();
+        synced = true;
+      };
+      auto load_q = [&]() {
         mbar_expect_tx(bar(L::Q_FULL), MT * (D / 64) * prm.q_box_bytes);
 #pragma unroll
         for (int t = 0; t < MT; ++t)
@@ -505,6 +520,13 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           for (int h = 0; h < D / 64; ++h)
             tma_load_4d(sbase + L::kQ + t * L::kTileBytes + h * L::kHalf, &map_q, bar(L::Q_FULL), h * 64,
                         it.hk * prm.G, (pair * MT + t) * prm.NPT, it.b);
+      };
+      while (ok && next_item(g, it)) {
+        ok = mbar_wait(bar(L::Q_EMPTY), (item_idx & 1) ^ 1, abort_flag);
+        if (!ok) break;
+        tr.mark(0x1000u | item_idx);
+        bool q_pending = !synced;          // first item: Q goes out after the first prefix tiles
+        if (!q_pending) load_q();
         ++item_idx;
         for (int j = it.j0; j < it.j1 && ok; ++j) {
           const int tt = j - (it.len - prm.TT);      // >= 0: index of the tree key tile
@@ -512,10 +534,11 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 #pragma unroll
           for (int kv = 0; kv < 2; ++kv) {
             const uint32_t slot = fill % kSlots, round = fill / kSlots;
-            // At kernel start every CTA asks for its whole ring at once; let Q and the first K/V tile land
-            // before queueing the rest, so that the first MMA can start a few microseconds earlier.
-            if (item_idx == 1 && fill == 2) ok = mbar_wait(bar(L::Q_FULL), 0, abort_flag);
-            if (!ok) break;
+            if (q_pending && (tree || fill >= (uint32_t)kSlots)) {      // before the first wait for a ring slot
+              sync_with_predecessor();
+              load_q();
+              q_pending = false;
+            }
             ok = mbar_wait(bar(L::KV_EMPTY + slot), (round & 1) ^ 1, abort_flag);
             if (!ok) break;
             tr.mark(0x2000u | (fill & 0xfffu));
@@ -532,7 +555,15 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             ++fill;
           }
         }
+        if (ok && q_pending) {
+          sync_with_predecessor();
+          load_q();
+        }
       }
+      if (!synced) sync_with_predecessor();        // a CTA without work still has to let the next kernel go
+    } else if (lane == 0) {
+      gdc_wait();
+      gdc_launch_dependents();
     }
   } else if (warp == 1) {
     // =========================================================== MMA issuer
@@ -650,6 +681,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const int row = ((warp & 3) << 5) | lane;        // TMEM lane = row inside the tile
     const uint32_t lane_addr = (uint32_t)((warp & 3) << 5) << 16;
     const bool wg_active = wg < MT;
+    gdc_wait();      // anc_bits, the workspace and the outputs may belong to the kernel in front until it is done
     if (wg_active && !*abort_flag) {
       int g = g_begin;
       Item it;
@@ -1182,7 +1214,7 @@ bool encode_map(CUtensorMap* m, const void* base, int rank, const cuuint64_t* di
 
 struct Geometry {
   int G, NPT, n_row_tiles, MT, NP, sms, groups, grid;
-  size_t counters_off, ml_off, o_off, total;
+  size_t counters_off, ml_off, o_off, half, total;
 };
 
 int sm_count() {
@@ -1215,11 +1247,21 @@ Geometry geometry(int B, int Nmax, int Hq, int Hkv, int d, bool query_device) {
   off = (off + 255) & ~size_t(255);
   g.o_off = off;
   off += max_ctas * 2 * (size_t)g.MT * 128 * d * sizeof(tv_bf16);
-  g.total = off;
+  off = (off + 255) & ~size_t(255);
+  g.half = off;          // two such halves: consecutive launches may overlap and take turns
+  g.total = 2 * off;
   return g;
 }
 
 std::atomic<unsigned long long*> g_trace{nullptr};
+
+// 0 or 1, alternating per workspace: which half of the workspace this call uses.
+int workspace_turn(const void* workspace) {
+  static std::mutex mu;
+  static std::unordered_map<const void*, unsigned> calls;
+  std::lock_guard<std::mutex> lock(mu);
+  return (int)(calls[workspace]++ & 1u);
+}
 
 unsigned long long next_epoch() {
   static std::atomic<unsigned long long> ctr{
@@ -1239,8 +1281,19 @@ cudaError_t launch(const Geometry& g, const CUtensorMap* maps, const AttnParams&
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) configured[dev].store(true, std::memory_order_release);
   }
-  kern<<<g.grid, kThreads, L::kTotal, s>>>(maps[0], maps[1], maps[2], maps[3], maps[4], prm);
-  return cudaGetLastError();
+  // Programmatic stream serialisation: this launch may be scheduled while the kernel in front is still
+  // running (if that kernel allows it); the kernel itself waits before it touches anything that kernel writes.
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(g.grid);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = L::kTotal;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, maps[0], maps[1], maps[2], maps[3], maps[4], prm);
 }
 
 }  // namespace
@@ -1311,7 +1364,8 @@ extern "C" int tree_verify_attn(const tv_bf16* q,
   prm.out = out;
   prm.lse = lse;
   prm.status = status;
-  char* ws = static_cast<char*>(workspace);
+  // consecutive calls on one workspace take turns on its two halves (they may overlap on the device)
+  char* ws = static_cast<char*>(workspace) + (workspace_turn(workspace) ? g.half : 0);
   prm.counters = reinterpret_cast<unsigned long long*>(ws + g.counters_off);
   prm.part_ml = reinterpret_cast<float*>(ws + g.ml_off);
   prm.part_o = reinterpret_cast<tv_bf16*>(ws + g.o_off);
