@@ -234,6 +234,44 @@ def test_repeated_launches_are_bit_reproducible_and_never_time_out():
             assert torch.equal(out, first[0]) and torch.equal(lse, first[1]), f"launch {it} differs from launch 0"
 
 
+def test_back_to_back_launches_on_one_workspace_match_isolated_launches():
+    """The layers of a step are launched back to back on one stream and one workspace, and a launch may
+    start while the one in front is still draining.  Every launch must give exactly what it gives alone:
+    no partial, counter or output of a neighbouring launch may leak in."""
+    cfg = CONFIGS[4].scaled(L=4, B=6, V=0)
+    dcase = make_case(cfg, seed=4100, device="cuda", with_logits=False)
+    B, N, L = cfg.B, cfg.N, cfg.L
+    bits = torch.zeros(B, N, (N + 31) // 32, dtype=torch.int32, device="cuda")
+    status = torch.zeros(B, dtype=torch.int32, device="cuda")
+    tv.tree_build_mask(dcase["parent"], dcase["n_nodes"], N - 1, 1, bits, status)
+    nbytes = tv.tv_attn_workspace_bytes(B, N, cfg.Hq, cfg.Hkv, cfg.d, cfg.Scap)
+    ws = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+
+    def launch(layer, out, lse, workspace):
+        tv.tree_verify_attn(dcase["q"][layer], dcase["k_cache"][layer], dcase["v_cache"][layer],
+                            dcase["k_tree"][layer], dcase["v_tree"][layer], dcase["prefix_len"], dcase["n_nodes"],
+                            bits, cfg.d ** -0.5, out, workspace, status, lse=lse)
+
+    alone = []
+    for layer in range(L):                      # isolated: own workspace, synchronised on both sides
+        out = torch.zeros(B, N, cfg.Hq, cfg.d, dtype=torch.bfloat16, device="cuda")
+        lse = torch.zeros(B, cfg.Hq, N, dtype=torch.float32, device="cuda")
+        launch(layer, out, lse, torch.zeros(nbytes, dtype=torch.uint8, device="cuda"))
+        torch.cuda.synchronize()
+        alone.append((out, lse))
+    for rep in range(5):                        # back to back, 3 rounds over the layers, nothing in between
+        outs = [torch.zeros(B, N, cfg.Hq, cfg.d, dtype=torch.bfloat16, device="cuda") for _ in range(3 * L)]
+        lses = [torch.zeros(B, cfg.Hq, N, dtype=torch.float32, device="cuda") for _ in range(3 * L)]
+        torch.cuda.synchronize()
+        for i in range(3 * L):
+            launch(i % L, outs[i], lses[i], ws)
+        torch.cuda.synchronize()
+        assert (status == 0).all(), f"status {status.cpu().tolist()}"
+        for i in range(3 * L):
+            assert torch.equal(outs[i], alone[i % L][0]) and torch.equal(lses[i], alone[i % L][1]), \
+                f"round {rep}, launch {i} (layer {i % L}) differs from the isolated launch"
+
+
 FULL = [(1, [(0, 0), (0, 17), (0, 31)]), (2, [(0, 0), (3, 5), (7, 7)]), (3, [(0, 0), (3, 7)]),
         (4, [(0, 0), (9, 3), (15, 7)])]
 
