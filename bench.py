@@ -322,6 +322,8 @@ def run_ours(args, cfg):
                      "tensor_tflops": attn_flops(cfg, S_host) / (attn_ms * 1e-3) / 1e12},
         "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e,
     }
+    if args.budget_sweep:
+        line["budget_sweep"] = budget_sweep(args.seed, dev)
     if args.context_split > 1:
         case["prefix_len"].copy_(prefix0)
         line["context_split"] = context_split_member(cfg, case, buf, args.context_split, dev)
@@ -330,6 +332,48 @@ def run_ours(args, cfg):
         line["cpu_baseline"] = {"value": 1.0 / sec, "unit": UNIT, "cores": threads, "kind": "oracle",
                                 "sample": desc, "est_seconds_per_step": sec}
     print(json.dumps(line))
+
+
+def budget_sweep(seed, dev):
+    """tree_verify_attn over the node budgets and depths of the paper's sensitivity sweep (Table 2: M from 16 to
+    256 draft nodes, depth bounds 4 to 16) on the ragged GQA batch of config 3: one layer, 20 back-to-back
+    launches per shape, CUDA events.  M counts draft nodes; the tree has M + 1 rows with the root, capped at
+    256 rows (the kernel's limit)."""
+    import paper_2603_08088_b200 as tv
+    peak, _ = measured_peaks()
+    rows = []
+    for M, D in ((16, 4), (32, 6), (64, 8), (128, 12), (256, 16)):
+        N = min(M + 1, 256)
+        cfg = get_config("gqa8b_ragged").scaled(N=N, D=D, tree="spine", L=1, V=0, P=0)
+        case = make_case(cfg, seed, device=dev, with_logits=False)
+        B = cfg.B
+        bits = torch.zeros(B, N, (N + 31) // 32, dtype=torch.int32, device=dev)
+        status = torch.zeros(B, dtype=torch.int32, device=dev)
+        tv.tree_build_mask(case["parent"], case["n_nodes"], N - 1, 1, bits, status)
+        out = torch.empty(B, N, cfg.Hq, cfg.d, dtype=torch.bfloat16, device=dev)
+        ws = torch.zeros(tv.tv_attn_workspace_bytes(B, N, cfg.Hq, cfg.Hkv, cfg.d, cfg.Scap), dtype=torch.uint8, device=dev)
+
+        def run():
+            tv.tree_verify_attn(case["q"][0], case["k_cache"][0], case["v_cache"][0], case["k_tree"][0], case["v_tree"][0],
+                                case["prefix_len"], case["n_nodes"], bits, cfg.d ** -0.5, out, ws, status)
+
+        for _ in range(3):
+            run()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(20):
+            run()
+        b.record()
+        torch.cuda.synchronize()
+        us = a.elapsed_time(b) / 20 * 1e3
+        S = case["prefix_len"].cpu().numpy()
+        if int(status.cpu().numpy().max()) != 0:
+            raise SystemExit(f"bench.py: budget sweep M={M}: status {status.cpu().numpy()}")
+        rows.append({"M": M, "rows": N, "Dmax": D, "attn_us": us,
+                     "hbm_frac": attn_algorithmic_bytes(cfg, S) / (us * 1e-6) / 1e9 / peak,
+                     "tensor_tflops": attn_flops(cfg, S) / (us * 1e-6) / 1e12})
+    return rows
 
 
 def context_split_member(cfg, case, buf, R, dev):
@@ -384,6 +428,8 @@ def main():
     ap.add_argument("--workload", default="full_step_32l", choices=[c.name for c in CONFIGS])
     ap.add_argument("--seed", type=int, default=4000)
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    ap.add_argument("--budget-sweep", action="store_true",
+                    help="also time tree_verify_attn over the node budgets of the paper's sweep (extra key in the JSON line)")
     ap.add_argument("--context-split", type=int, default=1,
                     help="also time one member of an R-way context split of the workload (extra key in the JSON line)")
     args = ap.parse_args()
