@@ -18,6 +18,8 @@ STEP_CASES = [
     ("llama7b_layer", 1, dict(Hq=8, Hkv=8, S_lo=300, S_hi=300, Scap=384)),
     ("gqa8b_ragged", 2, dict(B=4, Hq=16, Hkv=4, S_lo=60, S_hi=500, Scap=640, V=128256)),
     ("full_step", 4, dict(B=5, L=3, Hq=16, Hkv=4, S_lo=30, S_hi=260, Scap=320, V=153600)),
+    # the variant whose ten candidate rows name all 60 nodes (ten chains from the root)
+    ("full_step_covering_rows", 4, dict(B=4, L=2, Hq=16, Hkv=4, S_lo=30, S_hi=260, Scap=320, V=20000, tree="chains")),
 ]
 
 
@@ -34,7 +36,7 @@ def run_step(cfg, case, given_rows):
 @pytest.mark.parametrize("name,ci,over", STEP_CASES, ids=[s[0] for s in STEP_CASES])
 def test_whole_step_matches_oracle(name, ci, over):
     cfg = CONFIGS[ci].scaled(**over)
-    case = make_case(cfg, seed=1000 * ci + 7, ragged_nodes=(cfg.B > 2))
+    case = make_case(cfg, seed=1000 * ci + 7, ragged_nodes=(cfg.B > 2 and cfg.tree != "chains"))
     given_rows = cfg.P > 0
     ref = orc.verify_step(case_to_numpy(case), cfg.d ** -0.5, use_given_retrieve=given_rows)
     d, buf = run_step(cfg, case, given_rows)

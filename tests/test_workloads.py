@@ -41,3 +41,22 @@ def test_ragged_nodes_pad_with_device_defined_fill():
         assert (par[b, n[b]:] == 0).all()
         r = a["retrieve"].numpy()[b]
         assert r.max() < n[b]
+
+
+def test_covering_chains_tree_rows_name_every_node():
+    """The second variant of the full-step config: ten chains from the root, nine of depth 6 and one of
+    depth 5, so that the ten candidate rows of seven columns cover all 60 nodes."""
+    import numpy as np
+    from workloads import CONFIGS, make_case, covering_chains_tree, leaf_paths
+    p = covering_chains_tree(60, 10, 6, np.random.default_rng(3))
+    rows = leaf_paths(p)
+    assert len(rows) == 10 and sorted(len(r) - 1 for r in rows) == [5] + [6] * 9
+    assert sorted(n for r in rows for n in r[1:]) == list(range(1, 60)) and all(r[0] == 0 for r in rows)
+    assert (p[1:] < np.arange(1, 60)).all() and p[0] == -1
+    cfg = CONFIGS[4].scaled(L=1, B=3, S_lo=4, S_hi=9, Scap=32, V=64, tree="chains")
+    case = make_case(cfg, seed=1)
+    r = case["retrieve"].numpy()
+    assert r.shape == (3, 10, 7)
+    for b in range(3):
+        named = set(int(x) for x in r[b].ravel() if x >= 0)
+        assert named == set(range(60))

@@ -8,12 +8,12 @@ ancestor table, no attention, no argmax, no acceptance - and is the only code
 shared by the CPU oracle's tests and the CUDA path's tests and bench.
 """
 from .configs import CONFIGS, VerifyConfig, get_config
-from .trees import (random_parent_tree, topk_expansion_tree, spine_tree, chain_tree, star_tree, leaf_paths,
+from .trees import (random_parent_tree, topk_expansion_tree, spine_tree, covering_chains_tree, chain_tree, star_tree, leaf_paths,
                     capped_paths)
 from .cases import make_case, case_to_numpy, bf16_bits, bits_to_f32, randn_bf16
 
 __all__ = [
     "CONFIGS", "VerifyConfig", "get_config",
-    "random_parent_tree", "topk_expansion_tree", "spine_tree", "chain_tree", "star_tree",
+    "random_parent_tree", "topk_expansion_tree", "spine_tree", "covering_chains_tree", "chain_tree", "star_tree",
     "leaf_paths", "capped_paths", "make_case", "case_to_numpy", "bf16_bits", "bits_to_f32", "randn_bf16",
 ]

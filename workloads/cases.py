@@ -8,7 +8,7 @@ import numpy as np
 import torch
 
 from .configs import VerifyConfig
-from .trees import (random_parent_tree, topk_expansion_tree, spine_tree, leaf_paths, capped_paths,
+from .trees import (random_parent_tree, topk_expansion_tree, spine_tree, covering_chains_tree, leaf_paths, capped_paths,
                     rows_to_retrieve)
 
 PLANT_LOGIT = 16.0  # far above any N(0,1) draw that survives bf16 rounding
@@ -47,6 +47,8 @@ def _draw_tree(cfg: VerifyConfig, n, rng):
         return random_parent_tree(n, min(cfg.D, max(1, (n - 1) // 2)), rng)
     if cfg.tree == "spine":
         return spine_tree(n, min(cfg.D, n - 1), rng)
+    if cfg.tree == "chains":         # rows cover every node: P chains from the root
+        return covering_chains_tree(n, cfg.P if cfg.P > 0 else -(-(n - 1) // cfg.D), cfg.D, rng)
     if cfg.tree == "uniform":
         return random_parent_tree(n, min(cfg.D, n - 1), rng)
     return topk_expansion_tree(n, cfg.D, cfg.topk, rng)

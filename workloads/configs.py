@@ -20,7 +20,7 @@ class VerifyConfig:
     N: int            # tree nodes including the root (= Nmax)
     D: int            # max depth (edges from the root)
     V: int            # vocabulary (0: config has no logits)
-    tree: str         # "uniform" | "topk"
+    tree: str         # "uniform" | "topk" | "spine" | "chains"
     topk: int
     P: int            # candidate-path rows (0: one row per leaf, capacity = N)
     std: float        # std of Q/K/V entries

@@ -94,6 +94,24 @@ def spine_tree(N, D, rng):
     return parent
 
 
+def covering_chains_tree(N, n_chains, D, rng):
+    """Chains hanging from the root whose root-to-leaf rows cover every node: N - 1 nodes spread over
+    `n_chains` chains of depth <= D, as long as possible, the shorter ones at seeded positions (for N = 60,
+    ten chains, D = 6: nine chains of depth 6 and one of depth 5 - the only kind of 60-node tree whose ten
+    candidate rows of seven columns name all of its nodes).  Node ids run chain by chain."""
+    assert n_chains >= 1 and n_chains <= N - 1 <= n_chains * D
+    base, extra = divmod(N - 1, n_chains)
+    lengths = np.full(n_chains, base, dtype=np.int64)
+    lengths[rng.permutation(n_chains)[:extra]] += 1
+    parent = np.full(N, -1, dtype=np.int32)
+    i = 1
+    for ln in lengths:
+        for k in range(int(ln)):
+            parent[i] = 0 if k == 0 else i - 1
+            i += 1
+    return parent
+
+
 def chain_tree(N):
     """0 <- 1 <- 2 ... : the linear speculative proposal of Section 2.2."""
     return np.arange(-1, N - 1, dtype=np.int32)
