@@ -773,8 +773,54 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           if (jt == 0) prof[10] += pc1 - pitem;
 #endif
           tr.mark(0x1000u | (tj & 0xfffu));
+          // ---- whole-tile fast path (full, unmasked tiles after the first of the item): all 128 scores of the
+          // row in one load and P with the reference maximum as it stands; the row sum then tells whether
+          // anything left the lazy-rescale range (all P are >= 0, so the sum bounds every element; NaN and
+          // infinity fail the comparison).  P is only stored once the check has passed, so on a failure the
+          // scores are still in S and the chunk loop below does the tile again, maximum first.
+          bool tile_done = false;
+          if (jt > 0 && !tree && valid_keys == kTileN) {
+            uint32_t sall[128];
+            tmem_ld32(s_base, sall);
+            tmem_ld32(s_base + 32, sall + 32);
+            tmem_ld32(s_base + 64, sall + 64);
+            tmem_ld32(s_base + 96, sall + 96);
+            tmem_wait_ld();
+            const float* sa = reinterpret_cast<const float*>(sall);
+            const float2 c2 = make_float2(prm.scale_log2e, prm.scale_log2e);
+            const float nm = (m_used == -INFINITY) ? 0.f : -m_used;
+            const float2 nm2 = make_float2(nm, nm);
+            float2 sum = make_float2(0.f, 0.f);
+            uint32_t pkk[64];
 #pragma unroll
-          for (int h = 0; h < 2; ++h) {
+            for (int i = 0; i < 64; ++i) {
+              const float2 x = ffma2(make_float2(sa[2 * i], sa[2 * i + 1]), c2, nm2);
+              float2 pv;
+              if (TV_POLY_SEL(i)) {
+                pv = exp2_poly2(x);
+              } else {
+                pv.x = fast_exp2(x.x);
+                pv.y = fast_exp2(x.y);
+              }
+              sum = fadd2(sum, pv);
+              pkk[i] = pack_bf16(pv.x, pv.y);
+            }
+            const float fsum = sum.x + sum.y;
+            const bool overflow = row_active && !(fsum <= 2.f * kMaxFastSum);
+            if (!__any_sync(0xffffffffu, overflow)) {
+              l_sum += fsum;
+#pragma unroll
+              for (int q = 0; q < 8; ++q)
+                asm volatile(
+                    "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                    ::"r"(s_base + q * 8), "r"(pkk[q * 8 + 0]), "r"(pkk[q * 8 + 1]), "r"(pkk[q * 8 + 2]), "r"(pkk[q * 8 + 3]),
+                      "r"(pkk[q * 8 + 4]), "r"(pkk[q * 8 + 5]), "r"(pkk[q * 8 + 6]), "r"(pkk[q * 8 + 7])
+                    : "memory");
+              tile_done = true;
+            }
+          }
+#pragma unroll
+          for (int h = 0; h < 2 && !tile_done; ++h) {
             const int valid_half = min(64, max(0, valid_keys - 64 * h));
             uint32_t sreg[64];
             const uint32_t s_addr = s_base + h * 64;
@@ -807,44 +853,9 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             }
             uint32_t pk[32];                 // P of this chunk, bf16 pairs
             const bool first = (jt == 0 && h == 0);
-            // Full, unmasked chunks after the first keep the reference maximum, compute P directly and only
-            // check afterwards (from the row sum) that nothing left the lazy-rescale range.  Every other
-            // chunk, and a chunk that fails the check, takes the true maximum first.
-            bool with_max = first || masked;
-            if (!with_max) {
-              const float2 c2 = make_float2(prm.scale_log2e, prm.scale_log2e);
-              const float nm = (m_used == -INFINITY) ? 0.f : -m_used;
-              const float2 nm2 = make_float2(nm, nm);
-              float2 sum = make_float2(0.f, 0.f);
-#pragma unroll
-              for (int i = 0; i < 32; ++i) {
-                const float2 x = ffma2(make_float2(s[2 * i], s[2 * i + 1]), c2, nm2);
-                float2 pv;
-#ifdef TV_EXP_SKIP_EXP
-                if (true) {
-                  pv = x;
-                } else
-#endif
-                if (TV_POLY_SEL(i)) {
-                  pv = exp2_poly2(x);
-                } else {
-                  pv.x = fast_exp2(x.x);
-                  pv.y = fast_exp2(x.y);
-                }
-                sum = fadd2(sum, pv);
-                pk[i] = pack_bf16(pv.x, pv.y);
-              }
-              // All P are >= 0, so the row sum bounds every element: a sum inside the accepted range means
-              // no element overflowed it (NaN and infinity fail the comparison).
-              const float fsum = sum.x + sum.y;
-              const bool overflow = row_active && !(fsum <= kMaxFastSum);
-              if (!__any_sync(0xffffffffu, overflow)) {
-                l_sum += fsum;
-              } else {
-                with_max = true;
-              }
-            }
-            if (with_max) {
+            // the tiles that get here (first of an item, masked, or rejected by the fast path) take the true
+            // maximum of the chunk first
+            {
               float mx0 = s[0], mx1 = s[1], mx2_ = s[2], mx3 = s[3];
 #pragma unroll
               for (int c = 4; c < 64; c += 4) {
