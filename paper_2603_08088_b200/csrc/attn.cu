@@ -124,6 +124,12 @@ __device__ __forceinline__ void fence_proxy_async_smem() {
 // this grid has got here or has exited.
 __device__ __forceinline__ void gdc_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void gdc_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+// One lane of a converged warp (the compiler keeps what it guards in the uniform datapath).
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+  return pred != 0;
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -567,13 +573,13 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     //     that the softmax of one row tile runs while the pipe works for the other one;
     //   one row tile (buffers alternate by key tile):  S_next = Q K_next^T -> wait P -> O += P V.
     asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
-    if (lane == 0 && !*abort_flag) {
+    if (!*abort_flag) {      // the whole warp walks the items; one elected lane issues
       int g = g_begin;
       Item it;
       uint32_t item_idx = 0, fill = 0, tj = 0;
       bool ok = true;
       Tracer tr;
-      tr.init(prm.trace, 1);
+      tr.init(lane == 0 ? prm.trace : nullptr, 1);
       tr.mark(0);
       // descriptor words: low = start address >> 4 | LBO field, high = SBO 1024 B | version 1 | 128-byte swizzle
       const uint32_t desc_hi = (uint32_t)(smem_desc(0, 0, 1024) >> 32);
@@ -584,21 +590,29 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       // S(buf) = Q_t K^T for the 128 keys of the K tile in `slot`
       auto issue_qk = [&](int t, int buf, uint32_t slot) {
         const uint32_t qa = q_lo + t * kTile16, ka = k_lo + slot * kTile16;
+        if (elect_one()) {
 #pragma unroll
-        for (int ks = 0; ks < D / 16; ++ks) {
-          const uint32_t off = (ks / 4) * kHalf16 + (ks % 4) * 2;        // 16 columns = 32 bytes inside a swizzled row
-          mma_ss_lohi(tmem + kTmemS0 + buf * 128, qa + off, ka + off, desc_hi, kIdescQK, ks > 0);
+          for (int ks = 0; ks < D / 16; ++ks) {
+            const uint32_t off = (ks / 4) * kHalf16 + (ks % 4) * 2;        // 16 columns = 32 bytes inside a swizzled row
+            mma_ss_lohi(tmem + kTmemS0 + buf * 128, qa + off, ka + off, desc_hi, kIdescQK, ks > 0);
+          }
+          mma_commit(bar(L::S_FULL + buf));
         }
-        mma_commit(bar(L::S_FULL + buf));
+        __syncwarp();
       };
       // O_t += P(buf) V for the 128 keys of the V tile in `slot`
       auto issue_pv = [&](int t, int buf, uint32_t slot, bool first_tile) {
         const uint32_t va = v_lo + slot * kTile16;
+        if (elect_one()) {
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks)            // 16 keys = 16 rows of 128 bytes = 8 packed P columns
-          mma_ts_lohi(tmem + kTmemO0 + t * 128, tmem + kTmemS0 + buf * 128 + ks * 8, va + ks * 128, desc_hi, kIdescPV,
-                      (!first_tile || ks > 0) ? 1u : 0u);
-        mma_commit(bar(L::O_DONE + t));
+          for (int ks = 0; ks < 8; ++ks)            // 16 keys = 16 rows of 128 bytes = 8 packed P columns
+            mma_ts_lohi(tmem + kTmemO0 + t * 128, tmem + kTmemS0 + buf * 128 + ks * 8, va + ks * 128, desc_hi, kIdescPV,
+                        (!first_tile || ks > 0) ? 1u : 0u);
+        // With two row tiles the S tile that the softmax waits for next is committed after this PV, so its
+        // completion is known without a commit of its own (a commit stalls the pipe for some 45 cycles).
+          if (MT == 1) mma_commit(bar(L::O_DONE + t));
+        }
+        __syncwarp();
       };
       while (ok && next_item(g, it)) {
         const int nt = it.j1 - it.j0;
@@ -616,8 +630,8 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           } else {
             issue_qk(0, tj & 1, slot);
           }
-          mma_commit(bar(L::KV_EMPTY + slot));
-          if (nt == 1) mma_commit(bar(L::Q_EMPTY));
+          if (elect_one()) mma_commit(bar(L::KV_EMPTY + slot));
+          if (nt == 1 && elect_one()) mma_commit(bar(L::Q_EMPTY));
         }
         for (int jt = 0; jt < nt && ok; ++jt, ++tj) {
           const uint32_t fv = fill + 2 * jt + 1, vslot = fv % kSlots;
@@ -636,7 +650,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               tc_fence_after();
               tr.mark(0x4000u | ((2 * tj + t) & 0xfffu));
               issue_pv(t, t, vslot, jt == 0);
-              if (!more) mma_commit(bar(L::ITEM_DONE + t));      // all MMAs of the item's row tile are done
+              if (!more && elect_one()) mma_commit(bar(L::ITEM_DONE + t));      // all MMAs of the item's row tile are done
               if (more) issue_qk(t, t, kslot);
               tr.mark(0x2000u | ((2 * tj + t) & 0xfffu));
             }
@@ -655,12 +669,15 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             tc_fence_after();
             tr.mark(0x4000u | (tj & 0xfffu));
             issue_pv(0, buf, vslot, jt == 0);
-            if (!more) mma_commit(bar(L::ITEM_DONE));
+            if (!more && elect_one()) mma_commit(bar(L::ITEM_DONE));
             tr.mark(0x2000u | (tj & 0xfffu));
           }
-          mma_commit(bar(L::KV_EMPTY + vslot));
-          if (more) mma_commit(bar(L::KV_EMPTY + kslot));
-          if (jt + 2 == nt) mma_commit(bar(L::Q_EMPTY));
+          if (elect_one()) {
+            mma_commit(bar(L::KV_EMPTY + vslot));
+            if (more) mma_commit(bar(L::KV_EMPTY + kslot));
+            if (jt + 2 == nt) mma_commit(bar(L::Q_EMPTY));
+          }
+          __syncwarp();
         }
         fill += 2 * nt;
         ++item_idx;
@@ -875,8 +892,10 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               l_sum *= alpha;
               if (__any_sync(0xffffffffu, scales)) {
                 tr.mark(0x9000u | (tj & 0xfffu));
-                // the PV of the previous key tile may still be running: wait for its completion (number tj - 1)
-                ok = wwait(bar(L::O_DONE + wg), (tj - 1) & 1);
+                // O must be at rest.  With two row tiles the PV of the previous key tile was issued before the
+                // S = Q K^T this warpgroup has just waited for, and the pipe runs in issue order: it is done.
+                // With one row tile the next S is issued ahead of the PV: wait for its completion (number tj - 1).
+                if (MT == 1) ok = wwait(bar(L::O_DONE + wg), (tj - 1) & 1);
                 if (!ok) break;
                 tc_fence_after();
 #pragma unroll 1
