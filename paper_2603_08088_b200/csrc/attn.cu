@@ -489,13 +489,13 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   if (warp == 0) {
     // =========================================================== TMA producer
     asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
-    if (lane == 0 && !*abort_flag) {
+    if (!*abort_flag) {        // the whole warp walks the items; one elected lane issues the copies
       int g = g_begin;
       Item it;
       uint32_t item_idx = 0, fill = 0;
       bool ok = true;
       Tracer tr;
-      tr.init(prm.trace, 0);
+      tr.init(lane == 0 ? prm.trace : nullptr, 0);
       tr.mark(0);
       uint64_t kv_policy;      // the committed prefix is streamed once: first in line for eviction from L2
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(kv_policy));
@@ -507,17 +507,21 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       bool synced = false;
       auto sync_with_predecessor = [&]() {
         gdc_wait();
-        gdc_launch_dependents();
+        if (elect_one()) gdc_launch_dependents();
+        __syncwarp();
         synced = true;
       };
       auto load_q = [&]() {
-        mbar_expect_tx(bar(L::Q_FULL), MT * (D / 64) * prm.q_box_bytes);
+        if (elect_one()) {
+          mbar_expect_tx(bar(L::Q_FULL), MT * (D / 64) * prm.q_box_bytes);
 #pragma unroll
-        for (int t = 0; t < MT; ++t)
+          for (int t = 0; t < MT; ++t)
 #pragma unroll
-          for (int h = 0; h < D / 64; ++h)
-            tma_load_4d(sbase + L::kQ + t * L::kTileBytes + h * L::kHalf, &map_q, bar(L::Q_FULL), h * 64,
-                        it.hk * prm.G, (pair * MT + t) * prm.NPT, it.b);
+            for (int h = 0; h < D / 64; ++h)
+              tma_load_4d(sbase + L::kQ + t * L::kTileBytes + h * L::kHalf, &map_q, bar(L::Q_FULL), h * 64,
+                          it.hk * prm.G, (pair * MT + t) * prm.NPT, it.b);
+        }
+        __syncwarp();
       };
       while (ok && next_item(g, it)) {
         ok = mbar_wait(bar(L::Q_EMPTY), (item_idx & 1) ^ 1, abort_flag);
@@ -540,16 +544,19 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             ok = mbar_wait(bar(L::KV_EMPTY + slot), (round & 1) ^ 1, abort_flag);
             if (!ok) break;
             tr.mark(0x2000u | (fill & 0xfffu));
-            mbar_expect_tx(bar(L::KV_FULL + slot), L::kTileBytes);
             const uint32_t dst = sbase + L::kRing + slot * L::kTileBytes;
+            if (elect_one()) {
+              mbar_expect_tx(bar(L::KV_FULL + slot), L::kTileBytes);
 #pragma unroll
-            for (int h = 0; h < D / 64; ++h) {
-              if (tree)
-                tma_load_4d(dst + h * L::kHalf, kv ? &map_vt : &map_kt, bar(L::KV_FULL + slot), h * 64, it.hk, tt * kTileN, it.b);
-              else
-                tma_load_3d_hint(dst + h * L::kHalf, kv ? &map_vc : &map_kc, bar(L::KV_FULL + slot), h * 64, j * kTileN,
-                                 it.b * prm.Hkv + it.hk, kv_policy);
+              for (int h = 0; h < D / 64; ++h) {
+                if (tree)
+                  tma_load_4d(dst + h * L::kHalf, kv ? &map_vt : &map_kt, bar(L::KV_FULL + slot), h * 64, it.hk, tt * kTileN, it.b);
+                else
+                  tma_load_3d_hint(dst + h * L::kHalf, kv ? &map_vc : &map_kc, bar(L::KV_FULL + slot), h * 64, j * kTileN,
+                                   it.b * prm.Hkv + it.hk, kv_policy);
+              }
             }
+            __syncwarp();
             ++fill;
           }
         }
@@ -559,9 +566,9 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
       }
       if (!synced) sync_with_predecessor();        // a CTA without work still has to let the next kernel go
-    } else if (lane == 0) {
+    } else {
       gdc_wait();
-      gdc_launch_dependents();
+      if (elect_one()) gdc_launch_dependents();
     }
   } else if (warp == 1) {
     // =========================================================== MMA issuer
