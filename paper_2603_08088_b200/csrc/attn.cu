@@ -752,11 +752,17 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         int claim_cnt = 0;
         if (piece && threadIdx.x == 128) claim_assumed = *reinterpret_cast<volatile unsigned long long*>(claim_ctr);
         const uint32_t o_addr_loop = tmem + lane_addr + kTmemO0 + wg * 128;
+        // key tiles below this index are full tiles of the committed prefix (no mask of any kind)
+        const int j_full = min(it.S / kTileN, it.len - prm.TT);
         for (int jt = 0; jt < nt && ok; ++jt, ++tj) {
           const int j = it.j0 + jt;
-          const int tt = j - (it.len - prm.TT);      // >= 0: index of the tree key tile
+          const bool full_tile = j < j_full;
+          int tt = -1, valid_keys = kTileN;          // tt >= 0: index of the tree key tile
+          if (!full_tile) {
+            tt = j - (it.len - prm.TT);
+            valid_keys = tt >= 0 ? max(0, min(kTileN, it.n - tt * kTileN)) : min(kTileN, it.S - j * kTileN);
+          }
           const bool tree = tt >= 0;
-          const int valid_keys = tree ? max(0, min(kTileN, it.n - tt * kTileN)) : min(kTileN, it.S - j * kTileN);
           if (piece && threadIdx.x == 128 && jt == nt - 1) {
             claim_cnt = ((claim_assumed >> 16) == prm.epoch) ? (int)(claim_assumed & 0xffffu) : 0;
             claim_ret = atomicCAS(claim_ctr, claim_assumed, (prm.epoch << 16) | (unsigned long long)(claim_cnt + 1));
@@ -803,7 +809,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           // infinity fail the comparison).  P is only stored once the check has passed, so on a failure the
           // scores are still in S and the chunk loop below does the tile again, maximum first.
           bool tile_done = false;
-          if (jt > 0 && !tree && valid_keys == kTileN) {
+          if (jt > 0 && full_tile) {
             uint32_t sall[128];
             tmem_ld32(s_base, sall);
             tmem_ld32(s_base + 32, sall + 32);
