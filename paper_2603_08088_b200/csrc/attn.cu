@@ -130,6 +130,11 @@ __device__ __forceinline__ bool elect_one() {
   asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
   return pred != 0;
 }
+// 32 bytes per thread in one store (a whole sector); the address must be 32-byte aligned.
+__device__ __forceinline__ void st_global_32B(void* p, uint4 a, uint4 b) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w),
+               "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w) : "memory");
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -301,6 +306,7 @@ struct AttnParams {
   int TT;                        // key tiles of the tree's own K/V: ceil(Nmax / 128), 1 or 2
   uint32_t q_box_bytes;
   unsigned long long* trace;     // optional event trace [cta][role 0..3][kTraceCap] of (tag << 48 | ns), or NULL          // bytes of one Q box {64, G, NPT}: 16 KB when G divides 128
+  int out_al32;                  // out is 32-byte aligned: rows can be written 32 bytes per thread and store
   float scale_log2e;             // scale * log2(e)
   float scale;
 };
@@ -995,15 +1001,21 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               tmem_ld32(o_addr + q * 32, o);
               tmem_wait_ld();
               if (do_store) {
+                uint4 v[4];
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
-                  uint4 v;
-                  v.x = pack_bf16(__uint_as_float(o[8 * c + 0]) * inv, __uint_as_float(o[8 * c + 1]) * inv);
-                  v.y = pack_bf16(__uint_as_float(o[8 * c + 2]) * inv, __uint_as_float(o[8 * c + 3]) * inv);
-                  v.z = pack_bf16(__uint_as_float(o[8 * c + 4]) * inv, __uint_as_float(o[8 * c + 5]) * inv);
-                  v.w = pack_bf16(__uint_as_float(o[8 * c + 6]) * inv, __uint_as_float(o[8 * c + 7]) * inv);
-                  if (zero) v = make_uint4(0, 0, 0, 0);       // rows of padded nodes: O may hold anything
-                  dst[(size_t)(q * 4 + c) * stride_u4] = v;
+                  v[c].x = pack_bf16(__uint_as_float(o[8 * c + 0]) * inv, __uint_as_float(o[8 * c + 1]) * inv);
+                  v[c].y = pack_bf16(__uint_as_float(o[8 * c + 2]) * inv, __uint_as_float(o[8 * c + 3]) * inv);
+                  v[c].z = pack_bf16(__uint_as_float(o[8 * c + 4]) * inv, __uint_as_float(o[8 * c + 5]) * inv);
+                  v[c].w = pack_bf16(__uint_as_float(o[8 * c + 6]) * inv, __uint_as_float(o[8 * c + 7]) * inv);
+                  if (zero) v[c] = make_uint4(0, 0, 0, 0);       // rows of padded nodes: O may hold anything
+                }
+                if (stride_u4 == 1 && prm.out_al32) {     // a row of the output: whole 32-byte sectors per store
+                  st_global_32B(dst + q * 4, v[0], v[1]);
+                  st_global_32B(dst + q * 4 + 2, v[2], v[3]);
+                } else {
+#pragma unroll
+                  for (int c = 0; c < 4; ++c) dst[(size_t)(q * 4 + c) * stride_u4] = v[c];
                 }
               }
             }
@@ -1163,14 +1175,22 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 }
                 if (row_exists) {
 #pragma unroll
-                  for (int c = 0; c < 8; ++c) {
-                    uint4 v;
-                    v.x = pack_bf16(acc[8 * c + 0] * inv, acc[8 * c + 1] * inv);
-                    v.y = pack_bf16(acc[8 * c + 2] * inv, acc[8 * c + 3] * inv);
-                    v.z = pack_bf16(acc[8 * c + 4] * inv, acc[8 * c + 5] * inv);
-                    v.w = pack_bf16(acc[8 * c + 6] * inv, acc[8 * c + 7] * inv);
-                    if (!row_active) v = make_uint4(0, 0, 0, 0);
-                    *reinterpret_cast<uint4*>(orow + hq * 64 + c * 8) = v;
+                  for (int c = 0; c < 8; c += 2) {
+                    uint4 v[2];
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                      v[e].x = pack_bf16(acc[8 * (c + e) + 0] * inv, acc[8 * (c + e) + 1] * inv);
+                      v[e].y = pack_bf16(acc[8 * (c + e) + 2] * inv, acc[8 * (c + e) + 3] * inv);
+                      v[e].z = pack_bf16(acc[8 * (c + e) + 4] * inv, acc[8 * (c + e) + 5] * inv);
+                      v[e].w = pack_bf16(acc[8 * (c + e) + 6] * inv, acc[8 * (c + e) + 7] * inv);
+                      if (!row_active) v[e] = make_uint4(0, 0, 0, 0);
+                    }
+                    if (prm.out_al32) {
+                      st_global_32B(orow + hq * 64 + c * 8, v[0], v[1]);
+                    } else {
+                      *reinterpret_cast<uint4*>(orow + hq * 64 + c * 8) = v[0];
+                      *reinterpret_cast<uint4*>(orow + hq * 64 + c * 8 + 8) = v[1];
+                    }
                   }
                 }
               }
@@ -1409,6 +1429,7 @@ extern "C" int tree_verify_attn(const tv_bf16* q,
   prm.G = g.G; prm.NPT = g.NPT; prm.NP = g.NP; prm.W = (Nmax + 31) / 32; prm.groups = g.groups;
   prm.TT = (Nmax + kTileN - 1) / kTileN;
   prm.scale = scale;
+  prm.out_al32 = (reinterpret_cast<uintptr_t>(out) & 31u) == 0 ? 1 : 0;
   prm.q_box_bytes = 64u * (uint32_t)g.G * (uint32_t)g.NPT * 2u;
   prm.trace = g_trace.load(std::memory_order_relaxed);
   prm.scale_log2e = scale * kLog2e;
