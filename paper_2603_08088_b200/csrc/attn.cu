@@ -698,6 +698,10 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     }
   } else if (warp >= 4) {
     // =========================================================== softmax / epilogue warpgroups
+    // Register budget: the CTA starts with 168 registers per thread; warps 0-3 give up 96 each (168 -> 72) and
+    // warps 4-11 take 48 each (168 -> 216).  4 x 96 = 8 x 48: the increase below can only complete once the
+    // other warpgroup has released enough, so any other split has to keep 4 (168 - low) >= 8 (high - 168) or the
+    // kernel never gets past this instruction.
     asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
     const int wg = (warp - 4) >> 2;                  // row tile of this warpgroup
     const int row = ((warp & 3) << 5) | lane;        // TMEM lane = row inside the tile
