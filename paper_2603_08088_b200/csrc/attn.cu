@@ -741,6 +741,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       while (ok && next_item(g, it)) {
 #ifdef TV_PROF
         const unsigned int pitem = clock();
+        unsigned int ep[6], ep_kind = 0, ep_others = 0, ep_own = 0;
 #endif
         const int nt = it.j1 - it.j0;
         const int node = (pair * MT + wg) * prm.NPT + row / prm.G;
@@ -993,6 +994,9 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           prof[7] += pc1 - pc0;
 #endif
           tr.mark(0x5000u);
+#ifdef TV_PROF
+          for (int i = 0; i < 6; ++i) ep[i] = pc1;
+#endif
           const uint32_t o_addr = o_addr_loop;
           const bool whole = (it.j0 == 0 && it.j1 == it.len);
           const int h = it.hk * prm.G + gm;
@@ -1046,27 +1050,20 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             // and reads 512 contiguous bytes per instruction.
             constexpr int kRows = MT * 128;
             const int rr = wg * 128 + row;
-            // unit geometry in the virtual tile space: real tiles occupy [real0, uend)
+            // The unit's real tiles occupy [real0, uend) of the virtual tile space.  CTA groups k_first..k_last
+            // hold them, one piece each (a group between the two lies wholly inside the unit), and this CTA's
+            // group is one of them: two short walks over the cut table find both ends.
             const int real0 = prm.Hkv * cum[it.b] + it.hk * (it.len + kSetupCost) + kSetupCost;
             const int uend = real0 + it.len;
-            const int k_first = sch.find_group(real0, groups);
-            const int k_last = sch.find_group(uend - 1, groups);
-            // slot of the piece CTA group k holds of this unit, or -1 if it holds none
-            auto piece_slot = [&](int k) -> int {
-              const int ks = gs[k], ke = gs[k + 1];
-              const int lo = ks > real0 ? ks : real0, hi = ke < uend ? ke : uend;
-              if (lo >= hi) return -1;
-              return (k * prm.NP + pair) * 2 + (ks > real0 ? 0 : 1);
-            };
-            const int my_slot = blockIdx.x * 2 + (it.j0 > 0 ? 0 : 1);
-            int n_frag = 0;
-#pragma unroll 1
-            for (int k = k_first; k <= k_last; ++k) {
-              const int sid = piece_slot(k);
-              if (sid < 0) continue;
-              ++n_frag;
-            }
+            int k_first = group, k_last = group;
+            while (gs[k_first] > real0) --k_first;
+            while (gs[k_last + 1] < uend) ++k_last;
+            const int n_frag = k_last - k_first + 1;
+            // slot of the piece CTA group k holds: slot 1 of its CTA if the unit starts in that group, else slot 0
+            auto piece_slot = [&](int k) -> int { return (k * prm.NP + pair) * 2 + (k == k_first ? 1 : 0); };
+            const int my_slot = piece_slot(group);
             unsigned long long* ctr = prm.counters + (((size_t)it.b * prm.Hkv + it.hk) * prm.NP + pair) * 2;
+            TV_PROF_T(ep[1]);
             if (threadIdx.x == 128) {
               int ticket;
               if (claim_ret == claim_assumed) {
@@ -1094,6 +1091,10 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             ok = epi_sync();
             if (!ok || *abort_flag) { ok = false; break; }
             tr.mark(0x7000u | (*last_flag ? 1u : 0u));
+            TV_PROF_T(ep[2]);
+#ifdef TV_PROF
+            ep_kind = (*last_flag ? 2u : 1u) | ((unsigned)n_frag << 4);
+#endif
             const float inv_own = (row_active && l_sum > 0.f) ? 1.f / l_sum : 0.f;
             if (!*last_flag) {
               uint4* po = reinterpret_cast<uint4*>(prm.part_o) + (size_t)my_slot * (D / 8) * kRows;
@@ -1104,51 +1105,70 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 pml[kRows + rr] = l_sum;
               }
               tc_fence_before();
+              TV_PROF_T(ep[3]);
               __threadfence();
+              TV_PROF_T(ep[4]);
               tr.mark(0x6000u);
               ok = epi_sync();
               if (!ok) break;
+              TV_PROF_T(ep[5]);
               if (threadIdx.x == 128) {
                 const unsigned long long seen = *reinterpret_cast<volatile unsigned long long*>(ctr + 1);
                 bump_counter(ctr + 1, seen, prm.epoch);
               }
             } else {
-              // ---- pass 1: reference maximum and total weight of the row, pieces in order.  Loads are issued
-              // by every thread (row rr always lies inside a slot; rows that are not active read stale bytes
-              // and are masked by selects): no thread-divergent branch sits between the warp-wide TMEM ops.
-              float mm = m_used, lt = 0.f;
-#pragma unroll 1
-              for (int k = k_first; k <= k_last; ++k) {
-                const int sid = piece_slot(k);
-                if (sid < 0 || sid == my_slot) continue;
-                mm = fmaxf(mm, __ldcg(prm.part_ml + (size_t)sid * 2 * kRows + rr));
+              // ---- pass 1: reference maximum and total weight of the row.  (m, l) of the first four pieces
+              // are fetched together (one round trip; a unit rarely has more), the rest one by one.  Loads are
+              // issued by every thread (row rr always lies inside a slot; rows that are not active read stale
+              // bytes and are masked by selects): no thread-divergent branch sits between the warp-wide TMEM ops.
+              float pm[4], w4[4];
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const int k = k_first + i;
+                const bool other = k <= k_last && k != group;
+                const float* q_ml = prm.part_ml + (size_t)piece_slot(other ? k : group) * 2 * kRows;
+                const float m_k = __ldcg(q_ml + rr), l_k = __ldcg(q_ml + kRows + rr);
+                pm[i] = other ? m_k : (k == group ? m_used : -INFINITY);
+                w4[i] = other ? l_k : (k == group ? l_sum : 0.f);
               }
+              float mm = fmaxf(fmaxf(pm[0], pm[1]), fmaxf(pm[2], pm[3]));
 #pragma unroll 1
-              for (int k = k_first; k <= k_last; ++k) {
-                const int sid = piece_slot(k);
-                if (sid < 0) continue;
-                if (sid == my_slot) {
-                  lt = fmaf(l_sum * fast_exp2(m_used - mm), 1.f, lt);
-                } else {
-                  const float* q_ml = prm.part_ml + (size_t)sid * 2 * kRows;
-                  lt = fmaf(__ldcg(q_ml + kRows + rr) * fast_exp2(__ldcg(q_ml + rr) - mm), 1.f, lt);
-                }
+              for (int k = k_first + 4; k <= k_last; ++k)
+                mm = fmaxf(mm, k == group ? m_used : __ldcg(prm.part_ml + (size_t)piece_slot(k) * 2 * kRows + rr));
+              float lt = 0.f;
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {       // weights w_p = l_p 2^(m_p - mm), summed in piece order
+                w4[i] *= fast_exp2(pm[i] - mm);
+                lt += w4[i];
               }
+              auto late_weight = [&](int k) -> float {     // pieces past the fourth
+                if (k == group) return l_sum * fast_exp2(m_used - mm);
+                const float* q_ml = prm.part_ml + (size_t)piece_slot(k) * 2 * kRows;
+                return __ldcg(q_ml + kRows + rr) * fast_exp2(__ldcg(q_ml + rr) - mm);
+              };
+#pragma unroll 1
+              for (int k = k_first + 4; k <= k_last; ++k) lt += late_weight(k);
               if (!row_active) lt = 0.f;
               const float inv = (row_active && lt > 0.f) ? 1.f / lt : 0.f;
-              const float w_own = l_sum * fast_exp2(m_used - mm);
+              TV_PROF_USE(__float_as_uint(inv));
+              TV_PROF_T(ep[3]);
               // ---- pass 2: 64 output columns at a time, pieces in order (one fused multiply-add per piece and
-              // element); the own piece comes from TMEM and enters as its bf16-rounded normalised output
+              // element, two elements per instruction); the own piece comes from TMEM and enters as its
+              // bf16-rounded normalised output, like every other piece
+              const float2 inv_own2 = make_float2(inv_own, inv_own), inv2 = make_float2(inv, inv);
 #pragma unroll 1
               for (int hq = 0; hq < D / 64; ++hq) {
-                float acc[64];
+                float2 acc[32];
 #pragma unroll
-                for (int c = 0; c < 64; ++c) acc[c] = 0.f;
+                for (int c = 0; c < 32; ++c) acc[c] = make_float2(0.f, 0.f);
 #pragma unroll 1
                 for (int k = k_first; k <= k_last; ++k) {
-                  const int sid = piece_slot(k);
-                  if (sid < 0) continue;
-                  if (sid == my_slot) {
+                  const int i = k - k_first;
+                  float w = i == 0 ? w4[0] : (i == 1 ? w4[1] : (i == 2 ? w4[2] : w4[3]));
+                  if (i >= 4) w = late_weight(k);
+                  const float2 w2 = make_float2(w, w);
+                  if (k == group) {
+                    TV_PROF_T(pc0);
 #pragma unroll
                     for (int q = 0; q < 2; ++q) {
                       uint32_t o[32];
@@ -1156,28 +1176,35 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                       tmem_wait_ld();
 #pragma unroll
                       for (int c = 0; c < 16; ++c) {
-                        const uint32_t own = pack_bf16(__uint_as_float(o[2 * c]) * inv_own, __uint_as_float(o[2 * c + 1]) * inv_own);
-                        acc[q * 32 + 2 * c] = fmaf(w_own, __uint_as_float(own << 16), acc[q * 32 + 2 * c]);
-                        acc[q * 32 + 2 * c + 1] = fmaf(w_own, __uint_as_float(own & 0xffff0000u), acc[q * 32 + 2 * c + 1]);
+                        const float2 t = __fmul2_rn(make_float2(__uint_as_float(o[2 * c]), __uint_as_float(o[2 * c + 1])), inv_own2);
+                        const uint32_t own = pack_bf16(t.x, t.y);
+                        acc[q * 16 + c] = ffma2(w2, make_float2(__uint_as_float(own << 16), __uint_as_float(own & 0xffff0000u)),
+                                                acc[q * 16 + c]);
                       }
                     }
+#ifdef TV_PROF
+                    TV_PROF_USE(__float_as_uint(acc[31].y));
+                    ep_own += clock() - pc0;
+#endif
                     continue;
                   }
-                  const float* q_ml = prm.part_ml + (size_t)sid * 2 * kRows;
-                  const uint4* q_o = reinterpret_cast<const uint4*>(prm.part_o) + (size_t)sid * (D / 8) * kRows;
+                  const uint4* q_o = reinterpret_cast<const uint4*>(prm.part_o) + (size_t)piece_slot(k) * (D / 8) * kRows;
                   uint4 v[8];
+                  TV_PROF_T(pc0);
 #pragma unroll
                   for (int c = 0; c < 8; ++c) v[c] = __ldcg(q_o + (size_t)(hq * 8 + c) * kRows + rr);
-                  const float w = __ldcg(q_ml + kRows + rr) * fast_exp2(__ldcg(q_ml + rr) - mm);
 #pragma unroll
                   for (int c = 0; c < 8; ++c) {
                     const uint32_t wv[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                      acc[8 * c + 2 * e] = fmaf(w, __uint_as_float(wv[e] << 16), acc[8 * c + 2 * e]);
-                      acc[8 * c + 2 * e + 1] = fmaf(w, __uint_as_float(wv[e] & 0xffff0000u), acc[8 * c + 2 * e + 1]);
-                    }
+                    for (int e = 0; e < 4; ++e)
+                      acc[4 * c + e] = ffma2(w2, make_float2(__uint_as_float(wv[e] << 16), __uint_as_float(wv[e] & 0xffff0000u)),
+                                             acc[4 * c + e]);
                   }
+#ifdef TV_PROF
+                  TV_PROF_USE(__float_as_uint(acc[31].y));
+                  ep_others += clock() - pc0;
+#endif
                 }
                 if (row_exists) {
 #pragma unroll
@@ -1185,10 +1212,13 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     uint4 v[2];
 #pragma unroll
                     for (int e = 0; e < 2; ++e) {
-                      v[e].x = pack_bf16(acc[8 * (c + e) + 0] * inv, acc[8 * (c + e) + 1] * inv);
-                      v[e].y = pack_bf16(acc[8 * (c + e) + 2] * inv, acc[8 * (c + e) + 3] * inv);
-                      v[e].z = pack_bf16(acc[8 * (c + e) + 4] * inv, acc[8 * (c + e) + 5] * inv);
-                      v[e].w = pack_bf16(acc[8 * (c + e) + 6] * inv, acc[8 * (c + e) + 7] * inv);
+                      float2 t[4];
+#pragma unroll
+                      for (int x = 0; x < 4; ++x) t[x] = __fmul2_rn(acc[4 * (c + e) + x], inv2);
+                      v[e].x = pack_bf16(t[0].x, t[0].y);
+                      v[e].y = pack_bf16(t[1].x, t[1].y);
+                      v[e].z = pack_bf16(t[2].x, t[2].y);
+                      v[e].w = pack_bf16(t[3].x, t[3].y);
                       if (!row_active) v[e] = make_uint4(0, 0, 0, 0);
                     }
                     if (prm.out_al32) {
@@ -1202,14 +1232,22 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               }
               if (row_exists && lse_p) *lse_p = (row_active && lt > 0.f) ? (mm + log2f(lt)) / kLog2e : -INFINITY;
               tc_fence_before();
+              TV_PROF_T(ep[4]);
               ok = epi_sync();   // keeps the two warpgroups' barrier phases in step with the other branch
               if (!ok) break;
+              TV_PROF_T(ep[5]);
             }
           }
         }
         tr.mark(0x8000u);
 #ifdef TV_PROF
         prof[8] += clock() - pc1;
+        if (tr.base && prof[9] < 24) {
+          unsigned long long* e = tr.base + prof[9] * 8;
+          e[0] = ep_kind; e[1] = ep_own;
+          for (int i = 1; i < 6; ++i) e[1 + i] = ep[i] - ep[i - 1];
+          e[7] = ep_others;      // pass 2: cycles from the loads of the other pieces to the end of their sums
+        }
         prof[9] += 1;
 #endif
         fill += 2 * nt;
