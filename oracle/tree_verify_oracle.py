@@ -393,6 +393,40 @@ def kv_commit(k_cache, v_cache, k_tree, v_tree, accepted_nodes, accept_len, pref
     return kc, vc, new_len, status
 
 
+def kv_commit_inplace(k_cache, v_cache, accepted_nodes, accept_len, prefix_len, Nmax, status_in=None):
+    """Path-index commit as a full reorder (Section 3.1, "Full reordering"),
+    for a cache the teacher forward extended in place: node i of the tree sits
+    at row S_b + i.  The new committed cache is the gather of the OLD one along
+    the sequence axis by path_indices = [0..S_b-1, S_b + accepted_nodes[b,0..A_b]]:
+    new[l,b,h,t,:] = old[l,b,h,path_indices[t],:] for t < S_b + A_b + 1.  Rows
+    below S_b map to themselves; rows at or past S_b + A_b + 1 are outside the
+    new committed length and keep their bytes.  Works on copies.  Skips and
+    flags a sequence as kv_commit does; a source row at or past the capacity
+    is a capacity error too.
+    """
+    kc, vc = k_cache.copy(), v_cache.copy()
+    L, B, Hkv, Scap, d = kc.shape
+    Dp1 = accepted_nodes.shape[1]
+    new_len = np.array(prefix_len, dtype=np.int32).copy()
+    status = np.zeros(B, dtype=np.int32) if status_in is None else np.array(status_in, dtype=np.int32).copy()
+    for b in range(B):
+        if status[b] & ST_FATAL:
+            continue
+        S, A = int(prefix_len[b]), int(accept_len[b])
+        if A < 0 or A >= Dp1 or any(not (0 <= int(accepted_nodes[b, j]) < Nmax) for j in range(A + 1)):
+            status[b] |= ST_BAD_INDEX
+            continue
+        if S < 0 or S + A + 1 > Scap or any(S + int(accepted_nodes[b, j]) >= Scap for j in range(A + 1)):
+            status[b] |= ST_CAPACITY
+            continue
+        path_indices = list(range(S)) + [S + int(accepted_nodes[b, j]) for j in range(A + 1)]
+        T = len(path_indices)
+        kc[:, b, :, :T, :] = k_cache[:, b][:, :, path_indices, :]      # gather from the old cache
+        vc[:, b, :, :T, :] = v_cache[:, b][:, :, path_indices, :]
+        new_len[b] = T
+    return kc, vc, new_len, status
+
+
 def verify_step(case_np, scale, Dcap=None, Pcap=None, use_given_retrieve=True):
     """One whole step in the paper's order: tensorise + mask, attention per
     layer, safe gather + argmax + accept, commit (Section 3 call order)."""

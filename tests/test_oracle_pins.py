@@ -486,6 +486,64 @@ def test_commit_equivalence_with_sequential_decoding():
     assert (kc3[0, 0, :, 7:11] == kt[0, 0:4].transpose(1, 0, 2)).all()
 
 
+def test_inplace_commit_worked_example_with_overlapping_rows():
+    """Full reorder inside the cache: the expected rows are typed out by hand.  Rows carry their own
+    index as content (row r holds the value 100 + r), prefix 3, tree of 6 nodes at rows 3..8, accepted
+    path {0, 2, 3}: row 5 (node 2) is the source of slot 1 AND the destination of slot 2, so a copy
+    that writes slot 2 before it reads slot 1's source would put 106 into row 4."""
+    L, B, Hkv, Scap, d, N = 1, 1, 1, 10, 2, 6
+    kc = np.zeros((L, B, Hkv, Scap, d), dtype=np.uint16)
+    kc[0, 0, 0, :, 0] = 100 + np.arange(Scap)
+    kc[0, 0, 0, :, 1] = 200 + np.arange(Scap)
+    vc = kc + 1000
+    nodes = np.array([[0, 2, 3, 0]], dtype=np.int32)
+    kc2, vc2, S2, st = orc.kv_commit_inplace(kc, vc, nodes, np.array([2]), np.array([3]), N)
+    assert st.tolist() == [0] and S2.tolist() == [6]
+    #            prefix rows 0..2   | slot0 = node0 (row 3) | slot1 = node2 (row 5) | slot2 = node3 (row 6) | stale rows
+    assert kc2[0, 0, 0, :, 0].tolist() == [100, 101, 102, 103, 105, 106, 106, 107, 108, 109]
+    assert kc2[0, 0, 0, :, 1].tolist() == [200, 201, 202, 203, 205, 206, 206, 207, 208, 209]
+    assert (vc2 == kc2 + 1000).all()
+    # a descending path order (not produced by a tree, but allowed by the definition) is still a gather
+    # from the old state: slot 1 <- old row 3+3, slot 2 <- old row 3+1
+    nodes = np.array([[0, 3, 1, 0]], dtype=np.int32)
+    kc3, _, _, _ = orc.kv_commit_inplace(kc, vc, nodes, np.array([2]), np.array([3]), N)
+    assert kc3[0, 0, 0, :, 0].tolist() == [100, 101, 102, 103, 106, 104, 106, 107, 108, 109]
+
+
+def test_inplace_commit_equals_separate_buffer_commit_and_flags():
+    """With the tree's rows placed behind the prefix, the in-cache reorder and the separate-buffer
+    commit give the same committed rows [0, S+A+1); a chain path is the identity (length-based commit);
+    capacity and index errors skip the sequence."""
+    rng = np.random.default_rng(15)
+    L, B, Hkv, Scap, d, N, Dp1 = 2, 3, 2, 24, 4, 7, 4
+    kt = rng.integers(0, 2 ** 16, size=(L, B, N, Hkv, d)).astype(np.uint16)
+    vt = rng.integers(0, 2 ** 16, size=(L, B, N, Hkv, d)).astype(np.uint16)
+    kc = rng.integers(0, 2 ** 16, size=(L, B, Hkv, Scap, d)).astype(np.uint16)
+    vc = rng.integers(0, 2 ** 16, size=(L, B, Hkv, Scap, d)).astype(np.uint16)
+    S = np.array([10, 0, 17], dtype=np.int32)
+    kin, vin = kc.copy(), vc.copy()
+    for b in range(B):                                   # the forward pass extended the cache in place
+        kin[:, b, :, S[b]:S[b] + N] = kt[:, b].transpose(0, 2, 1, 3)
+        vin[:, b, :, S[b]:S[b] + N] = vt[:, b].transpose(0, 2, 1, 3)
+    nodes = np.array([[0, 2, 5, 0], [0, 1, 2, 3], [0, 1, 3, 6]], dtype=np.int32)
+    A = np.array([2, 3, 3], dtype=np.int32)
+    k1, v1, S1, st1 = orc.kv_commit(kc, vc, kt, vt, nodes, A, S)
+    k2, v2, S2, st2 = orc.kv_commit_inplace(kin, vin, nodes, A, S, N)
+    assert st1.tolist() == st2.tolist() == [0, 0, 0] and S1.tolist() == S2.tolist() == [13, 4, 21]
+    for b in range(B):
+        assert (k1[:, b, :, :S1[b]] == k2[:, b, :, :S2[b]]).all() and (v1[:, b, :, :S1[b]] == v2[:, b, :, :S2[b]]).all()
+        assert (k2[:, b, :, S2[b]:] == kin[:, b, :, S2[b]:]).all()        # rows behind the segment untouched
+    assert (k2[:, 1] == kin[:, 1]).all()                                   # chain path: nothing moves
+    # a source row past the capacity, a bad node id, a fatal incoming status
+    _, _, S3, st3 = orc.kv_commit_inplace(kin, vin, nodes, A, np.array([10, 0, 18], dtype=np.int32), N)
+    assert st3.tolist() == [0, 0, orc.ST_CAPACITY] and S3[2] == 18
+    bad = nodes.copy()
+    bad[0, 1] = N
+    k4, _, S4, st4 = orc.kv_commit_inplace(kin, vin, bad, A, S, N, status_in=np.array([0, orc.ST_BAD_TREE, 0]))
+    assert st4.tolist() == [orc.ST_BAD_INDEX, orc.ST_BAD_TREE, 0] and S4.tolist() == [10, 0, 21]
+    assert (k4[:, :2] == kin[:, :2]).all()
+
+
 def test_node_scores_gather_and_link_to_greedy_acceptance():
     """score[k] = logits[parent(k), token(k)]: checked against numpy fancy indexing, and against the
     acceptance rule - a node is accepted by the greedy rule exactly when its score equals the row
