@@ -344,6 +344,9 @@ def run_ours(args, cfg):
     }
     if args.budget_sweep:
         line["budget_sweep"] = budget_sweep(args.seed, dev)
+    if args.in_cache and has_accept:
+        line["in_cache"] = in_cache_step(cfg, case, buf, prefix0, scale, given_rows, min(args.steps, 20), dev)
+        case["prefix_len"].copy_(prefix0)
     if args.context_split > 1:
         case["prefix_len"].copy_(prefix0)
         line["context_split"] = context_split_member(cfg, case, buf, args.context_split, dev)
@@ -394,6 +397,60 @@ def budget_sweep(seed, dev):
                      "hbm_frac": attn_algorithmic_bytes(cfg, S) / (us * 1e-6) / 1e9 / peak,
                      "tensor_tflops": attn_flops(cfg, S) / (us * 1e-6) / 1e12})
     return rows
+
+
+def in_cache_step(cfg, case, buf, prefix0, scale, given_rows, steps, dev):
+    """The same step with the in-cache layout (Section 3.1: the forward pass extends the cache in place; the
+    commit is a reorder inside the cache): the tree's K/V are written behind each prefix once, outside the
+    timed region, then mask, L x attention (tree tiles read from the cache), accept and kv_commit_inplace are
+    timed.  Every step starts from the same state: prefix_len is reset and the rows the commit moved are
+    written again (both outside the events of the commit, inside those of the step)."""
+    import paper_2603_08088_b200 as tv
+    N = cfg.N
+    S = prefix0.cpu().tolist()
+    if max(s + N for s in S) > cfg.Scap:
+        return {"skipped": "a tree does not fit behind its prefix"}
+    rows = [(b, s) for b, s in enumerate(S)]
+    tree_k = [case["k_tree"][:, b].permute(0, 2, 1, 3).contiguous() for b, _ in rows]
+    tree_v = [case["v_tree"][:, b].permute(0, 2, 1, 3).contiguous() for b, _ in rows]
+
+    def place():
+        for (b, s), tk, tvv in zip(rows, tree_k, tree_v):
+            case["k_cache"][:, b, :, s:s + N] = tk
+            case["v_cache"][:, b, :, s:s + N] = tvv
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    t_step, t_attn, t_commit = [], [], []
+    for it in range(3 + steps):
+        case["prefix_len"].copy_(prefix0)
+        place()
+        m = [ev() for _ in range(5)]
+        m[0].record()
+        tv.tree_build_mask(case["parent"], case["n_nodes"], cfg.D, buf.retrieve.shape[1], buf.anc_bits, buf.status,
+                           retrieve_indices=None if given_rows else buf.retrieve, n_paths=buf.n_paths)
+        m[1].record()
+        for l in range(cfg.L):
+            tv.tree_verify_attn(case["q"][l], case["k_cache"][l], case["v_cache"][l], None, None, case["prefix_len"],
+                                case["n_nodes"], buf.anc_bits, scale, buf.out[l], buf.attn_ws, buf.status)
+        m[2].record()
+        tv.tree_accept(case["logits"], case["tokens"], case["retrieve"] if given_rows else buf.retrieve, case["n_nodes"],
+                       buf.argmax_tok, buf.accept_len, buf.best_path, buf.accepted_nodes, buf.next_token, buf.accept_ws,
+                       buf.status)
+        m[3].record()
+        tv.kv_commit_inplace(case["k_cache"], case["v_cache"], buf.accepted_nodes, buf.accept_len, case["prefix_len"], N,
+                             buf.status)
+        m[4].record()
+        torch.cuda.synchronize()
+        if it >= 3:
+            t_step.append(m[0].elapsed_time(m[4]))
+            t_attn.append(m[1].elapsed_time(m[2]) / cfg.L)
+            t_commit.append(m[3].elapsed_time(m[4]))
+    if (buf.status.cpu().numpy() & 15).any():
+        raise SystemExit(f"bench.py: fatal status in the in-cache step: {buf.status.cpu().numpy()}")
+    med = lambda v: sorted(v)[len(v) // 2]
+    return {"steps": steps, "ms_per_step_median": med(t_step), "steps_per_sec": 1e3 / med(t_step),
+            "attn_per_layer_us": med(t_attn) * 1e3, "commit_inplace_us": med(t_commit) * 1e3,
+            "note": "tree K/V read from the cache rows behind the prefix; commit = reorder inside the cache"}
 
 
 def context_split_member(cfg, case, buf, R, dev):
@@ -450,6 +507,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     ap.add_argument("--budget-sweep", action="store_true",
                     help="also time tree_verify_attn over the node budgets of the paper's sweep (extra key in the JSON line)")
+    ap.add_argument("--in-cache", action="store_true",
+                    help="also time the step with the tree's K/V inside the cache and the in-place commit")
     ap.add_argument("--context-split", type=int, default=1,
                     help="also time one member of an R-way context split of the workload (extra key in the JSON line)")
     args = ap.parse_args()

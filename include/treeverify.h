@@ -115,7 +115,17 @@ TV_API size_t tv_attn_workspace_bytes(int B, int Nmax, int Hq, int Hkv, int d, i
  *                                      (state safety, Section 3.3); rows at
  *                                      or past prefix_len[b] are ignored even
  *                                      if they hold NaN.
- *   k_tree,v_tree[B,Nmax,Hkv,d]    in  bf16, the speculative ("branch") K/V
+ *   k_tree,v_tree[B,Nmax,Hkv,d]    in  bf16, the speculative ("branch") K/V;
+ *                                      or both NULL = in-cache layout: the
+ *                                      teacher forward extended the cache in
+ *                                      place (Section 3.1) and node i's K/V
+ *                                      are rows prefix_len[b] + i of k_cache /
+ *                                      v_cache, written behind the committed
+ *                                      prefix and not part of it until
+ *                                      kv_commit_inplace.  A tree that does not
+ *                                      fit (prefix_len[b] + n_nodes[b] > Scap)
+ *                                      gets TV_ST_CAPACITY and an unspecified
+ *                                      output.
  *   prefix_len[B], n_nodes[B]      in
  *   anc_bits[B,Nmax,W]             in  from tree_build_mask
  *   out[B,Nmax,Hq,d]               out bf16; padded rows are written as 0
@@ -265,7 +275,8 @@ TV_API int tree_accept_noalloc(const tv_bf16* logits, const int32_t* tokens,
  *                     TV_ST_BAD_INDEX if accept_len or a node id is out of
  *                     range; such a sequence is left untouched.
  * Must follow the last tree_verify_attn of the step on the same stream.
- * Limits: d*2 bytes a multiple of 16; tensors 16-byte aligned.
+ * Limits: d*2 bytes a multiple of 16; tensors 16-byte aligned; Dp1 <= 1024;
+ * L <= 65535.
  */
 TV_API int kv_commit(tv_bf16* k_cache, tv_bf16* v_cache,
               const tv_bf16* k_tree, const tv_bf16* v_tree,
@@ -273,6 +284,35 @@ TV_API int kv_commit(tv_bf16* k_cache, tv_bf16* v_cache,
               int32_t* prefix_len,
               int L, int B, int Nmax, int Hkv, int d, int Scap, int Dp1,
               int64_t cache_layer_stride, int64_t tree_layer_stride,
+              int32_t* status, tv_stream stream);
+
+/*
+ * Path-index commit as a full reorder inside the cache (Section 3.1, "full
+ * reordering"), for the in-cache layout of tree_verify_attn: node i's K/V are
+ * rows prefix_len[b] + i, and the accepted path is gathered to the front of
+ * that region, for all layers in one call:
+ *   cache[l,b,h,S+j,:] = OLD cache[l,b,h,S+accepted_nodes[b,j],:], j = 0..accept_len[b], S = prefix_len[b]
+ *   prefix_len[b] += accept_len[b] + 1
+ * Source and destination rows overlap (with accepted_nodes = {0,2,3} row S+2
+ * is the source of slot 1 and the destination of slot 2), so every source row
+ * is read before any row is written: the result is the gather from the state
+ * before the call, whatever the order of the node ids.  Rows behind the
+ * accepted segment keep their (now stale) speculative contents; rows below S
+ * are never touched.
+ *
+ *   k_cache,v_cache   in/out [L,B,Hkv,Scap,d] with layer stride cache_layer_stride (elements)
+ *   accepted_nodes[B,Dp1], accept_len[B]  in (device)
+ *   prefix_len[B]     in/out
+ *   status[B]         in/out, as for kv_commit; TV_ST_CAPACITY also if a
+ *                     source row S + node lies at or past Scap.
+ * Limits: Dp1 * d / 8 <= 2048; d*2 bytes a multiple of 16; tensors 16-byte
+ * aligned; Hkv <= 32767.
+ */
+TV_API int kv_commit_inplace(tv_bf16* k_cache, tv_bf16* v_cache,
+              const int32_t* accepted_nodes, const int32_t* accept_len,
+              int32_t* prefix_len,
+              int L, int B, int Nmax, int Hkv, int d, int Scap, int Dp1,
+              int64_t cache_layer_stride,
               int32_t* status, tv_stream stream);
 
 /*

@@ -16,7 +16,7 @@ TV_ST_BAD_TREE, TV_ST_BAD_INDEX, TV_ST_CAPACITY, TV_ST_TIMEOUT, TV_ST_PATHS_TRUN
 
 EXPORTS = ["tv_last_error", "tv_version", "tv_launch_count", "tree_build_mask", "tv_attn_workspace_bytes", "tree_verify_attn",
            "tv_accept_workspace_bytes", "tree_accept", "tree_node_scores", "tree_merge_partials", "tv_accept_noalloc_max_bytes", "tree_accept_noalloc",
-           "kv_commit", "tv_step_staging_bytes",
+           "kv_commit", "kv_commit_inplace", "tv_step_staging_bytes",
            "tv_verify_step_host"]
 
 
@@ -75,6 +75,8 @@ def load():
     lib.tree_accept_noalloc.argtypes = [_c_vp] * 4 + [_c_int] * 5 + [_c_vp] * 7 + [_c_vp, _c_vp]
     lib.kv_commit.restype = _c_int
     lib.kv_commit.argtypes = [_c_vp] * 7 + [_c_int] * 7 + [_c_i64, _c_i64, _c_vp, _c_vp]
+    lib.kv_commit_inplace.restype = _c_int
+    lib.kv_commit_inplace.argtypes = [_c_vp] * 5 + [_c_int] * 7 + [_c_i64, _c_vp, _c_vp]
     lib.tv_step_staging_bytes.restype = _c_sz
     lib.tv_step_staging_bytes.argtypes = [_c_int] * 10
     lib.tv_verify_step_host.restype = _c_int
@@ -199,6 +201,16 @@ def kv_commit(k_cache, v_cache, k_tree, v_tree, accepted_nodes, accept_len, pref
     _check(load().kv_commit(_ptr(k_cache), _ptr(v_cache), _ptr(k_tree), _ptr(v_tree), _ptr(accepted_nodes),
                             _ptr(accept_len), _ptr(prefix_len), L, B, Nmax, Hkv, d, Scap, Dp1,
                             k_cache.stride(0), k_tree.stride(0), _ptr(status), _stream(stream)))
+
+
+def kv_commit_inplace(k_cache, v_cache, accepted_nodes, accept_len, prefix_len, Nmax, status, stream=None):
+    """In-cache layout: node i's K/V are rows prefix_len[b] + i of the cache; the accepted path is gathered to
+    the front of that region and prefix_len advances."""
+    L, B, Hkv, Scap, d = k_cache.shape
+    Dp1 = accepted_nodes.shape[1]
+    _check(load().kv_commit_inplace(_ptr(k_cache), _ptr(v_cache), _ptr(accepted_nodes), _ptr(accept_len),
+                                    _ptr(prefix_len), L, B, Nmax, Hkv, d, Scap, Dp1, k_cache.stride(0),
+                                    _ptr(status), _stream(stream)))
 
 
 def tv_verify_step_host(host, k_cache, v_cache, prefix_len, staging, scale, V, stream=None):

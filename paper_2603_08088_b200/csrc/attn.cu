@@ -308,6 +308,7 @@ struct AttnParams {
   int TT;                        // key tiles of the tree's own K/V: ceil(Nmax / 128), 1 or 2
   uint32_t q_box_bytes;
   unsigned long long* trace;     // optional event trace [cta][role 0..3][kTraceCap] of (tag << 48 | ns), or NULL          // bytes of one Q box {64, G, NPT}: 16 KB when G divides 128
+  int tree_in_cache;             // the tree's K/V rows live in the cache behind the prefix (rows S_b + node)
   int out_al32;                  // out is 32-byte aligned: rows can be written 32 bytes per thread and store
   float scale_log2e;             // scale * log2(e)
   float scale;
@@ -399,6 +400,9 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         int S = prm.prefix_len[b];
         S = S < 0 ? 0 : (S > prm.Scap ? prm.Scap : S);
         len = (S + kTileN - 1) / kTileN + prm.TT + kSetupCost;
+        // in-cache layout: a tree that does not fit behind its prefix is reported, not read past the capacity
+        // (rows past Scap arrive as zeros and the sequence's output is unspecified)
+        if (prm.tree_in_cache && blockIdx.x == 0 && S + prm.n_nodes[b] > prm.Scap) atomicOr(prm.status + b, TV_ST_CAPACITY);
       }
       int inc = len;
 #pragma unroll
@@ -557,7 +561,10 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               mbar_expect_tx(bar(L::KV_FULL + slot), L::kTileBytes);
 #pragma unroll
               for (int h = 0; h < D / 64; ++h) {
-                if (tree)
+                if (tree && prm.tree_in_cache)
+                  tma_load_3d_hint(dst + h * L::kHalf, kv ? &map_vc : &map_kc, bar(L::KV_FULL + slot), h * 64,
+                                   it.S + tt * kTileN, it.b * prm.Hkv + it.hk, kv_policy);
+                else if (tree)
                   tma_load_4d(dst + h * L::kHalf, kv ? &map_vt : &map_kt, bar(L::KV_FULL + slot), h * 64, it.hk, tt * kTileN, it.b);
                 else
                   tma_load_3d_hint(dst + h * L::kHalf, kv ? &map_vc : &map_kc, bar(L::KV_FULL + slot), h * 64, j * kTileN,
@@ -1419,9 +1426,14 @@ extern "C" int tree_verify_attn(const tv_bf16* q,
                                 tv_bf16* out, float* lse,
                                 void* workspace, size_t workspace_bytes,
                                 int32_t* status, tv_stream stream) {
-  TV_REQUIRE(q && k_cache && v_cache && k_tree && v_tree && prefix_len && n_nodes && anc_bits && out && status &&
-                 workspace,
+  TV_REQUIRE(q && k_cache && v_cache && prefix_len && n_nodes && anc_bits && out && status && workspace,
              "tree_verify_attn: NULL pointer");
+  TV_REQUIRE((k_tree == nullptr) == (v_tree == nullptr), "tree_verify_attn: k_tree and v_tree must both be given or both be NULL");
+  const bool in_cache = (k_tree == nullptr);       // the tree's K/V rows sit in the cache behind the prefix
+  if (in_cache) {
+    k_tree = k_cache;       // placeholders for the two descriptors the kernel then never uses
+    v_tree = v_cache;
+  }
   TV_REQUIRE(B >= 0 && B <= kMaxB, "tree_verify_attn: need 0 <= B <= 512");
   TV_REQUIRE(Nmax >= 1 && Nmax <= 256, "tree_verify_attn: Nmax must be in 1..256");
   TV_REQUIRE(d == 64 || d == 128, "tree_verify_attn: d must be 64 or 128");
@@ -1473,6 +1485,7 @@ extern "C" int tree_verify_attn(const tv_bf16* q,
   prm.G = g.G; prm.NPT = g.NPT; prm.NP = g.NP; prm.W = (Nmax + 31) / 32; prm.groups = g.groups;
   prm.TT = (Nmax + kTileN - 1) / kTileN;
   prm.scale = scale;
+  prm.tree_in_cache = in_cache ? 1 : 0;
   prm.out_al32 = (reinterpret_cast<uintptr_t>(out) & 31u) == 0 ? 1 : 0;
   prm.q_box_bytes = 64u * (uint32_t)g.G * (uint32_t)g.NPT * 2u;
   prm.trace = g_trace.load(std::memory_order_relaxed);

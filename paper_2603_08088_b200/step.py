@@ -40,12 +40,13 @@ class StepBuffers:
             self.candidates = torch.zeros(B, max(P, 1), Dp1, **i32) if want_gather else None
 
 
-def verify_step(case, buf: StepBuffers, scale, retrieve=None, commit=True, stream=None):
+def verify_step(case, buf: StepBuffers, scale, retrieve=None, commit=True, stream=None, in_cache=False):
     """Enqueue one whole step on ``stream`` (default: torch's current stream).
 
     ``case`` holds device tensors parent, n_nodes, tokens, prefix_len, q, k_tree, v_tree
     [L,...], k_cache, v_cache [L,...] and logits (optional).  ``retrieve`` overrides the
-    candidate rows; by default the rows tree_build_mask emits are used.
+    candidate rows; by default the rows tree_build_mask emits are used.  ``in_cache``: the tree's K/V are
+    rows prefix_len[b] + node of the caches (k_tree / v_tree are not read) and the commit reorders in place.
     """
     L, B, Nmax, Hq, Hkv, d, Scap, V, P, Dp1 = buf.dims
     own_rows = retrieve is None
@@ -54,8 +55,9 @@ def verify_step(case, buf: StepBuffers, scale, retrieve=None, commit=True, strea
                        retrieve_indices=buf.retrieve if own_rows else None,
                        n_paths=buf.n_paths, stream=stream)
     for l in range(L):
-        tv.tree_verify_attn(case["q"][l], case["k_cache"][l], case["v_cache"][l], case["k_tree"][l],
-                            case["v_tree"][l], case["prefix_len"], case["n_nodes"], buf.anc_bits, scale,
+        tv.tree_verify_attn(case["q"][l], case["k_cache"][l], case["v_cache"][l],
+                            None if in_cache else case["k_tree"][l], None if in_cache else case["v_tree"][l],
+                            case["prefix_len"], case["n_nodes"], buf.anc_bits, scale,
                             buf.out[l], buf.attn_ws, buf.status,
                             lse=None if buf.lse is None else buf.lse[l], stream=stream)
     if V > 0 and "logits" in case:
@@ -63,6 +65,9 @@ def verify_step(case, buf: StepBuffers, scale, retrieve=None, commit=True, strea
         tv.tree_accept(case["logits"], case["tokens"], rows, case["n_nodes"], buf.argmax_tok, buf.accept_len,
                        buf.best_path, buf.accepted_nodes, buf.next_token, buf.accept_ws, buf.status,
                        safe_idx=buf.safe_idx, candidates=buf.candidates, stream=stream)
-        if commit:
+        if commit and in_cache:
+            tv.kv_commit_inplace(case["k_cache"], case["v_cache"], buf.accepted_nodes, buf.accept_len,
+                                 case["prefix_len"], Nmax, buf.status, stream=stream)
+        elif commit:
             tv.kv_commit(case["k_cache"], case["v_cache"], case["k_tree"], case["v_tree"], buf.accepted_nodes,
                          buf.accept_len, case["prefix_len"], buf.status, stream=stream)
