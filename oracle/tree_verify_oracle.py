@@ -427,6 +427,61 @@ def kv_commit_inplace(k_cache, v_cache, accepted_nodes, accept_len, prefix_len, 
     return kc, vc, new_len, status
 
 
+# ---------------------------------------------------------------------------
+# Paged cache ("backend-specific layouts", Section 3.1): the same committed
+# rows, stored in pages of 128 rows named by a block table
+# ---------------------------------------------------------------------------
+PAGE_ROWS = 128
+
+
+def paged_to_contiguous(pages, block_table):
+    """pages [n_pages,Hkv,128,d], block_table [B,max_blocks] -> the cache as
+    [B,Hkv,128*max_blocks,d]: row s of sequence b is row s % 128 of page
+    block_table[b, s // 128].  Every table entry must name a page."""
+    n_pages = pages.shape[0]
+    bt = np.asarray(block_table)
+    assert ((0 <= bt) & (bt < n_pages)).all()
+    g = pages[bt]                                   # [B, max_blocks, Hkv, 128, d]
+    B, nb, Hkv, R, d = g.shape
+    return g.transpose(0, 2, 1, 3, 4).reshape(B, Hkv, nb * R, d)
+
+
+def kv_commit_paged(k_pages, v_pages, block_table, k_tree, v_tree, accepted_nodes, accept_len, prefix_len,
+                    status_in=None):
+    """kv_commit on a paged cache: row S_b + j of sequence b lives in page
+    block_table[b, (S_b+j) // 128] at row (S_b+j) % 128.  pages are
+    [L,n_pages,Hkv,128,d]; works on copies.  The capacity is 128 * max_blocks;
+    a page id outside [0, n_pages) under the accepted segment is an index
+    error and skips the sequence."""
+    kp, vp = k_pages.copy(), v_pages.copy()
+    L, n_pages, Hkv, R, d = kp.shape
+    B, max_blocks = block_table.shape
+    Nmax = k_tree.shape[2]
+    Dp1 = accepted_nodes.shape[1]
+    new_len = np.array(prefix_len, dtype=np.int32).copy()
+    status = np.zeros(B, dtype=np.int32) if status_in is None else np.array(status_in, dtype=np.int32).copy()
+    for b in range(B):
+        if status[b] & ST_FATAL:
+            continue
+        S, A = int(prefix_len[b]), int(accept_len[b])
+        if A < 0 or A >= Dp1 or any(not (0 <= int(accepted_nodes[b, j]) < Nmax) for j in range(A + 1)):
+            status[b] |= ST_BAD_INDEX
+            continue
+        if S < 0 or S + A + 1 > R * max_blocks:
+            status[b] |= ST_CAPACITY
+            continue
+        if any(not (0 <= int(block_table[b, t]) < n_pages) for t in range(S // R, (S + A) // R + 1)):
+            status[b] |= ST_BAD_INDEX
+            continue
+        for j in range(A + 1):
+            row, node = S + j, int(accepted_nodes[b, j])
+            pg = int(block_table[b, row // R])
+            kp[:, pg, :, row % R, :] = k_tree[:, b, node, :, :]
+            vp[:, pg, :, row % R, :] = v_tree[:, b, node, :, :]
+        new_len[b] = S + A + 1
+    return kp, vp, new_len, status
+
+
 def verify_step(case_np, scale, Dcap=None, Pcap=None, use_given_retrieve=True):
     """One whole step in the paper's order: tensorise + mask, attention per
     layer, safe gather + argmax + accept, commit (Section 3 call order)."""

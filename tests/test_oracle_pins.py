@@ -544,6 +544,41 @@ def test_inplace_commit_equals_separate_buffer_commit_and_flags():
     assert (k4[:, :2] == kin[:, :2]).all()
 
 
+def test_paged_cache_is_the_contiguous_cache_behind_a_block_table():
+    """Layout pins: a hand-typed two-page example of the row mapping, and the paged commit equal to the
+    contiguous commit seen through the block table (sequences own disjoint pages; a segment that crosses a
+    page boundary; untouched pages stay untouched; bad page id, capacity)."""
+    pages = np.zeros((3, 1, orc.PAGE_ROWS, 1), dtype=np.uint16)
+    for pg in range(3):
+        pages[pg, 0, :, 0] = 1000 * pg + np.arange(orc.PAGE_ROWS)
+    bt = np.array([[2, 0]], dtype=np.int32)
+    flat = orc.paged_to_contiguous(pages, bt)
+    assert flat.shape == (1, 1, 256, 1)
+    assert flat[0, 0, [0, 5, 127, 128, 130, 255], 0].tolist() == [2000, 2005, 2127, 0, 2, 127]
+
+    rng = np.random.default_rng(16)
+    L, B, Hkv, d, N, Dp1, n_pages, nb = 2, 3, 2, 4, 9, 4, 10, 3
+    u16 = lambda *s_: rng.integers(0, 2 ** 16, size=s_).astype(np.uint16)
+    kp, vp = u16(L, n_pages, Hkv, orc.PAGE_ROWS, d), u16(L, n_pages, Hkv, orc.PAGE_ROWS, d)
+    kt, vt = u16(L, B, N, Hkv, d), u16(L, B, N, Hkv, d)
+    bt = np.array([[7, 2, 9], [0, 5, 1], [3, 8, 4]], dtype=np.int32)      # page 6 belongs to nobody
+    nodes = np.array([[0, 2, 5, 8], [0, 1, 0, 0], [0, 3, 4, 0]], dtype=np.int32)
+    A = np.array([3, 1, 2], dtype=np.int32)
+    S = np.array([126, 0, 381], dtype=np.int32)          # b=0 crosses pages 7 -> 2; b=2 ends exactly at the capacity 384
+    kp2, vp2, S2, st = orc.kv_commit_paged(kp, vp, bt, kt, vt, nodes, A, S)
+    assert st.tolist() == [0, 0, 0] and S2.tolist() == [130, 2, 384]
+    cont = lambda pgs: np.stack([orc.paged_to_contiguous(pgs[l], bt) for l in range(L)])
+    rk, rv, rS, rst = orc.kv_commit(cont(kp), cont(vp), kt, vt, nodes, A, S)
+    assert (cont(kp2) == rk).all() and (cont(vp2) == rv).all() and rS.tolist() == S2.tolist()
+    assert (kp2[:, 6] == kp[:, 6]).all() and (vp2[:, 6] == vp[:, 6]).all()
+    assert (kp2[:, 7, :, 126] == kt[:, 0, 0]).all() and (kp2[:, 2, :, 1] == kt[:, 0, 8]).all()
+    bad_bt = bt.copy()
+    bad_bt[0, 1] = n_pages                                # the page the segment of b=0 runs into
+    kp3, _, S3, st3 = orc.kv_commit_paged(kp, vp, bad_bt, kt, vt, nodes, A, np.array([126, 0, 382], dtype=np.int32))
+    assert st3.tolist() == [orc.ST_BAD_INDEX, 0, orc.ST_CAPACITY] and S3.tolist() == [126, 2, 382]
+    assert (kp3[:, 7] == kp[:, 7]).all()
+
+
 def test_node_scores_gather_and_link_to_greedy_acceptance():
     """score[k] = logits[parent(k), token(k)]: checked against numpy fancy indexing, and against the
     acceptance rule - a node is accepted by the greedy rule exactly when its score equals the row
