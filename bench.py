@@ -347,6 +347,9 @@ def run_ours(args, cfg):
     if args.in_cache and has_accept:
         line["in_cache"] = in_cache_step(cfg, case, buf, prefix0, scale, given_rows, min(args.steps, 20), dev)
         case["prefix_len"].copy_(prefix0)
+    if args.paged and has_accept:
+        line["paged"] = paged_step(cfg, case, buf, prefix0, scale, given_rows, min(args.steps, 20), dev, args.seed)
+        case["prefix_len"].copy_(prefix0)
     if args.context_split > 1:
         case["prefix_len"].copy_(prefix0)
         line["context_split"] = context_split_member(cfg, case, buf, args.context_split, dev)
@@ -453,6 +456,61 @@ def in_cache_step(cfg, case, buf, prefix0, scale, given_rows, steps, dev):
             "note": "tree K/V read from the cache rows behind the prefix; commit = reorder inside the cache"}
 
 
+def paged_step(cfg, case, buf, prefix0, scale, given_rows, steps, dev, seed):
+    """The same step over a paged committed cache: every sequence's rows cut into pages of 128 rows that are
+    scattered over a pool in a seeded random order (one block table for all layers), then mask, L x
+    tree_verify_attn_paged, accept and kv_commit_paged are timed.  The pool is built once, outside the timed
+    region; every step starts from the same prefix lengths (the commit rewrites the same rows)."""
+    import paper_2603_08088_b200 as tv
+    L, B, Hkv, Scap, d = case["k_cache"].shape
+    nb = (Scap + 127) // 128
+    n_pages = B * nb
+    g = torch.Generator().manual_seed(seed)
+    order = torch.randperm(n_pages, generator=g).to(dev)
+    bt = order.view(B, nb).to(torch.int32).contiguous()
+    def paginate(cache):
+        pool = torch.zeros(L, n_pages, Hkv, 128, d, dtype=cache.dtype, device=dev)
+        for b in range(B):
+            rows = torch.zeros(L, Hkv, nb * 128, d, dtype=cache.dtype, device=dev)
+            rows[:, :, :Scap] = cache[:, b]
+            pool[:, bt[b].long()] = rows.view(L, Hkv, nb, 128, d).permute(0, 2, 1, 3, 4)
+        return pool
+    k_pages, v_pages = paginate(case["k_cache"]), paginate(case["v_cache"])
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    t_step, t_attn, t_commit = [], [], []
+    for it in range(3 + steps):
+        case["prefix_len"].copy_(prefix0)
+        m = [ev() for _ in range(5)]
+        m[0].record()
+        tv.tree_build_mask(case["parent"], case["n_nodes"], cfg.D, buf.retrieve.shape[1], buf.anc_bits, buf.status,
+                           retrieve_indices=None if given_rows else buf.retrieve, n_paths=buf.n_paths)
+        m[1].record()
+        for l in range(L):
+            tv.tree_verify_attn_paged(case["q"][l], k_pages[l], v_pages[l], bt, case["k_tree"][l], case["v_tree"][l],
+                                      case["prefix_len"], case["n_nodes"], buf.anc_bits, scale, buf.out[l], buf.attn_ws,
+                                      buf.status)
+        m[2].record()
+        tv.tree_accept(case["logits"], case["tokens"], case["retrieve"] if given_rows else buf.retrieve, case["n_nodes"],
+                       buf.argmax_tok, buf.accept_len, buf.best_path, buf.accepted_nodes, buf.next_token, buf.accept_ws,
+                       buf.status)
+        m[3].record()
+        tv.kv_commit_paged(k_pages, v_pages, bt, case["k_tree"], case["v_tree"], buf.accepted_nodes, buf.accept_len,
+                           case["prefix_len"], buf.status)
+        m[4].record()
+        torch.cuda.synchronize()
+        if it >= 3:
+            t_step.append(m[0].elapsed_time(m[4]))
+            t_attn.append(m[1].elapsed_time(m[2]) / L)
+            t_commit.append(m[3].elapsed_time(m[4]))
+    if (buf.status.cpu().numpy() & 15).any():
+        raise SystemExit(f"bench.py: fatal status in the paged step: {buf.status.cpu().numpy()}")
+    med = lambda v: sorted(v)[len(v) // 2]
+    return {"steps": steps, "page_rows": 128, "n_pages": n_pages, "ms_per_step_median": med(t_step),
+            "steps_per_sec": 1e3 / med(t_step), "attn_per_layer_us": med(t_attn) * 1e3,
+            "commit_paged_us": med(t_commit) * 1e3,
+            "note": "committed cache in pages of 128 rows scattered over the pool, one block table for all layers"}
+
+
 def context_split_member(cfg, case, buf, R, dev):
     """What one member of an R-way context split of this workload does per layer, timed on this GPU: attention
     over its 1/R of every prefix (it owns the tree keys, the worst case) and the merge of R gathered partials.
@@ -509,6 +567,8 @@ def main():
                     help="also time tree_verify_attn over the node budgets of the paper's sweep (extra key in the JSON line)")
     ap.add_argument("--in-cache", action="store_true",
                     help="also time the step with the tree's K/V inside the cache and the in-place commit")
+    ap.add_argument("--paged", action="store_true",
+                    help="also time the step over a paged committed cache (pages of 128 rows, block table)")
     ap.add_argument("--context-split", type=int, default=1,
                     help="also time one member of an R-way context split of the workload (extra key in the JSON line)")
     args = ap.parse_args()

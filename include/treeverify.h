@@ -157,6 +157,33 @@ TV_API int tree_verify_attn(const tv_bf16* q,
                      void* workspace, size_t workspace_bytes,
                      int32_t* status, tv_stream stream);
 
+/*
+ * tree_verify_attn over a paged committed cache (Section 3.1 speaks of
+ * backend-specific KV layouts behind one cache interface; this is the block
+ * layout of serving stacks).  A page holds 128 consecutive rows - one key tile
+ * of the kernel - of all KV heads: k_pages, v_pages [n_pages,Hkv,128,d] bf16
+ * (one layer).  block_table[B,max_blocks] names, for sequence b, the page of
+ * rows 128 t .. 128 t + 127 at [b, t]; only entries t < ceil(prefix_len[b]/128)
+ * are read.  The capacity of a sequence is 128 * max_blocks rows.  The tree's
+ * K/V come in their own buffers.  Everything else - arguments, outputs,
+ * workspace (tv_attn_workspace_bytes with any Scap), limits, stream order - is
+ * as for tree_verify_attn; the block table is read like prefix_len, before
+ * earlier kernels of the stream have finished, so it must not be written by a
+ * tree_verify_attn call in front.  A page id outside [0, n_pages) raises
+ * TV_ST_BAD_INDEX for the sequence (its output is unspecified; nothing is
+ * read outside the pool).
+ */
+TV_API int tree_verify_attn_paged(const tv_bf16* q,
+                     const tv_bf16* k_pages, const tv_bf16* v_pages,
+                     const int32_t* block_table,
+                     const tv_bf16* k_tree, const tv_bf16* v_tree,
+                     const int32_t* prefix_len, const int32_t* n_nodes,
+                     const uint32_t* anc_bits,
+                     int B, int Nmax, int Hq, int Hkv, int d, int n_pages, int max_blocks, float scale,
+                     tv_bf16* out, float* lse,
+                     void* workspace, size_t workspace_bytes,
+                     int32_t* status, tv_stream stream);
+
 /* Scratch needed by tree_accept (bytes). */
 TV_API size_t tv_accept_workspace_bytes(int B, int Nmax, int V);
 
@@ -284,6 +311,27 @@ TV_API int kv_commit(tv_bf16* k_cache, tv_bf16* v_cache,
               int32_t* prefix_len,
               int L, int B, int Nmax, int Hkv, int d, int Scap, int Dp1,
               int64_t cache_layer_stride, int64_t tree_layer_stride,
+              int32_t* status, tv_stream stream);
+
+/*
+ * kv_commit on the paged cache of tree_verify_attn_paged: accepted row j of
+ * sequence b goes to row (S+j) % 128 of page block_table[b, (S+j) / 128],
+ * S = prefix_len[b], for all layers; prefix_len[b] += accept_len[b] + 1.  The
+ * pages under the accepted segment must already be in the block table (the
+ * caller allocates pages; the library never does).
+ *   k_pages,v_pages   in/out [L,n_pages,Hkv,128,d] with layer stride page_layer_stride (elements)
+ *   k_tree,v_tree     in     [L,B,Nmax,Hkv,d] with layer stride tree_layer_stride
+ *   status[B]         in/out as for kv_commit; capacity = 128 * max_blocks;
+ *                     TV_ST_BAD_INDEX also for a page id outside [0, n_pages)
+ *                     under the segment.  A flagged sequence is left untouched.
+ * Limits as for kv_commit; max_blocks <= 2^20.
+ */
+TV_API int kv_commit_paged(tv_bf16* k_pages, tv_bf16* v_pages, const int32_t* block_table,
+              const tv_bf16* k_tree, const tv_bf16* v_tree,
+              const int32_t* accepted_nodes, const int32_t* accept_len,
+              int32_t* prefix_len,
+              int L, int B, int Nmax, int Hkv, int d, int n_pages, int max_blocks, int Dp1,
+              int64_t page_layer_stride, int64_t tree_layer_stride,
               int32_t* status, tv_stream stream);
 
 /*

@@ -16,7 +16,7 @@ TV_ST_BAD_TREE, TV_ST_BAD_INDEX, TV_ST_CAPACITY, TV_ST_TIMEOUT, TV_ST_PATHS_TRUN
 
 EXPORTS = ["tv_last_error", "tv_version", "tv_launch_count", "tree_build_mask", "tv_attn_workspace_bytes", "tree_verify_attn",
            "tv_accept_workspace_bytes", "tree_accept", "tree_node_scores", "tree_merge_partials", "tv_accept_noalloc_max_bytes", "tree_accept_noalloc",
-           "kv_commit", "kv_commit_inplace", "tv_step_staging_bytes",
+           "kv_commit", "kv_commit_inplace", "tree_verify_attn_paged", "kv_commit_paged", "tv_step_staging_bytes",
            "tv_verify_step_host"]
 
 
@@ -75,6 +75,10 @@ def load():
     lib.tree_accept_noalloc.argtypes = [_c_vp] * 4 + [_c_int] * 5 + [_c_vp] * 7 + [_c_vp, _c_vp]
     lib.kv_commit.restype = _c_int
     lib.kv_commit.argtypes = [_c_vp] * 7 + [_c_int] * 7 + [_c_i64, _c_i64, _c_vp, _c_vp]
+    lib.tree_verify_attn_paged.restype = _c_int
+    lib.tree_verify_attn_paged.argtypes = [_c_vp] * 9 + [_c_int] * 7 + [_c_f, _c_vp, _c_vp, _c_vp, _c_sz, _c_vp, _c_vp]
+    lib.kv_commit_paged.restype = _c_int
+    lib.kv_commit_paged.argtypes = [_c_vp] * 8 + [_c_int] * 8 + [_c_i64, _c_i64, _c_vp, _c_vp]
     lib.kv_commit_inplace.restype = _c_int
     lib.kv_commit_inplace.argtypes = [_c_vp] * 5 + [_c_int] * 7 + [_c_i64, _c_vp, _c_vp]
     lib.tv_step_staging_bytes.restype = _c_sz
@@ -201,6 +205,30 @@ def kv_commit(k_cache, v_cache, k_tree, v_tree, accepted_nodes, accept_len, pref
     _check(load().kv_commit(_ptr(k_cache), _ptr(v_cache), _ptr(k_tree), _ptr(v_tree), _ptr(accepted_nodes),
                             _ptr(accept_len), _ptr(prefix_len), L, B, Nmax, Hkv, d, Scap, Dp1,
                             k_cache.stride(0), k_tree.stride(0), _ptr(status), _stream(stream)))
+
+
+def tree_verify_attn_paged(q, k_pages, v_pages, block_table, k_tree, v_tree, prefix_len, n_nodes, anc_bits, scale, out,
+                           workspace, status, lse=None, stream=None):
+    """k_pages, v_pages [n_pages,Hkv,128,d] (one layer), block_table [B,max_blocks] int32."""
+    B, Nmax, Hq, d = q.shape
+    n_pages, Hkv = k_pages.shape[0], k_pages.shape[1]
+    assert k_pages.shape[2] == 128 and block_table.shape[0] == B
+    _check(load().tree_verify_attn_paged(_ptr(q), _ptr(k_pages), _ptr(v_pages), _ptr(block_table), _ptr(k_tree),
+                                         _ptr(v_tree), _ptr(prefix_len), _ptr(n_nodes), _ptr(anc_bits), B, Nmax, Hq,
+                                         Hkv, d, n_pages, block_table.shape[1], float(scale), _ptr(out), _ptr(lse),
+                                         _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                         _ptr(status), _stream(stream)))
+
+
+def kv_commit_paged(k_pages, v_pages, block_table, k_tree, v_tree, accepted_nodes, accept_len, prefix_len, status,
+                    stream=None):
+    """k_pages, v_pages [L,n_pages,Hkv,128,d]."""
+    L, n_pages, Hkv, _, d = k_pages.shape
+    B, Nmax = k_tree.shape[1], k_tree.shape[2]
+    _check(load().kv_commit_paged(_ptr(k_pages), _ptr(v_pages), _ptr(block_table), _ptr(k_tree), _ptr(v_tree),
+                                  _ptr(accepted_nodes), _ptr(accept_len), _ptr(prefix_len), L, B, Nmax, Hkv, d,
+                                  n_pages, block_table.shape[1], accepted_nodes.shape[1], k_pages.stride(0),
+                                  k_tree.stride(0), _ptr(status), _stream(stream)))
 
 
 def kv_commit_inplace(k_cache, v_cache, accepted_nodes, accept_len, prefix_len, Nmax, status, stream=None):

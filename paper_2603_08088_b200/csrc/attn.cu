@@ -309,6 +309,8 @@ struct AttnParams {
   uint32_t q_box_bytes;
   unsigned long long* trace;     // optional event trace [cta][role 0..3][kTraceCap] of (tag << 48 | ns), or NULL          // bytes of one Q box {64, G, NPT}: 16 KB when G divides 128
   int tree_in_cache;             // the tree's K/V rows live in the cache behind the prefix (rows S_b + node)
+  const int32_t* block_table;    // paged cache: page of key tile j of sequence b at [b * max_blocks + j]; else nullptr
+  int max_blocks, n_pages;
   int out_al32;                  // out is 32-byte aligned: rows can be written 32 bytes per thread and store
   float scale_log2e;             // scale * log2(e)
   float scale;
@@ -542,9 +544,24 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         bool q_pending = !synced;          // first item: Q goes out after the first prefix tiles
         if (!q_pending) load_q();
         ++item_idx;
+        // paged cache: the page of a prefix key tile comes from the block table, fetched one tile ahead of its use
+        auto page_of = [&](int jj) -> int {
+          if (!prm.block_table || jj >= it.len - prm.TT || jj >= it.j1) return 0;
+          int pg = prm.block_table[(size_t)it.b * prm.max_blocks + jj];
+          if ((unsigned)pg >= (unsigned)prm.n_pages) {       // reported; the tile then reads page 0
+            if (lane == 0) atomicOr(prm.status + it.b, TV_ST_BAD_INDEX);
+            pg = 0;
+          }
+          return pg;
+        };
+        int page_next = page_of(it.j0);
         for (int j = it.j0; j < it.j1 && ok; ++j) {
           const int tt = j - (it.len - prm.TT);      // >= 0: index of the tree key tile
           const bool tree = tt >= 0;
+          const int page = page_next;
+          page_next = page_of(j + 1);
+          const int row0 = prm.block_table ? 0 : j * kTileN;                                // of the tile in its slab
+          const int slab = (prm.block_table ? page : it.b) * prm.Hkv + it.hk;               // (page or sequence, KV head)
 #pragma unroll
           for (int kv = 0; kv < 2; ++kv) {
             const uint32_t slot = fill % kSlots, round = fill / kSlots;
@@ -567,8 +584,8 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 else if (tree)
                   tma_load_4d(dst + h * L::kHalf, kv ? &map_vt : &map_kt, bar(L::KV_FULL + slot), h * 64, it.hk, tt * kTileN, it.b);
                 else
-                  tma_load_3d_hint(dst + h * L::kHalf, kv ? &map_vc : &map_kc, bar(L::KV_FULL + slot), h * 64, j * kTileN,
-                                   it.b * prm.Hkv + it.hk, kv_policy);
+                  tma_load_3d_hint(dst + h * L::kHalf, kv ? &map_vc : &map_kc, bar(L::KV_FULL + slot), h * 64, row0, slab,
+                                   kv_policy);
               }
             }
             __syncwarp();
@@ -1417,15 +1434,18 @@ extern "C" size_t tv_attn_workspace_bytes(int B, int Nmax, int Hq, int Hkv, int 
   return geometry(B, Nmax, Hq, Hkv, d, false).total;
 }
 
-extern "C" int tree_verify_attn(const tv_bf16* q,
-                                const tv_bf16* k_cache, const tv_bf16* v_cache,
-                                const tv_bf16* k_tree, const tv_bf16* v_tree,
-                                const int32_t* prefix_len, const int32_t* n_nodes,
-                                const uint32_t* anc_bits,
-                                int B, int Nmax, int Hq, int Hkv, int d, int Scap, float scale,
-                                tv_bf16* out, float* lse,
-                                void* workspace, size_t workspace_bytes,
-                                int32_t* status, tv_stream stream) {
+// Both layouts of the committed cache: contiguous [B,Hkv,Scap,d] (block_table == nullptr) or pages
+// [n_pages,Hkv,128,d] named by block_table[B,max_blocks] (then Scap = 128 * max_blocks).
+static int attn_entry(const tv_bf16* q,
+                      const tv_bf16* k_cache, const tv_bf16* v_cache,
+                      const int32_t* block_table, int n_pages, int max_blocks,
+                      const tv_bf16* k_tree, const tv_bf16* v_tree,
+                      const int32_t* prefix_len, const int32_t* n_nodes,
+                      const uint32_t* anc_bits,
+                      int B, int Nmax, int Hq, int Hkv, int d, int Scap, float scale,
+                      tv_bf16* out, float* lse,
+                      void* workspace, size_t workspace_bytes,
+                      int32_t* status, tv_stream stream) {
   TV_REQUIRE(q && k_cache && v_cache && prefix_len && n_nodes && anc_bits && out && status && workspace,
              "tree_verify_attn: NULL pointer");
   TV_REQUIRE((k_tree == nullptr) == (v_tree == nullptr), "tree_verify_attn: k_tree and v_tree must both be given or both be NULL");
@@ -1457,8 +1477,11 @@ extern "C" int tree_verify_attn(const tv_bf16* q,
     cuuint64_t qd[4] = {(cuuint64_t)d, (cuuint64_t)Hq, (cuuint64_t)Nmax, (cuuint64_t)B};
     cuuint64_t qs[3] = {(cuuint64_t)d * e, (cuuint64_t)Hq * d * e, (cuuint64_t)Nmax * Hq * d * e};
     cuuint32_t qb[4] = {64, (cuuint32_t)g.G, (cuuint32_t)g.NPT, 1};
-    cuuint64_t cd[3] = {(cuuint64_t)d, (cuuint64_t)Scap, (cuuint64_t)B * Hkv};
-    cuuint64_t cs[2] = {(cuuint64_t)d * e, (cuuint64_t)Scap * d * e};
+    // rows of one (sequence, KV head) slab, or of one (page, KV head) slab of 128 rows
+    const cuuint64_t slab_rows = block_table ? (cuuint64_t)kTileN : (cuuint64_t)Scap;
+    const cuuint64_t slabs = block_table ? (cuuint64_t)n_pages * Hkv : (cuuint64_t)B * Hkv;
+    cuuint64_t cd[3] = {(cuuint64_t)d, slab_rows, slabs};
+    cuuint64_t cs[2] = {(cuuint64_t)d * e, slab_rows * d * e};
     cuuint32_t cb[3] = {64, kTileN, 1};
     cuuint64_t td[4] = {(cuuint64_t)d, (cuuint64_t)Hkv, (cuuint64_t)Nmax, (cuuint64_t)B};
     cuuint64_t ts[3] = {(cuuint64_t)d * e, (cuuint64_t)Hkv * d * e, (cuuint64_t)Nmax * Hkv * d * e};
@@ -1486,6 +1509,9 @@ extern "C" int tree_verify_attn(const tv_bf16* q,
   prm.TT = (Nmax + kTileN - 1) / kTileN;
   prm.scale = scale;
   prm.tree_in_cache = in_cache ? 1 : 0;
+  prm.block_table = block_table;
+  prm.max_blocks = max_blocks;
+  prm.n_pages = n_pages;
   prm.out_al32 = (reinterpret_cast<uintptr_t>(out) & 31u) == 0 ? 1 : 0;
   prm.q_box_bytes = 64u * (uint32_t)g.G * (uint32_t)g.NPT * 2u;
   prm.trace = g_trace.load(std::memory_order_relaxed);
@@ -1497,4 +1523,34 @@ extern "C" int tree_verify_attn(const tv_bf16* q,
   if (e != cudaSuccess) return tv::fail(TV_ERR_CUDA, "tree_verify_attn: launch failed: %s", cudaGetErrorString(e));
   tv::count_launches(1);
   return TV_OK;
+}
+
+extern "C" int tree_verify_attn(const tv_bf16* q,
+                                const tv_bf16* k_cache, const tv_bf16* v_cache,
+                                const tv_bf16* k_tree, const tv_bf16* v_tree,
+                                const int32_t* prefix_len, const int32_t* n_nodes,
+                                const uint32_t* anc_bits,
+                                int B, int Nmax, int Hq, int Hkv, int d, int Scap, float scale,
+                                tv_bf16* out, float* lse,
+                                void* workspace, size_t workspace_bytes,
+                                int32_t* status, tv_stream stream) {
+  return attn_entry(q, k_cache, v_cache, nullptr, 0, 0, k_tree, v_tree, prefix_len, n_nodes, anc_bits, B, Nmax, Hq, Hkv,
+                    d, Scap, scale, out, lse, workspace, workspace_bytes, status, stream);
+}
+
+extern "C" int tree_verify_attn_paged(const tv_bf16* q,
+                                      const tv_bf16* k_pages, const tv_bf16* v_pages,
+                                      const int32_t* block_table,
+                                      const tv_bf16* k_tree, const tv_bf16* v_tree,
+                                      const int32_t* prefix_len, const int32_t* n_nodes,
+                                      const uint32_t* anc_bits,
+                                      int B, int Nmax, int Hq, int Hkv, int d, int n_pages, int max_blocks, float scale,
+                                      tv_bf16* out, float* lse,
+                                      void* workspace, size_t workspace_bytes,
+                                      int32_t* status, tv_stream stream) {
+  TV_REQUIRE(block_table && k_tree && v_tree, "tree_verify_attn_paged: NULL pointer");
+  TV_REQUIRE(n_pages >= 1 && max_blocks >= 1 && max_blocks <= (1 << 20) && (long long)n_pages * Hkv < (1ll << 31),
+             "tree_verify_attn_paged: need n_pages >= 1, 1 <= max_blocks <= 2^20, n_pages * Hkv < 2^31");
+  return attn_entry(q, k_pages, v_pages, block_table, n_pages, max_blocks, k_tree, v_tree, prefix_len, n_nodes, anc_bits,
+                    B, Nmax, Hq, Hkv, d, max_blocks * kTileN, scale, out, lse, workspace, workspace_bytes, status, stream);
 }

@@ -150,7 +150,102 @@ __global__ void commit_inplace_finish_kernel(const int32_t* __restrict__ accepte
   else if (r > 0) status[b] |= r;
 }
 
+// Paged cache: pages [n_pages,Hkv,128,d] per layer, block_table[b, t] = page of rows 128 t .. 128 t + 127 of
+// sequence b.  Row S + j of the sequence is row (S + j) % 128 of page block_table[b, (S + j) / 128].
+constexpr int kPageRows = 128;
+
+__device__ __forceinline__ bool paged_segment_ok(const int32_t* block_table, int b, int S, int A, int max_blocks,
+                                                 int n_pages) {
+  for (int t = S / kPageRows; t <= (S + A) / kPageRows; ++t) {
+    const int pg = block_table[(size_t)b * max_blocks + t];
+    if (pg < 0 || pg >= n_pages) return false;
+  }
+  return true;
+}
+
+__global__ void __launch_bounds__(kCopyThreads)
+commit_paged_kernel(uint4* __restrict__ k_pages, uint4* __restrict__ v_pages, const int32_t* __restrict__ block_table,
+                    const uint4* __restrict__ k_tree, const uint4* __restrict__ v_tree,
+                    const int32_t* __restrict__ accepted_nodes, const int32_t* __restrict__ accept_len,
+                    const int32_t* __restrict__ prefix_len, const int32_t* __restrict__ status,
+                    int B, int Nmax, int Hkv, int dvec, int n_pages, int max_blocks, int Dp1,
+                    int64_t page_layer_vec, int64_t tree_layer_vec) {
+  __shared__ int s_nodes[kCopyMaxDp1];
+  const int b = blockIdx.x, l = blockIdx.y;
+  const int A = accept_len[b];
+  const int S = prefix_len[b];
+  const int st = status[b];
+  for (int j = threadIdx.x; j < Dp1; j += kCopyThreads) s_nodes[j] = accepted_nodes[(size_t)b * Dp1 + j];
+  int bad = (st & tv::kFatalStatus) || A < 0 || A >= Dp1 || S < 0 || S + A + 1 > max_blocks * kPageRows;
+  __syncthreads();
+  if (!bad) {
+    for (int j = threadIdx.x; j <= A; j += kCopyThreads) bad |= (s_nodes[j] < 0 || s_nodes[j] >= Nmax);
+    if (threadIdx.x == 0) bad |= !paged_segment_ok(block_table, b, S, A, max_blocks, n_pages);
+  }
+  if (__syncthreads_or(bad)) return;
+  const size_t src0 = (size_t)l * tree_layer_vec + (size_t)b * Nmax * Hkv * dvec;       // [node, h, :]
+  const size_t dst0 = (size_t)l * page_layer_vec;                                       // [page, h, row, :]
+  const int per = Hkv * dvec;
+  const int total = 2 * (A + 1) * per;
+  for (int t = threadIdx.x; t < total; t += kCopyThreads) {
+    const int kv = t >= (A + 1) * per;
+    const int u = kv ? t - (A + 1) * per : t;
+    const int j = u / per, w = u - j * per;
+    const int h = w / dvec, c = w - h * dvec;
+    const int row = S + j;
+    const int pg = block_table[(size_t)b * max_blocks + row / kPageRows];
+    const uint4 val = (kv ? v_tree : k_tree)[src0 + (size_t)s_nodes[j] * per + w];
+    (kv ? v_pages : k_pages)[dst0 + (((size_t)pg * Hkv + h) * kPageRows + row % kPageRows) * dvec + c] = val;
+  }
+}
+
+__global__ void commit_paged_finish_kernel(const int32_t* __restrict__ accepted_nodes,
+                                           const int32_t* __restrict__ accept_len,
+                                           const int32_t* __restrict__ block_table,
+                                           int32_t* __restrict__ prefix_len, int32_t* __restrict__ status,
+                                           int B, int Nmax, int n_pages, int max_blocks, int Dp1) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= B) return;
+  const int A = accept_len[b];
+  const int S = prefix_len[b];
+  int r = commit_check(accepted_nodes, A, S, status[b], Nmax, max_blocks * kPageRows, Dp1, b);
+  if (r == 0 && !paged_segment_ok(block_table, b, S, A, max_blocks, n_pages)) r = TV_ST_BAD_INDEX;
+  if (r == 0) prefix_len[b] = S + A + 1;
+  else if (r > 0) status[b] |= r;
+}
+
 }  // namespace
+
+extern "C" int kv_commit_paged(tv_bf16* k_pages, tv_bf16* v_pages, const int32_t* block_table,
+                               const tv_bf16* k_tree, const tv_bf16* v_tree,
+                               const int32_t* accepted_nodes, const int32_t* accept_len,
+                               int32_t* prefix_len,
+                               int L, int B, int Nmax, int Hkv, int d, int n_pages, int max_blocks, int Dp1,
+                               int64_t page_layer_stride, int64_t tree_layer_stride,
+                               int32_t* status, tv_stream stream) {
+  TV_REQUIRE(k_pages && v_pages && block_table && k_tree && v_tree && accepted_nodes && accept_len && prefix_len && status,
+             "kv_commit_paged: NULL pointer");
+  TV_REQUIRE(L >= 0 && B >= 0 && Nmax >= 1 && Hkv >= 1 && d >= 8 && n_pages >= 1 && max_blocks >= 1 && Dp1 >= 1,
+             "kv_commit_paged: bad dimension");
+  TV_REQUIRE(max_blocks <= (1 << 20), "kv_commit_paged: max_blocks must be <= 2^20");
+  TV_REQUIRE(d % 8 == 0, "kv_commit_paged: d must be a multiple of 8 (16-byte rows)");
+  TV_REQUIRE(page_layer_stride % 8 == 0 && tree_layer_stride % 8 == 0, "kv_commit_paged: layer strides must be multiples of 8 elements");
+  TV_REQUIRE(tv::aligned16(k_pages) && tv::aligned16(v_pages) && tv::aligned16(k_tree) && tv::aligned16(v_tree),
+             "kv_commit_paged: tensors must be 16-byte aligned");
+  TV_REQUIRE(L <= 65535 && Dp1 <= kCopyMaxDp1, "kv_commit_paged: L must be <= 65535 and Dp1 <= 1024");
+  if (L == 0 || B == 0) return TV_OK;
+  cudaStream_t s = (cudaStream_t)stream;
+  commit_paged_kernel<<<dim3(B, L), kCopyThreads, 0, s>>>(
+      reinterpret_cast<uint4*>(k_pages), reinterpret_cast<uint4*>(v_pages), block_table,
+      reinterpret_cast<const uint4*>(k_tree), reinterpret_cast<const uint4*>(v_tree), accepted_nodes, accept_len,
+      prefix_len, status, B, Nmax, Hkv, d / 8, n_pages, max_blocks, Dp1, page_layer_stride / 8, tree_layer_stride / 8);
+  TV_CUDA_OK(cudaGetLastError());
+  commit_paged_finish_kernel<<<(B + 127) / 128, 128, 0, s>>>(accepted_nodes, accept_len, block_table, prefix_len, status,
+                                                             B, Nmax, n_pages, max_blocks, Dp1);
+  TV_CUDA_OK(cudaGetLastError());
+  tv::count_launches(2);
+  return TV_OK;
+}
 
 extern "C" int kv_commit_inplace(tv_bf16* k_cache, tv_bf16* v_cache,
                                  const int32_t* accepted_nodes, const int32_t* accept_len,
