@@ -805,8 +805,10 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             claim_ret = atomicCAS(claim_ctr, claim_assumed, (prm.epoch << 16) | (unsigned long long)(claim_cnt + 1));
           }
           // ---- V rows past the valid keys may hold anything (stale cache rows, padded tree slots): zero
-          // them so that 0 * NaN never reaches O.  Idempotent, so both warpgroups may do it.
-          if (valid_keys < kTileN) {
+          // them so that 0 * NaN never reaches O.  Idempotent, so both warpgroups may do it.  Rows that lie
+          // outside the tensor arrive as zeros from the copy itself: a tree tile whose tree is full (the
+          // usual case) needs nothing.
+          if (valid_keys < kTileN && !(tree && !prm.tree_in_cache && tt * kTileN + valid_keys >= prm.Nmax)) {
             const uint32_t f = fill + 2 * jt + 1, slot = f % kSlots;
             ok = wwait(bar(L::KV_FULL + slot), (f / kSlots) & 1);
             if (!ok) break;
@@ -840,13 +842,15 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           if (jt == 0) prof[10] += pc1 - pitem;
 #endif
           tr.mark(0x1000u | (tj & 0xfffu));
-          // ---- whole-tile fast path (full, unmasked tiles after the first of the item): all 128 scores of the
-          // row in one load and P with the reference maximum as it stands; the row sum then tells whether
-          // anything left the lazy-rescale range (all P are >= 0, so the sum bounds every element; NaN and
-          // infinity fail the comparison).  P is only stored once the check has passed, so on a failure the
-          // scores are still in S and the chunk loop below does the tile again, maximum first.
+          // ---- whole-tile fast path (full, unmasked tiles): all 128 scores of the row in one load and P with
+          // the reference maximum as it stands; the row sum then tells whether anything left the lazy-rescale
+          // range (all P are >= 0, so the sum bounds every element; NaN and infinity fail the comparison).  P
+          // is only stored once the check has passed, so on a failure the scores are still in S and the chunk
+          // loop below does the tile again, maximum first.  A row without a reference yet (the first tile of
+          // an item) takes the score of the tile's first key: it is one of the row's scores, hence not above
+          // their maximum, and if it lies too far below it the check fails like any other.
           bool tile_done = false;
-          if (jt > 0 && full_tile) {
+          if (full_tile) {
             uint32_t sall[128];
             tmem_ld32(s_base, sall);
             tmem_ld32(s_base + 32, sall + 32);
@@ -855,8 +859,9 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             tmem_wait_ld();
             const float* sa = reinterpret_cast<const float*>(sall);
             const float2 c2 = make_float2(prm.scale_log2e, prm.scale_log2e);
-            const float nm = (m_used == -INFINITY) ? 0.f : -m_used;
-            const float2 nm2 = make_float2(nm, nm);
+            const bool opens = (m_used == -INFINITY);
+            const float m_ref = opens ? sa[0] * prm.scale_log2e : m_used;
+            const float2 nm2 = make_float2(-m_ref, -m_ref);
             float2 sum = make_float2(0.f, 0.f);
             uint32_t pkk[64];
 #pragma unroll
@@ -876,6 +881,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             const bool overflow = row_active && !(fsum <= 2.f * kMaxFastSum);
             if (!__any_sync(0xffffffffu, overflow)) {
               l_sum += fsum;
+              if (opens && row_active) m_used = m_ref;
 #pragma unroll
               for (int q = 0; q < 8; ++q)
                 asm volatile(
