@@ -63,11 +63,19 @@ constexpr float kMaxFastSum = 16384.0f;               // 64 keys x 2^threshold: 
 #define TV_POLY_SEL(i) (((i) & 7) == 3)
 #endif
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
-constexpr int kSetupCost = 4;      // virtual tiles charged per unit by the scheduler
+// virtual tiles charged per unit by the scheduler (32-layer shape, five seeds: 2 is 0.2-2 % faster than 4,
+// 0 and 1 are slower)
+#ifndef TV_SETUP_COST
+#define TV_SETUP_COST 2
+#endif
+constexpr int kSetupCost = TV_SETUP_COST;
 constexpr int kMaxGroups = 160;
 // do not spread a small problem over more CTA groups than this allows (measured on the 7B-shaped single
 // sequence: 12 -> 26 us, 6 -> 22 us, 4 -> 23 us per launch)
-constexpr int kMinVirtualTilesPerGroup = 6;
+#ifndef TV_MIN_VT
+#define TV_MIN_VT 6
+#endif
+constexpr int kMinVirtualTilesPerGroup = TV_MIN_VT;
 constexpr int kTraceCap = 256;     // events per (CTA, role) kept by the optional trace
 
 // ---------------------------------------------------------------- PTX helpers
@@ -454,6 +462,13 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const unsigned total = (unsigned)(prm.Hkv * cum[prm.B]);
     const unsigned want = total / (unsigned)kMinVirtualTilesPerGroup;
     groups = want < 1u ? 1 : (want < (unsigned)prm.groups ? (int)want : prm.groups);
+    // A group count just above a multiple of the unit count is rounded down to it: with units of equal length
+    // (one sequence, all heads) every unit is then cut into the same number of equal pieces and no cut falls
+    // just behind a unit boundary.  Not worth more than 1/16 of the groups.
+    {
+      const int units = prm.B * prm.Hkv, over = groups % units;
+      if (groups > units && over * 16 <= groups) groups -= over;
+    }
     // gs[k] = floor(total * k / groups) in 32-bit arithmetic: total = q * groups + r
     const unsigned q = total / (unsigned)groups, r = total % (unsigned)groups;
 #pragma unroll 1
