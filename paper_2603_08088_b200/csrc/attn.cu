@@ -57,10 +57,11 @@ constexpr int kMaxB = 512;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kRescaleThreshold = 8.0f;            // in log2 units
 constexpr float kMaxFastSum = 16384.0f;               // 64 keys x 2^threshold: largest row sum the fast path accepts
-// Of every 8 element pairs of the softmax fast path, one takes 2^x on the FMA pipe (measured optimum between
-// the special-function unit and the FMA pipe on the long-context shape).
+// Of every 16 element pairs of the softmax fast path, three take 2^x on the FMA pipe (measured optimum between
+// the special-function unit and the FMA pipe: 2/16 and 4/16 are 1-2 % slower on the 32-layer and the
+// long-context shape, 1/16 and 5/16 far slower).
 #ifndef TV_POLY_SEL
-#define TV_POLY_SEL(i) (((i) & 7) == 3)
+#define TV_POLY_SEL(i) ((((i) & 7) == 3) || (((i) & 15) == 7))
 #endif
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 // virtual tiles charged per unit by the scheduler (32-layer shape, five seeds: 2 is 0.2-2 % faster than 4,
