@@ -314,6 +314,75 @@ def node_scores(logits_bits, tokens, parent, n_nodes):
     return scores, status
 
 
+def stochastic_accept(logits_bits, tokens, parent, n_nodes, u_node, u_bonus, temperature, Dp1):
+    """Sampling-mode acceptance over the tree (Section 2.2: an acceptance rule "rejection sampling
+    style ... so that the resulting marginal distribution matches the teacher distribution"; Section
+    3.3: the node scores l(k) are what the rule consumes).  The paper prints no formula; this is the
+    speculative-sampling rule of the work it cites, for proposals that carry no draft probability
+    (q = one-hot on the proposed token), walked down the tree:
+
+      at the current node c (the root first) the teacher distribution is p = softmax(logits[c] / T);
+      its children k (parent[k] = c, increasing node id, valid slots only) are tried in turn:
+        x = tokens[k]; a token already rejected at this node is skipped;
+        accept k iff u_node[k] < p(x) / (1 - mass rejected so far at this node)
+        (= min(1, p'/q) with q = 1 and p' the distribution renormalised after the rejections);
+        otherwise x is rejected: its mass is removed and the next child is tried;
+      an accepted child becomes the current node (at most Dp1 - 1 accepted nodes);
+      when no child is accepted, the next token is drawn from p with the rejected tokens removed,
+      by inversion of the cumulative sum in vocabulary order at u_bonus.
+
+    The uniforms are inputs: u_node[B,Nmax] (one per node, read when that node is tried) and
+    u_bonus[B], all in [0,1).  Returns accept_len, accepted_nodes [B,Dp1] (first A+1 valid, rest 0),
+    next_token, status (BAD_INDEX for a proposed token outside [0,V); that child is never accepted).
+    T -> 0 gives the greedy rule; every output token is distributed as under plain sampling from the
+    teacher (the property the pins check).
+    """
+    B, Nmax, V = logits_bits.shape
+    accept_len = np.zeros(B, dtype=np.int32)
+    accepted_nodes = np.zeros((B, Dp1), dtype=np.int32)
+    next_token = np.zeros(B, dtype=np.int32)
+    status = np.zeros(B, dtype=np.int32)
+    for b in range(B):
+        n = int(min(max(int(n_nodes[b]), 0), Nmax))
+        c, depth = 0, 0
+        while True:
+            row = decode_bf16(logits_bits[b, c]).astype(np.float64) / float(temperature)
+            e = np.exp(row - row.max())
+            rejected = []
+            accepted = -1
+            if depth < Dp1 - 1:
+                for k in range(max(c, 0) + 1, n):
+                    pk = int(parent[b, k])
+                    if (pk if 0 <= pk < n else 0) != c:
+                        continue
+                    x = int(tokens[b, k])
+                    if not (0 <= x < V):
+                        status[b] |= ST_BAD_INDEX
+                        continue
+                    if x in rejected:
+                        continue
+                    kept = e.copy()
+                    kept[rejected] = 0.0
+                    rem = kept.sum()
+                    prob = e[x] / rem if rem > 0 else 0.0
+                    if float(u_node[b, k]) < prob:
+                        accepted = k
+                        break
+                    rejected.append(x)
+            if accepted < 0:
+                kept = e.copy()
+                kept[rejected] = 0.0
+                cum = np.cumsum(kept)
+                target = float(u_bonus[b]) * cum[-1]
+                next_token[b] = min(int(np.searchsorted(cum, target, side="right")), V - 1)
+                break
+            depth += 1
+            accepted_nodes[b, depth] = accepted
+            c = accepted
+        accept_len[b] = depth
+    return {"accept_len": accept_len, "accepted_nodes": accepted_nodes, "next_token": next_token, "status": status}
+
+
 def greedy_accept(retrieve, tokens, n_nodes, am):
     """Longest accepted prefix over all candidate rows (Section 2.3: accepted
     nodes form a single root-to-leaf path prefix; greedy rule, Section 5).

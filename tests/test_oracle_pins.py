@@ -579,6 +579,99 @@ def test_paged_cache_is_the_contiguous_cache_behind_a_block_table():
     assert (kp3[:, 7] == kp[:, 7]).all()
 
 
+# ---------------------------------------------------- sampling-mode acceptance ----
+def _stoch_case():
+    """V = 4, logits [2,1,0,0] in every row and T = 1/ln 2, so that p = [1/2, 1/4, 1/8, 1/8] exactly.
+    Tree: root 0 -> node 1 (token 1), node 2 (token 0); node 2 -> node 3 (token 3)."""
+    logits = _bf16(np.tile(np.array([2.0, 1.0, 0.0, 0.0], dtype=np.float32), (1, 4, 1)))
+    tokens = np.array([[9, 1, 0, 3]], dtype=np.int32)
+    parent = np.array([[-1, 0, 0, 2]], dtype=np.int32)
+    return logits, tokens, parent, np.array([4]), 1.0 / np.log(2.0)
+
+
+def test_stochastic_accept_hand_worked_example():
+    logits, tokens, parent, n, T = _stoch_case()
+    run = lambda un, ub: orc.stochastic_accept(logits, tokens, parent, n, np.array([un]), np.array([ub]), T, 4)
+    # root: node 1 (p = 1/4) fails at u = 0.3; node 2 has p = (1/2)/(3/4) = 2/3 and passes at 0.5; node 3 (p = 1/8)
+    # passes at 0.1; leaf: token from [1/2, 3/4, 7/8, 1] at 0.6 -> 1
+    r = run([0.0, 0.3, 0.5, 0.1], 0.6)
+    assert r["accept_len"].tolist() == [2] and r["accepted_nodes"].tolist() == [[0, 2, 3, 0]] and r["next_token"].tolist() == [1]
+    # node 2 fails at 0.7 > 2/3: tokens 1 and 0 are out, the rest is [0, 0, 1/2, 1/2]
+    r = run([0.0, 0.3, 0.7, 0.1], 0.4)
+    assert r["accept_len"].tolist() == [0] and r["accepted_nodes"].tolist() == [[0, 0, 0, 0]] and r["next_token"].tolist() == [2]
+    assert run([0.0, 0.3, 0.7, 0.1], 0.5)["next_token"].tolist() == [3]
+    assert run([0.0, 0.3, 0.7, 0.1], 0.0)["next_token"].tolist() == [2]       # never a rejected token, even at u = 0
+    # node 1 passes at once; it has no children: token drawn from the unmodified p
+    r = run([0.0, 0.2, 0.9, 0.9], 0.49)
+    assert r["accept_len"].tolist() == [1] and r["accepted_nodes"].tolist() == [[0, 1, 0, 0]] and r["next_token"].tolist() == [0]
+    # capacity of the accepted list: Dp1 = 2 keeps one accepted node and then samples at it
+    r = orc.stochastic_accept(logits, tokens, parent, n, np.array([[0.0, 0.3, 0.5, 0.0]]), np.array([0.8]), T, 2)
+    assert r["accept_len"].tolist() == [1] and r["accepted_nodes"].tolist() == [[0, 2]] and r["next_token"].tolist() == [2]
+    # a proposed token outside the vocabulary is never accepted and is reported
+    bad = tokens.copy()
+    bad[0, 1] = 4
+    r = orc.stochastic_accept(logits, bad, parent, n, np.array([[0.0, 0.0, 0.4, 0.9]]), np.array([0.1]), T, 4)
+    assert r["status"].tolist() == [orc.ST_BAD_INDEX] and r["accepted_nodes"].tolist() == [[0, 2, 0, 0]]
+
+
+def test_stochastic_accept_becomes_greedy_at_low_temperature():
+    rng = np.random.default_rng(31)
+    B, N, V, D = 3, 14, 50, 4
+    parent = np.stack([random_parent_tree(N, D, rng) for _ in range(B)])
+    n = np.array([N, N, 9])
+    vals = rng.standard_normal((B, N, V)).astype(np.float32)
+    for b in range(B):
+        for i in range(N):
+            vals[b, i, rng.integers(V)] = 6.0                  # a unique maximum per row
+    bits = _bf16(vals)
+    am = orc.argmax_rows(bits, n)
+    tokens = rng.integers(0, V, size=(B, N)).astype(np.int32)
+    for b in range(B):                                          # let some children carry the teacher's token
+        for k in range(1, int(n[b])):
+            if rng.random() < 0.6:
+                tokens[b, k] = am[b, parent[b, k]]
+    u = rng.random((B, N))
+    r = orc.stochastic_accept(bits, tokens, parent, n, u, rng.random(B), 1e-3, D + 1)
+    for b in range(B):                                          # the greedy walk: follow the child that carries the argmax
+        c, path = 0, [0]
+        while len(path) < D + 1:
+            nxt = [k for k in range(c + 1, int(n[b])) if parent[b, k] == c and tokens[b, k] == am[b, c]]
+            if not nxt:
+                break
+            c = nxt[0]
+            path.append(c)
+        assert r["accept_len"][b] == len(path) - 1 and r["accepted_nodes"][b, :len(path)].tolist() == path
+        assert r["next_token"][b] == am[b, c]
+
+
+def test_stochastic_accept_first_token_follows_the_teacher_distribution():
+    """The property the rule exists for: whatever the tree proposes (here with a duplicated sibling token and
+    a zero-probability-ish one), the first token that leaves the step is distributed as softmax(logits/T)
+    at the root.  30000 draws, every probability within 4.5 standard errors."""
+    rng = np.random.default_rng(32)
+    V, T = 6, 0.9
+    row = np.array([1.5, 0.25, 1.0, -2.0, 0.5, 0.0], dtype=np.float32)
+    bits = _bf16(np.tile(row, (1, 6, 1)))
+    tokens = np.array([[0, 2, 4, 2, 3, 1]], dtype=np.int32)       # children of the root: 2, 4, 2 (again), 3; node 5 under node 1
+    parent = np.array([[-1, 0, 0, 0, 0, 1]], dtype=np.int32)
+    n = np.array([6])
+    p = np.exp(orc.decode_bf16(bits[0, 0]).astype(np.float64) / T)
+    p /= p.sum()
+    draws = 30000
+    counts = np.zeros(V)
+    accepted = 0
+    for _ in range(draws):
+        r = orc.stochastic_accept(bits, tokens, parent, n, rng.random((1, 6)), rng.random(1), T, 3)
+        if r["accept_len"][0] >= 1:
+            counts[tokens[0, r["accepted_nodes"][0, 1]]] += 1
+            accepted += 1
+        else:
+            counts[r["next_token"][0]] += 1
+    se = np.sqrt(p * (1 - p) / draws)
+    assert (np.abs(counts / draws - p) < 4.5 * se).all(), (counts / draws, p)
+    assert 0.3 * draws < accepted < 0.9 * draws                  # both branches of the rule were exercised
+
+
 def test_node_scores_gather_and_link_to_greedy_acceptance():
     """score[k] = logits[parent(k), token(k)]: checked against numpy fancy indexing, and against the
     acceptance rule - a node is accepted by the greedy rule exactly when its score equals the row
