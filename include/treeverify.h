@@ -285,6 +285,46 @@ TV_API int tree_accept_noalloc(const tv_bf16* logits, const int32_t* tokens,
                                int32_t* accept_len, int32_t* best_path, int32_t* accepted_nodes,
                                int32_t* next_token, int32_t* status, tv_stream stream);
 
+/* Scratch needed by tree_accept_sample (bytes). */
+TV_API size_t tv_sample_workspace_bytes(int B, int Nmax, int V);
+
+/*
+ * Sampling-mode acceptance (temperature > 0) over the tree.  Section 2.2 asks
+ * for an acceptance rule "rejection sampling style" under which the output
+ * keeps the teacher's distribution, Section 3.3 names the node scores as its
+ * input; no formula is printed, so this is the reading: speculative sampling
+ * for proposals without a draft probability (q = one-hot on the proposed
+ * token), walked down the tree.  With p = softmax(logits[b,c,:] / temperature)
+ * at the current node c (the root first):
+ *   - the children of c (parent[k] = c after the dummy-root remap, valid
+ *     slots, increasing node id) are tried in turn; a token already rejected
+ *     at c is skipped; child k with token x is accepted iff
+ *       u_node[b,k] < p(x) / (1 - mass rejected so far at c);
+ *     otherwise x is rejected and its mass removed;
+ *   - an accepted child becomes the current node (at most Dp1 - 1 of them);
+ *   - when no child passes, next_token is drawn from p without the rejected
+ *     tokens: the first v whose cumulative mass in vocabulary order exceeds
+ *     u_bonus[b] times the remaining mass.
+ * Every token that leaves the step is then distributed as under plain
+ * sampling from the teacher; temperature -> 0 gives tree_accept's greedy rule.
+ * The uniforms are inputs (the library draws nothing): u_node[B,Nmax] and
+ * u_bonus[B], float32 in [0,1).  All probabilities are computed in fp32.
+ *
+ *   logits[B,Nmax,V] bf16, tokens[B,Nmax], parent[B,Nmax], n_nodes[B]   in
+ *   accept_len[B], accepted_nodes[B,Dp1] (first accept_len+1 valid, rest 0),
+ *   next_token[B] (-1 for a sequence without nodes)                     out
+ *   status[B]  in/out: TV_ST_BAD_INDEX is ORed in if a valid non-root slot
+ *              proposes a token outside [0,V) (that child is never accepted).
+ * The tree is taken as validated by tree_build_mask (parent[k] < k).
+ * Limits: Nmax <= 256, B * Nmax <= 65535, temperature > 0.
+ */
+TV_API int tree_accept_sample(const tv_bf16* logits, const int32_t* tokens, const int32_t* parent,
+                              const int32_t* n_nodes, const float* u_node, const float* u_bonus,
+                              float temperature, int B, int Nmax, int V, int Dp1,
+                              int32_t* accept_len, int32_t* accepted_nodes, int32_t* next_token,
+                              void* workspace, size_t workspace_bytes,
+                              int32_t* status, tv_stream stream);
+
 /*
  * Path-index commit with the prefix-sharing fast reorder (Section 3.1): the
  * committed prefix keeps its place and only the accepted segment is gathered

@@ -333,7 +333,8 @@ def stochastic_accept(logits_bits, tokens, parent, n_nodes, u_node, u_bonus, tem
 
     The uniforms are inputs: u_node[B,Nmax] (one per node, read when that node is tried) and
     u_bonus[B], all in [0,1).  Returns accept_len, accepted_nodes [B,Dp1] (first A+1 valid, rest 0),
-    next_token, status (BAD_INDEX for a proposed token outside [0,V); that child is never accepted).
+    next_token, status (BAD_INDEX if any valid non-root slot proposes a token outside [0,V); such a
+    child is never accepted).  A sequence without nodes returns accept_len 0 and next_token -1.
     T -> 0 gives the greedy rule; every output token is distributed as under plain sampling from the
     teacher (the property the pins check).
     """
@@ -344,6 +345,11 @@ def stochastic_accept(logits_bits, tokens, parent, n_nodes, u_node, u_bonus, tem
     status = np.zeros(B, dtype=np.int32)
     for b in range(B):
         n = int(min(max(int(n_nodes[b]), 0), Nmax))
+        if n == 0:
+            next_token[b] = -1
+            continue
+        if any(not (0 <= int(tokens[b, k]) < V) for k in range(1, n)):
+            status[b] |= ST_BAD_INDEX
         c, depth = 0, 0
         while True:
             row = decode_bf16(logits_bits[b, c]).astype(np.float64) / float(temperature)
@@ -357,7 +363,6 @@ def stochastic_accept(logits_bits, tokens, parent, n_nodes, u_node, u_bonus, tem
                         continue
                     x = int(tokens[b, k])
                     if not (0 <= x < V):
-                        status[b] |= ST_BAD_INDEX
                         continue
                     if x in rejected:
                         continue

@@ -16,6 +16,7 @@ TV_ST_BAD_TREE, TV_ST_BAD_INDEX, TV_ST_CAPACITY, TV_ST_TIMEOUT, TV_ST_PATHS_TRUN
 
 EXPORTS = ["tv_last_error", "tv_version", "tv_launch_count", "tree_build_mask", "tv_attn_workspace_bytes", "tree_verify_attn",
            "tv_accept_workspace_bytes", "tree_accept", "tree_node_scores", "tree_merge_partials", "tv_accept_noalloc_max_bytes", "tree_accept_noalloc",
+           "tv_sample_workspace_bytes", "tree_accept_sample",
            "kv_commit", "kv_commit_inplace", "tree_verify_attn_paged", "kv_commit_paged", "tv_step_staging_bytes",
            "tv_verify_step_host"]
 
@@ -75,6 +76,10 @@ def load():
     lib.tree_accept_noalloc.argtypes = [_c_vp] * 4 + [_c_int] * 5 + [_c_vp] * 7 + [_c_vp, _c_vp]
     lib.kv_commit.restype = _c_int
     lib.kv_commit.argtypes = [_c_vp] * 7 + [_c_int] * 7 + [_c_i64, _c_i64, _c_vp, _c_vp]
+    lib.tv_sample_workspace_bytes.restype = _c_sz
+    lib.tv_sample_workspace_bytes.argtypes = [_c_int] * 3
+    lib.tree_accept_sample.restype = _c_int
+    lib.tree_accept_sample.argtypes = [_c_vp] * 6 + [_c_f] + [_c_int] * 4 + [_c_vp] * 4 + [_c_sz, _c_vp, _c_vp]
     lib.tree_verify_attn_paged.restype = _c_int
     lib.tree_verify_attn_paged.argtypes = [_c_vp] * 9 + [_c_int] * 7 + [_c_f, _c_vp, _c_vp, _c_vp, _c_sz, _c_vp, _c_vp]
     lib.kv_commit_paged.restype = _c_int
@@ -180,6 +185,20 @@ def tree_merge_partials(o_parts, lse_parts, out, lse=None, stream=None):
     R, B, Nmax, Hq, d = o_parts.shape
     _check(load().tree_merge_partials(_ptr(o_parts), _ptr(lse_parts), R, B, Nmax, Hq, d, _ptr(out),
                                       _ptr(lse) if lse is not None else None, _stream(stream)))
+
+
+def tv_sample_workspace_bytes(B, Nmax, V):
+    return load().tv_sample_workspace_bytes(B, Nmax, V)
+
+
+def tree_accept_sample(logits, tokens, parent, n_nodes, u_node, u_bonus, temperature, accept_len, accepted_nodes,
+                       next_token, workspace, status, stream=None):
+    """Sampling-mode acceptance over the tree; u_node [B,Nmax] and u_bonus [B] are float32 uniforms in [0,1)."""
+    B, Nmax, V = logits.shape
+    _check(load().tree_accept_sample(_ptr(logits), _ptr(tokens), _ptr(parent), _ptr(n_nodes), _ptr(u_node),
+                                     _ptr(u_bonus), float(temperature), B, Nmax, V, accepted_nodes.shape[1],
+                                     _ptr(accept_len), _ptr(accepted_nodes), _ptr(next_token), _ptr(workspace),
+                                     workspace.numel() * workspace.element_size(), _ptr(status), _stream(stream)))
 
 
 def tv_accept_noalloc_max_bytes():
