@@ -347,6 +347,8 @@ def run_ours(args, cfg):
     if args.in_cache and has_accept:
         line["in_cache"] = in_cache_step(cfg, case, buf, prefix0, scale, given_rows, min(args.steps, 20), dev)
         case["prefix_len"].copy_(prefix0)
+    if args.sample_accept and has_accept:
+        line["sample_accept"] = sample_accept_leg(cfg, case, min(args.steps, 20), dev, args.seed)
     if args.paged and has_accept:
         line["paged"] = paged_step(cfg, case, buf, prefix0, scale, given_rows, min(args.steps, 20), dev, args.seed)
         case["prefix_len"].copy_(prefix0)
@@ -454,6 +456,34 @@ def in_cache_step(cfg, case, buf, prefix0, scale, given_rows, steps, dev):
     return {"steps": steps, "ms_per_step_median": med(t_step), "steps_per_sec": 1e3 / med(t_step),
             "attn_per_layer_us": med(t_attn) * 1e3, "commit_inplace_us": med(t_commit) * 1e3,
             "note": "tree K/V read from the cache rows behind the prefix; commit = reorder inside the cache"}
+
+
+def sample_accept_leg(cfg, case, steps, dev, seed):
+    """tree_accept_sample (temperature 1, seeded uniforms) on the workload's logits, L2 flushed between calls,
+    beside the greedy tree_accept of the step."""
+    import paper_2603_08088_b200 as tv
+    B, N, V, Dp1 = cfg.B, cfg.N, cfg.V, cfg.D + 1
+    g = torch.Generator(device=dev).manual_seed(seed)
+    u_node = torch.rand(B, N, device=dev, generator=g)
+    u_bonus = torch.rand(B, device=dev, generator=g)
+    z = lambda *s_: torch.zeros(s_, dtype=torch.int32, device=dev)
+    alen, nodes, nxt, status = z(B), z(B, Dp1), z(B), z(B)
+    ws = torch.zeros(max(16, tv.tv_sample_workspace_bytes(B, N, V)), dtype=torch.uint8, device=dev)
+    flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev)
+    ts = []
+    for it in range(2 + steps):
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        tv.tree_accept_sample(case["logits"], case["tokens"], case["parent"], case["n_nodes"], u_node, u_bonus, 1.0, alen,
+                              nodes, nxt, ws, status)
+        e1.record()
+        torch.cuda.synchronize()
+        if it >= 2:
+            ts.append(e0.elapsed_time(e1) * 1e3)
+    ts.sort()
+    return {"steps": steps, "temperature": 1.0, "us_median": ts[len(ts) // 2], "us_min": ts[0],
+            "mean_accept_len": float(alen.float().mean().item()), "logits_mb": case["logits"].numel() * 2 / 1e6}
 
 
 def paged_step(cfg, case, buf, prefix0, scale, given_rows, steps, dev, seed):
@@ -567,6 +597,8 @@ def main():
                     help="also time tree_verify_attn over the node budgets of the paper's sweep (extra key in the JSON line)")
     ap.add_argument("--in-cache", action="store_true",
                     help="also time the step with the tree's K/V inside the cache and the in-place commit")
+    ap.add_argument("--sample-accept", action="store_true",
+                    help="also time the sampling-mode acceptance (tree_accept_sample) on the workload's logits")
     ap.add_argument("--paged", action="store_true",
                     help="also time the step over a paged committed cache (pages of 128 rows, block table)")
     ap.add_argument("--context-split", type=int, default=1,
