@@ -316,6 +316,46 @@ def run_ours(args, cfg):
         if (host["status"].numpy() & 15).any():
             raise SystemExit(f"bench.py: fatal status from the host-buffer step: {host['status'].numpy()}")
 
+    # ---- the same step replayed from a captured CUDA graph (one graph per input copy): what the step costs
+    # once the host's launch path is out of the way
+    graph_leg = None
+    if args.graph:
+        try:
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            graphs = []
+            with torch.cuda.stream(side):
+                for i in range(n_sets):
+                    step_no[0] = i
+                    one_step()
+                    torch.cuda.synchronize()
+                    step_no[0] = i
+                    g = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g, stream=side):
+                        one_step()
+                    graphs.append(g)
+            torch.cuda.current_stream().wait_stream(side)
+            for i in range(3):
+                graphs[i % n_sets].replay()
+            torch.cuda.synchronize()
+            g0, g1 = ev(), ev()
+            g0.record()
+            for i in range(args.steps):
+                graphs[i % n_sets].replay()
+            g1.record()
+            torch.cuda.synchronize()
+            gms = g0.elapsed_time(g1)           # this rank's own clock: no collective inside an optional leg
+            graph_leg = {"steps": args.steps, "ms_per_step": gms / args.steps,
+                         "steps_per_sec_per_gpu": args.steps / (gms * 1e-3)}
+            if (buf.status.cpu().numpy() & 15).any():
+                raise SystemExit(f"bench.py: fatal status in the graph replay: {buf.status.cpu().numpy()}")
+
+        except SystemExit:
+            raise
+        except Exception as exc:      # the optional leg never takes the main line down
+            graph_leg = {"error": f"{type(exc).__name__}: {exc}"[:200]}
+            torch.cuda.synchronize()
+
     if rank != 0:
         return
     peak, peak_kind = measured_peaks()
@@ -342,6 +382,8 @@ def run_ours(args, cfg):
                      "tensor_tflops": attn_flops(cfg, S_host) / (attn_ms * 1e-3) / 1e12},
         "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e,
     }
+    if graph_leg is not None:
+        line["graph_replay"] = graph_leg
     if args.budget_sweep:
         line["budget_sweep"] = budget_sweep(args.seed, dev)
     if args.in_cache and has_accept:
@@ -597,6 +639,8 @@ def main():
                     help="also time tree_verify_attn over the node budgets of the paper's sweep (extra key in the JSON line)")
     ap.add_argument("--in-cache", action="store_true",
                     help="also time the step with the tree's K/V inside the cache and the in-place commit")
+    ap.add_argument("--no-graph", dest="graph", action="store_false",
+                    help="skip the extra leg that times the step replayed from a captured CUDA graph")
     ap.add_argument("--sample-accept", action="store_true",
                     help="also time the sampling-mode acceptance (tree_accept_sample) on the workload's logits")
     ap.add_argument("--paged", action="store_true",

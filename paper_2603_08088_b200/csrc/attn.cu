@@ -1131,6 +1131,11 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                   }
                 }
                 __threadfence();
+                // every piece has drawn its ticket and published: nobody touches the two counters again in
+                // this launch.  Clearing them lets the same launch be replayed with the same epoch (a captured
+                // CUDA graph) and find them unused.
+                *reinterpret_cast<volatile unsigned long long*>(ctr) = 0ull;
+                *reinterpret_cast<volatile unsigned long long*>(ctr + 1) = 0ull;
               }
               *last_flag = merger;
             }
