@@ -148,7 +148,10 @@ TV_API size_t tv_attn_workspace_bytes(int B, int Nmax, int Hq, int Hkv, int d, i
  * Behind another tree_verify_attn launch (the layers of one step) it starts
  * while that one drains and requests its first committed-prefix tiles at once;
  * q, the tree's K/V, anc_bits, out, lse and the workspace are only touched
- * after every earlier kernel of the stream has finished.  Behind any other
+ * after every earlier kernel of the stream has finished.  Behind
+ * tree_build_mask it may likewise start while the mask kernel runs (which
+ * itself starts only after everything in front of it has finished, so a
+ * commit further up the stream is complete by then).  Behind any other
  * kernel it starts when that kernel has finished, as usual.
  */
 TV_API int tree_verify_attn(const tv_bf16* q,

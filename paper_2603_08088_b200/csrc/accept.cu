@@ -46,6 +46,7 @@ __device__ __forceinline__ float vec8_max(const uint4& u) {
 __global__ void __launch_bounds__(kScanThreads)
 argmax_scan_kernel(const tv_bf16* __restrict__ logits, const int32_t* __restrict__ n_nodes,
                    int Nmax, int V, int n_chunks, ArgPair* __restrict__ partial) {
+  tv::pdl_enter();
   const int row = blockIdx.y;            // b * Nmax + i
   const int b = row / Nmax, i = row - b * Nmax;
   if (i >= n_nodes[b]) return;           // padded row: never read
@@ -138,6 +139,7 @@ accept_kernel(const ArgPair* __restrict__ partial, int n_chunks,
               int32_t* __restrict__ candidates, int32_t* __restrict__ accept_len,
               int32_t* __restrict__ best_path, int32_t* __restrict__ accepted_nodes,
               int32_t* __restrict__ next_token, int32_t* __restrict__ status) {
+  tv::pdl_enter();
   extern __shared__ int32_t am[];          // [Nmax] teacher argmax of this sequence
   __shared__ unsigned long long best_key;  // (accepted length << 32) | ~row : max = longest, then lowest row
   __shared__ int bad_index;
@@ -289,12 +291,11 @@ extern "C" int tree_accept(const tv_bf16* logits, const int32_t* tokens,
   const int n_chunks = scan_chunks(V);
   ArgPair* partial = static_cast<ArgPair*>(workspace);
   cudaStream_t s = (cudaStream_t)stream;
-  argmax_scan_kernel<<<dim3(n_chunks, B * Nmax), kScanThreads, 0, s>>>(logits, n_nodes, Nmax, V, n_chunks, partial);
-  TV_CUDA_OK(cudaGetLastError());
-  accept_kernel<<<B, 256, Nmax * sizeof(int32_t), s>>>(partial, n_chunks, tokens, retrieve_indices, n_nodes,
-                                                        Nmax, P, Dp1, argmax_tok, safe_idx, candidates,
-                                                        accept_len, best_path, accepted_nodes, next_token, status);
-  TV_CUDA_OK(cudaGetLastError());
+  TV_CUDA_OK(tv::launch_pdl(argmax_scan_kernel, dim3(n_chunks, B * Nmax), dim3(kScanThreads), 0, s, logits, n_nodes, Nmax, V,
+                            n_chunks, partial));
+  TV_CUDA_OK(tv::launch_pdl(accept_kernel, dim3(B), dim3(256), Nmax * sizeof(int32_t), s, partial, n_chunks, tokens,
+                            retrieve_indices, n_nodes, Nmax, P, Dp1, argmax_tok, safe_idx, candidates, accept_len, best_path,
+                            accepted_nodes, next_token, status));
   tv::count_launches(2);
   return TV_OK;
 }

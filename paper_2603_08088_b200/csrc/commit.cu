@@ -38,6 +38,7 @@ commit_copy_kernel(uint4* __restrict__ k_cache, uint4* __restrict__ v_cache,
                    const int32_t* __restrict__ prefix_len, const int32_t* __restrict__ status,
                    int B, int Nmax, int Hkv, int dvec, int Scap, int Dp1,
                    int64_t cache_layer_vec, int64_t tree_layer_vec) {
+  tv::pdl_enter();
   __shared__ int s_nodes[kCopyMaxDp1];
   const int b = blockIdx.x, l = blockIdx.y;
   const int A = accept_len[b];
@@ -67,6 +68,7 @@ __global__ void commit_finish_kernel(const int32_t* __restrict__ accepted_nodes,
                                      const int32_t* __restrict__ accept_len,
                                      int32_t* __restrict__ prefix_len, int32_t* __restrict__ status,
                                      int B, int Nmax, int Scap, int Dp1) {
+  tv::pdl_enter();
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= B) return;
   const int A = accept_len[b];
@@ -298,15 +300,13 @@ extern "C" int kv_commit(tv_bf16* k_cache, tv_bf16* v_cache,
   if (L == 0 || B == 0) return TV_OK;
   const int dvec = d / 8;
   cudaStream_t s = (cudaStream_t)stream;
-  commit_copy_kernel<<<dim3(B, L), kCopyThreads, 0, s>>>(
-      reinterpret_cast<uint4*>(k_cache), reinterpret_cast<uint4*>(v_cache),
-      reinterpret_cast<const uint4*>(k_tree), reinterpret_cast<const uint4*>(v_tree),
-      accepted_nodes, accept_len, prefix_len, status, B, Nmax, Hkv, dvec, Scap, Dp1,
-      cache_layer_stride / 8, tree_layer_stride / 8);
-  TV_CUDA_OK(cudaGetLastError());
-  commit_finish_kernel<<<(B + 127) / 128, 128, 0, s>>>(accepted_nodes, accept_len, prefix_len, status,
-                                                       B, Nmax, Scap, Dp1);
-  TV_CUDA_OK(cudaGetLastError());
+  TV_CUDA_OK(tv::launch_pdl(commit_copy_kernel, dim3(B, L), dim3(kCopyThreads), 0, s,
+                            reinterpret_cast<uint4*>(k_cache), reinterpret_cast<uint4*>(v_cache),
+                            reinterpret_cast<const uint4*>(k_tree), reinterpret_cast<const uint4*>(v_tree),
+                            accepted_nodes, accept_len, prefix_len, status, B, Nmax, Hkv, dvec, Scap, Dp1,
+                            cache_layer_stride / 8, tree_layer_stride / 8));
+  TV_CUDA_OK(tv::launch_pdl(commit_finish_kernel, dim3((B + 127) / 128), dim3(128), 0, s, accepted_nodes, accept_len,
+                            prefix_len, status, B, Nmax, Scap, Dp1));
   tv::count_launches(2);
   return TV_OK;
 }

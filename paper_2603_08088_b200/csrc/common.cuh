@@ -27,6 +27,34 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
       return ::tv::fail(TV_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(e__));            \
   } while (0)
 
+#ifdef __CUDACC__
+// Programmatic dependent launch for the small kernels of a step.  Launched with programmatic stream
+// serialisation, such a kernel first waits for everything in front of it in the stream and only then lets the
+// next kernel be scheduled: the next launch overlaps this kernel's body, and no kernel ever runs ahead of data
+// it reads (a kernel that reads inputs before its own wait, as tree_verify_attn does with the committed
+// prefix, can therefore only overtake the body of the kernel directly in front of it).
+__device__ __forceinline__ void pdl_enter() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 // Process-wide count of kernels this library has launched (diagnostics only).
 void count_launches(int n);
 

@@ -16,6 +16,7 @@ build_mask_kernel(const int32_t* __restrict__ parent, const int32_t* __restrict_
                   int32_t* __restrict__ depth, int32_t* __restrict__ anc_table,
                   int32_t* __restrict__ retrieve, int32_t* __restrict__ n_paths,
                   int32_t* __restrict__ status) {
+  tv::pdl_enter();
   extern __shared__ int32_t sm[];
   int32_t* sp = sm;                 // safe parent (sentinel and padding -> 0)
   int32_t* dep = sm + Nmax;
@@ -161,10 +162,9 @@ extern "C" int tree_build_mask(const int32_t* parent, const int32_t* n_nodes,
   int threads = ((Nmax + 31) / 32) * 32;
   if (threads < 128) threads = 128;
   const size_t smem = 3 * (size_t)Nmax * sizeof(int32_t);
-  build_mask_kernel<<<B, threads, smem, (cudaStream_t)stream>>>(
-      parent, n_nodes, Nmax, Dcap, Pcap, W, anc_bits, dense_mask, depth, anc_table,
-      retrieve_indices, n_paths, status);
-  TV_CUDA_OK(cudaGetLastError());
+  TV_CUDA_OK(tv::launch_pdl(build_mask_kernel, dim3(B), dim3(threads), smem, (cudaStream_t)stream,
+                            parent, n_nodes, Nmax, Dcap, Pcap, W, anc_bits, dense_mask, depth, anc_table,
+                            retrieve_indices, n_paths, status));
   tv::count_launches(1);
   return TV_OK;
 }
