@@ -273,7 +273,7 @@ TV_API int tree_merge_partials(const tv_bf16* o_parts, const float* lse_parts, i
  * the scratch of the argmax reduction is a fixed 256 KiB array inside the
  * library image (every GPU that loads the library holds it until exit).
  * Same arguments and results as tree_accept, without the workspace.
- *   - Limit: B * Nmax * ceil(V / 8192) <= 32768 scratch entries
+ *   - Limit: B * Nmax * ceil(V / 16384) <= 32768 scratch entries
  *     (tv_accept_noalloc_max_bytes() / 8); larger problems are rejected with
  *     TV_ERR_WORKSPACE and must use tree_accept.
  *   - The first call on each device looks up the array's device address (with

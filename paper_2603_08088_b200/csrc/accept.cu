@@ -3,7 +3,7 @@
 // acceptance along root-to-leaf rows (Section 2.3).
 //
 // Phase 1 (argmax_scan_kernel) streams logits[B,Nmax,V] once with 16-byte
-// loads; every CTA reduces one vocabulary chunk of one row to a (value,
+// streaming loads; every CTA reduces one vocabulary chunk of one row to a (value,
 // index) pair in scratch.  Phase 2 (accept_kernel), one CTA per sequence,
 // folds the chunk pairs in index order, then remaps, gathers and compares.
 // Ties resolve to the lowest index at every level of the reduction.
@@ -16,8 +16,8 @@
 namespace {
 
 constexpr int kScanThreads = 256;
-constexpr int kVecPerThread = 4;                                   // 16-byte loads in flight per thread
-constexpr int kChunkElems = kScanThreads * kVecPerThread * 8;      // 8192 logits per CTA
+constexpr int kVecPerThread = 8;                                   // 16-byte loads in flight per thread
+constexpr int kChunkElems = kScanThreads * kVecPerThread * 8;      // 16384 logits per CTA
 
 struct ArgPair {
   float val;
@@ -68,7 +68,7 @@ argmax_scan_kernel(const tv_bf16* __restrict__ logits, const int32_t* __restrict
 #pragma unroll
     for (int k = 0; k < kVecPerThread; ++k) {
       vi[k] = v0 + k * kScanThreads + tid;
-      u[k] = vi[k] < v1 ? __ldg(vbase + vi[k]) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
+      u[k] = vi[k] < v1 ? __ldcs(vbase + vi[k]) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
     }
     int best_vec = -1;
 #pragma unroll

@@ -70,7 +70,7 @@ row_stats_kernel(const tv_bf16* __restrict__ logits, const int32_t* __restrict__
   for (int q = 0; q < kStatVecPerThread; ++q) {
     const int v0 = c0 + (q * kStatThreads + tid) * 8;
     if (vec_ok && v0 + 8 <= c1) {
-      const uint4 u = __ldg(reinterpret_cast<const uint4*>(base + v0));
+      const uint4 u = __ldcs(reinterpret_cast<const uint4*>(base + v0));
       const uint32_t e[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
       for (int t = 0; t < 8; ++t) vals[q * 8 + t] = bf16_to_float((t & 1) ? (e[t >> 1] >> 16) : (e[t >> 1] & 0xffffu));

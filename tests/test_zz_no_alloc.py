@@ -57,7 +57,7 @@ def test_noalloc_matches_workspace_entry_point_twice_in_a_row():
 
 def test_noalloc_rejects_problems_beyond_its_scratch():
     assert tv.tv_accept_noalloc_max_bytes() == 32768 * 8
-    cfg = CONFIGS[4].scaled(L=1, S_lo=1, S_hi=4, Scap=16, B=16, V=32768 * 9)    # 16*60*36 > 32768 entries
+    cfg = CONFIGS[4].scaled(L=1, S_lo=1, S_hi=4, Scap=16, B=16, V=16384 * 36)   # 16*60*36 > 32768 entries
     dev = "cuda"
     B, N, V, P, Dp1 = cfg.B, cfg.N, cfg.V, 10, cfg.D + 1
     logits = torch.zeros(1, dtype=torch.bfloat16, device=dev)     # never read: the call is rejected first
