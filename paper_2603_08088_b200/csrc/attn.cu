@@ -340,14 +340,6 @@ struct Sched {
   int B, Hkv;
   int total;         // Hkv * cum[B]; the host refuses problems whose tile count does not fit 31 bits
   __device__ __forceinline__ int group_start(int k, int) const { return gs[k]; }
-  __device__ __forceinline__ int find_group(int pos, int groups) const {
-    int lo = 0, hi = groups - 1;   // largest k with gs[k] <= pos
-    while (lo < hi) {
-      const int mid = (lo + hi + 1) >> 1;
-      if (gs[mid] <= pos) lo = mid; else hi = mid - 1;
-    }
-    return lo;
-  }
   __device__ __forceinline__ int find_b(int g) const {
     int lo = 0, hi = B - 1;   // largest b with Hkv*cum[b] <= g
     while (lo < hi) {
