@@ -100,6 +100,14 @@ TV_API int tree_build_mask(const int32_t* parent, const int32_t* n_nodes,
                     int32_t* anc_table, int32_t* retrieve_indices, int32_t* n_paths,
                     int32_t* status, tv_stream stream);
 
+/* Flags of tree_verify_attn_layers. */
+enum {
+  TV_ATTN_STABLE_INPUTS = 1   /* the caller promises: the kernel directly in front of this call on the stream does
+                                 not write prefix_len, n_nodes or rows [0, prefix_len) of the cache - or it does, but
+                                 lets no successor start before it has completed.  tree_build_mask in front (the
+                                 usual step) satisfies it; kv_commit in front does not. */
+};
+
 /* Scratch needed by tree_verify_attn for these dimensions (bytes). */
 TV_API size_t tv_attn_workspace_bytes(int B, int Nmax, int Hq, int Hkv, int d, int Scap);
 
@@ -140,19 +148,18 @@ TV_API size_t tv_attn_workspace_bytes(int B, int Nmax, int Hq, int Hkv, int d, i
  * Limits: d in {64,128}; Nmax <= 256 (the node budgets of the paper's sweep);
  * Hq % Hkv == 0, Hq / Hkv <= 128; B <= 512; all tensors 16-byte aligned;
  * 0 <= prefix_len[b] <= Scap; scale > 0.
+ * B > 192 is served by several launches over consecutive ranges of sequences.
  * CUDA graphs: every call of this header only launches on the given stream, so a
  * step can be captured into a CUDA graph and replayed; the split-KV counters in
  * the workspace are cleared by the piece that merges, so a replay (which
  * repeats the call's internal epoch) finds them unused.
- * Stream order: the kernel is launched with programmatic stream serialisation.
- * Behind another tree_verify_attn launch (the layers of one step) it starts
- * while that one drains and requests its first committed-prefix tiles at once;
- * q, the tree's K/V, anc_bits, out, lse and the workspace are only touched
- * after every earlier kernel of the stream has finished.  Behind
- * tree_build_mask it may likewise start while the mask kernel runs (which
- * itself starts only after everything in front of it has finished, so a
- * commit further up the stream is complete by then).  Behind any other
- * kernel it starts when that kernel has finished, as usual.
+ * Stream order: the kernel is launched with programmatic stream serialisation,
+ * so it may be scheduled while the kernel in front of it still runs (if that
+ * kernel allows it), but it reads and writes nothing of the problem before
+ * every earlier kernel of the stream has finished: only its own set-up
+ * (barriers, tensor memory, descriptor fetch) overlaps.  Reading
+ * the committed prefix earlier than that is what tree_verify_attn_layers
+ * offers, under a promise by the caller.
  */
 TV_API int tree_verify_attn(const tv_bf16* q,
                      const tv_bf16* k_cache, const tv_bf16* v_cache,
@@ -165,6 +172,32 @@ TV_API int tree_verify_attn(const tv_bf16* q,
                      int32_t* status, tv_stream stream);
 
 /*
+ * tree_verify_attn for all L layers of a step in one call (Section 2.3: the
+ * teacher evaluates the whole tree in one forward; every layer attends under
+ * the same mask and the same prefix lengths).  Layer l reads q, k_cache,
+ * v_cache, k_tree, v_tree (both NULL: in-cache layout) at l times the given
+ * layer stride (elements), writes out at l * out_layer_stride and lse (dense
+ * [L,B,Hq,Nmax], or NULL).  Everything else is as for tree_verify_attn, which
+ * this call equals layer by layer.
+ * What it adds is launch overlap that a single call cannot take by itself:
+ * the launch of layer l + 1 is scheduled while layer l drains and requests
+ * its first committed-prefix tiles at once - inside one call the library
+ * knows that the kernel in front is its own and leaves those inputs alone.
+ * With TV_ATTN_STABLE_INPUTS in flags the caller extends that promise to the
+ * kernel in front of the call, and layer 0 overlaps it too.
+ */
+TV_API int tree_verify_attn_layers(const tv_bf16* q,
+                     const tv_bf16* k_cache, const tv_bf16* v_cache,
+                     const tv_bf16* k_tree, const tv_bf16* v_tree,
+                     const int32_t* prefix_len, const int32_t* n_nodes,
+                     const uint32_t* anc_bits,
+                     int L, int B, int Nmax, int Hq, int Hkv, int d, int Scap, float scale,
+                     int64_t q_layer_stride, int64_t cache_layer_stride, int64_t tree_layer_stride,
+                     tv_bf16* out, int64_t out_layer_stride, float* lse,
+                     void* workspace, size_t workspace_bytes,
+                     int32_t* status, unsigned flags, tv_stream stream);
+
+/*
  * tree_verify_attn over a paged committed cache (Section 3.1 speaks of
  * backend-specific KV layouts behind one cache interface; this is the block
  * layout of serving stacks).  A page holds 128 consecutive rows - one key tile
@@ -174,9 +207,7 @@ TV_API int tree_verify_attn(const tv_bf16* q,
  * are read.  The capacity of a sequence is 128 * max_blocks rows.  The tree's
  * K/V come in their own buffers.  Everything else - arguments, outputs,
  * workspace (tv_attn_workspace_bytes with any Scap), limits, stream order - is
- * as for tree_verify_attn; the block table is read like prefix_len, before
- * earlier kernels of the stream have finished, so it must not be written by a
- * tree_verify_attn call in front.  A page id outside [0, n_pages) raises
+ * as for tree_verify_attn.  A page id outside [0, n_pages) raises
  * TV_ST_BAD_INDEX for the sequence (its output is unspecified; nothing is
  * read outside the pool).
  */

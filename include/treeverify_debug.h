@@ -1,0 +1,58 @@
+/*
+ * treeverify_debug.h - test and tuning aids exported by libtreeverify.so next
+ * to the public interface of treeverify.h.  None of them is on the product
+ * path: the library never calls them, the Python step never calls them; the
+ * parity tests use the first as an on-device cross-check of the tensor-core
+ * kernel and the second to see a bounded wait expire.
+ */
+#ifndef TREEVERIFY_DEBUG_H_
+#define TREEVERIFY_DEBUG_H_
+
+#include "treeverify.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/*
+ * tree_verify_attn computed by a plain CUDA-core kernel (one warp per query
+ * row, fp32 online softmax): same arguments and results, no workspace, no
+ * status.  A second, independently written GPU implementation of Sections
+ * 2.3 / 3.3 for cross-checks.
+ */
+TV_API int tv_debug_attn_simt(const tv_bf16* q, const tv_bf16* k_cache, const tv_bf16* v_cache,
+                              const tv_bf16* k_tree, const tv_bf16* v_tree,
+                              const int32_t* prefix_len, const int32_t* n_nodes, const uint32_t* anc_bits,
+                              int B, int Nmax, int Hq, int Hkv, int d, int Scap, float scale,
+                              tv_bf16* out, float* lse, tv_stream stream);
+
+/*
+ * tree_verify_attn with the limit of every bounded wait inside the kernel set
+ * to wait_limit_ns (the product uses 2 s).  mode bit 0: the producer warp
+ * issues no copy at all, so the first wait of the MMA-issuing warp expires.
+ * The launch then ends by itself: every role leaves its loop, the tensor
+ * memory is freed, and TV_ST_TIMEOUT is ORed into status[b] of every
+ * sequence (out and lse are unspecified).  Nothing traps or faults; the next
+ * launch on the device works as usual.  mode 0 is an ordinary launch.
+ * (Section 4.3 of the paper, the failure dump on a runtime error, is the
+ * nearest counterpart.)
+ */
+TV_API int tv_debug_attn_expire(const tv_bf16* q, const tv_bf16* k_cache, const tv_bf16* v_cache,
+                                const tv_bf16* k_tree, const tv_bf16* v_tree,
+                                const int32_t* prefix_len, const int32_t* n_nodes, const uint32_t* anc_bits,
+                                int B, int Nmax, int Hq, int Hkv, int d, int Scap, float scale,
+                                tv_bf16* out, float* lse, void* workspace, size_t workspace_bytes,
+                                int32_t* status, unsigned long long wait_limit_ns, int mode, tv_stream stream);
+
+/*
+ * Live only in a library built with -DTV_TRACE: while a device buffer of
+ * 160 * 5 * 256 uint64 is registered here, every tree_verify_attn launch
+ * records a per-CTA, per-role timeline (tag << 48 | globaltimer ns) into it.
+ * NULL switches it off.
+ */
+TV_API void tv_debug_set_attn_trace(unsigned long long* device_buffer);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TREEVERIFY_DEBUG_H_ */

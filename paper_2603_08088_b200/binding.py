@@ -13,8 +13,10 @@ LIB_PATH = os.path.join(_PKG, "libtreeverify.so")
 
 TV_OK, TV_ERR_INVALID_ARG, TV_ERR_CUDA, TV_ERR_WORKSPACE = 0, 1, 2, 3
 TV_ST_BAD_TREE, TV_ST_BAD_INDEX, TV_ST_CAPACITY, TV_ST_TIMEOUT, TV_ST_PATHS_TRUNCATED = 1, 2, 4, 8, 16
+TV_ATTN_STABLE_INPUTS = 1
 
 EXPORTS = ["tv_last_error", "tv_version", "tv_launch_count", "tree_build_mask", "tv_attn_workspace_bytes", "tree_verify_attn",
+           "tree_verify_attn_layers",
            "tv_accept_workspace_bytes", "tree_accept", "tree_node_scores", "tree_merge_partials", "tv_accept_noalloc_max_bytes", "tree_accept_noalloc",
            "tv_sample_workspace_bytes", "tree_accept_sample",
            "kv_commit", "kv_commit_inplace", "tree_verify_attn_paged", "kv_commit_paged", "tv_step_staging_bytes",
@@ -62,6 +64,9 @@ def load():
     lib.tv_attn_workspace_bytes.argtypes = [_c_int] * 6
     lib.tree_verify_attn.restype = _c_int
     lib.tree_verify_attn.argtypes = [_c_vp] * 8 + [_c_int] * 6 + [_c_f, _c_vp, _c_vp, _c_vp, _c_sz, _c_vp, _c_vp]
+    lib.tree_verify_attn_layers.restype = _c_int
+    lib.tree_verify_attn_layers.argtypes = ([_c_vp] * 8 + [_c_int] * 7 + [_c_f] + [_c_i64] * 3 + [_c_vp, _c_i64, _c_vp, _c_vp, _c_sz,
+                                            _c_vp, ctypes.c_uint, _c_vp])
     lib.tv_accept_workspace_bytes.restype = _c_sz
     lib.tv_accept_workspace_bytes.argtypes = [_c_int] * 3
     lib.tree_accept.restype = _c_int
@@ -90,6 +95,10 @@ def load():
     lib.tv_step_staging_bytes.argtypes = [_c_int] * 10
     lib.tv_verify_step_host.restype = _c_int
     lib.tv_verify_step_host.argtypes = [ctypes.POINTER(StepHostArgs)]
+    if hasattr(lib, "tv_debug_attn_expire"):
+        lib.tv_debug_attn_expire.restype = _c_int
+        lib.tv_debug_attn_expire.argtypes = ([_c_vp] * 8 + [_c_int] * 6 + [_c_f, _c_vp, _c_vp, _c_vp, _c_sz, _c_vp,
+                                              ctypes.c_ulonglong, _c_int, _c_vp])
     if hasattr(lib, "tv_debug_attn_simt"):
         lib.tv_debug_attn_simt.restype = _c_int
         lib.tv_debug_attn_simt.argtypes = [_c_vp] * 8 + [_c_int] * 6 + [_c_f, _c_vp, _c_vp, _c_vp]
@@ -153,6 +162,40 @@ def tree_verify_attn(q, k_cache, v_cache, k_tree, v_tree, prefix_len, n_nodes, a
                                    _ptr(prefix_len), _ptr(n_nodes), _ptr(anc_bits), B, Nmax, Hq, Hkv, d, Scap,
                                    float(scale), _ptr(out), _ptr(lse), _ptr(workspace),
                                    workspace.numel() * workspace.element_size(), _ptr(status), _stream(stream)))
+
+
+def tree_verify_attn_layers(q, k_cache, v_cache, k_tree, v_tree, prefix_len, n_nodes, anc_bits, scale, out,
+                            workspace, status, lse=None, flags=0, stream=None):
+    """All layers of a step in one call: q, out [L,B,Nmax,Hq,d], k_cache, v_cache [L,B,Hkv,Scap,d], k_tree, v_tree
+    [L,B,Nmax,Hkv,d] (or None: in-cache layout), lse [L,B,Hq,Nmax] or None; layer strides are taken from the tensors."""
+    L, B, Nmax, Hq, d = q.shape
+    _, _, Hkv, Scap, _ = k_cache.shape
+    for t in (q, k_cache, v_cache, k_tree, v_tree, out, lse):
+        assert t is None or t.shape[0] == L
+        assert t is None or t[0].is_contiguous(), "treeverify takes dense layers"
+    assert k_cache.stride(0) == v_cache.stride(0) and (k_tree is None or k_tree.stride(0) == v_tree.stride(0))
+    assert lse is None or lse.is_contiguous()
+    _check(load().tree_verify_attn_layers(q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(),
+                                          None if k_tree is None else k_tree.data_ptr(),
+                                          None if v_tree is None else v_tree.data_ptr(), _ptr(prefix_len), _ptr(n_nodes),
+                                          _ptr(anc_bits), L, B, Nmax, Hq, Hkv, d, Scap, float(scale), q.stride(0),
+                                          k_cache.stride(0), 0 if k_tree is None else k_tree.stride(0), out.data_ptr(),
+                                          out.stride(0), None if lse is None else lse.data_ptr(), _ptr(workspace),
+                                          workspace.numel() * workspace.element_size(), _ptr(status), int(flags),
+                                          _stream(stream)))
+
+
+def tv_debug_attn_expire(q, k_cache, v_cache, k_tree, v_tree, prefix_len, n_nodes, anc_bits, scale, out, workspace, status,
+                         wait_limit_ns, mode, lse=None, stream=None):
+    """Test aid (treeverify_debug.h): tree_verify_attn with a short limit on its bounded waits and, with mode bit 0,
+    a producer that never delivers, so that a wait expires."""
+    B, Nmax, Hq, d = q.shape
+    _, Hkv, Scap, _ = k_cache.shape
+    _check(load().tv_debug_attn_expire(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(k_tree), _ptr(v_tree),
+                                       _ptr(prefix_len), _ptr(n_nodes), _ptr(anc_bits), B, Nmax, Hq, Hkv, d, Scap,
+                                       float(scale), _ptr(out), _ptr(lse), _ptr(workspace),
+                                       workspace.numel() * workspace.element_size(), _ptr(status), int(wait_limit_ns),
+                                       int(mode), _stream(stream)))
 
 
 def tv_debug_attn_simt(q, k_cache, v_cache, k_tree, v_tree, prefix_len, n_nodes, anc_bits, scale, out,

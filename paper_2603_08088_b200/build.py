@@ -33,7 +33,8 @@ def _nvcc():
 
 
 def _newest_header():
-    hdrs = [os.path.join(ROOT, "include", "treeverify.h")]
+    inc = os.path.join(ROOT, "include")
+    hdrs = [os.path.join(inc, f) for f in os.listdir(inc) if f.endswith(".h")]
     hdrs += [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cuh", ".h"))]
     return max(os.path.getmtime(h) for h in hdrs)
 

@@ -6,6 +6,7 @@
 // set, padded rows give 0 / -inf, rows past the prefix and padded tree slots
 // are never multiplied in (their V rows are staged as zeros).
 #include "common.cuh"
+#include "treeverify_debug.h"
 
 #include <cuda_bf16.h>
 

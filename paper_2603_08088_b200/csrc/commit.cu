@@ -68,7 +68,9 @@ __global__ void commit_finish_kernel(const int32_t* __restrict__ accepted_nodes,
                                      const int32_t* __restrict__ accept_len,
                                      int32_t* __restrict__ prefix_len, int32_t* __restrict__ status,
                                      int B, int Nmax, int Scap, int Dp1) {
-  tv::pdl_enter();
+  // This kernel writes prefix_len, which a tree_verify_attn launch directly behind it reads before its own
+  // wait: the next launch must not start until this grid is complete, so nothing is released early here.
+  tv::pdl_wait_only();
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= B) return;
   const int A = accept_len[b];

@@ -37,6 +37,10 @@ __device__ __forceinline__ void pdl_enter() {
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
+// For a kernel that writes something a later kernel reads BEFORE that kernel's own wait (prefix_len, which
+// tree_verify_attn reads at once): wait for everything in front, and never release the next launch early - it is
+// released when this grid has completed and its writes are visible.
+__device__ __forceinline__ void pdl_wait_only() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,

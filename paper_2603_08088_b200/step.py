@@ -54,12 +54,12 @@ def verify_step(case, buf: StepBuffers, scale, retrieve=None, commit=True, strea
                        dense_mask=buf.dense, depth=buf.depth, anc_table=buf.anc_table,
                        retrieve_indices=buf.retrieve if own_rows else None,
                        n_paths=buf.n_paths, stream=stream)
-    for l in range(L):
-        tv.tree_verify_attn(case["q"][l], case["k_cache"][l], case["v_cache"][l],
-                            None if in_cache else case["k_tree"][l], None if in_cache else case["v_tree"][l],
-                            case["prefix_len"], case["n_nodes"], buf.anc_bits, scale,
-                            buf.out[l], buf.attn_ws, buf.status,
-                            lse=None if buf.lse is None else buf.lse[l], stream=stream)
+    # all layers in one call; the mask kernel in front leaves prefix_len and the cache alone, so the first layer
+    # may start under it as well
+    tv.tree_verify_attn_layers(case["q"], case["k_cache"], case["v_cache"],
+                               None if in_cache else case["k_tree"], None if in_cache else case["v_tree"],
+                               case["prefix_len"], case["n_nodes"], buf.anc_bits, scale, buf.out, buf.attn_ws,
+                               buf.status, lse=buf.lse, flags=tv.TV_ATTN_STABLE_INPUTS, stream=stream)
     if V > 0 and "logits" in case:
         rows = buf.retrieve if own_rows else retrieve
         tv.tree_accept(case["logits"], case["tokens"], rows, case["n_nodes"], buf.argmax_tok, buf.accept_len,

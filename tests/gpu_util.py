@@ -49,3 +49,29 @@ def oracle_attention_slice(case_np, layer, b, hk, G, vis, scale):
     vt = case_np["v_tree"][layer][b:b + 1, :, hk:hk + 1]
     return orc.tree_attention(q, kc, vc, kt, vt, case_np["prefix_len"][b:b + 1], case_np["n_nodes"][b:b + 1],
                               vis[b:b + 1], scale)
+
+
+def oracle_visibility(parent, n_nodes, dense_gpu=None, bits_gpu=None):
+    """The tree mask the ORACLE builds from the parent arrays, as dense[B,1,N,N] u8 (numpy).  The attention
+    parity tests feed this one to the oracle's attention, never the mask the CUDA kernel produced; when the
+    CUDA mask is passed in as well it must be the same bit for bit."""
+    parent = np.asarray(parent.detach().cpu().numpy() if isinstance(parent, torch.Tensor) else parent)
+    n_nodes = np.asarray(n_nodes.detach().cpu().numpy() if isinstance(n_nodes, torch.Tensor) else n_nodes)
+    B, N = parent.shape
+    # the ancestor relation does not depend on the depth bound once it covers the deepest node: take the
+    # deepest level of these trees (a plain parent walk) so that the oracle's loops stay short
+    deepest = 0
+    for b in range(B):
+        for i in range(int(n_nodes[b])):
+            k, j = 0, i
+            while j > 0 and k <= N:
+                j = int(parent[b, j])
+                k += 1
+            deepest = max(deepest, k)
+    mk = orc.build_mask(parent, n_nodes, min(deepest, max(N - 1, 0)), 1, emit_paths=False)
+    assert (mk["status"] & orc.ST_BAD_TREE == 0).all(), "the oracle rejects a tree of this case"
+    if dense_gpu is not None:
+        assert np.array_equal(i32(dense_gpu), mk["dense"]), "CUDA dense mask differs from the oracle's"
+    if bits_gpu is not None:
+        assert np.array_equal(i32(bits_gpu).view(np.uint32), mk["anc_bits"]), "CUDA ancestor words differ from the oracle's"
+    return mk["dense"]

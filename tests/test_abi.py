@@ -18,8 +18,8 @@ def lib():
     return tv.load()
 
 
-def _declared_symbols():
-    text = open(os.path.join(ROOT, "include", "treeverify.h")).read()
+def _declared_symbols(header="treeverify.h"):
+    text = open(os.path.join(ROOT, "include", header)).read()
     return re.findall(r"^TV_API\s+[\w\s\*]+?\b(\w+)\(", text, flags=re.M)
 
 
@@ -30,6 +30,11 @@ def test_header_symbols_are_exported(lib):
     for n in names:
         assert hasattr(lib, n), f"{n} declared in treeverify.h but not exported"
     assert set(names) == set(tv.EXPORTS)
+    debug = _declared_symbols("treeverify_debug.h")            # test and tuning aids: declared apart, exported too
+    assert set(debug) == {"tv_debug_attn_simt", "tv_debug_attn_expire", "tv_debug_set_attn_trace"}
+    for n in debug:
+        assert hasattr(lib, n), f"{n} declared in treeverify_debug.h but not exported"
+    assert not set(debug) & set(names)
 
 
 def test_version_and_size_queries(lib):

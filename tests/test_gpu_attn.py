@@ -11,13 +11,15 @@ import paper_2603_08088_b200 as tv
 from oracle import tree_verify_oracle as orc
 from workloads import (CONFIGS, make_case, case_to_numpy, bf16_bits, random_parent_tree, topk_expansion_tree,
                        chain_tree)
-from gpu_util import to_device, f32, assert_attention_close, oracle_attention_slice, ATTN_ATOL
+from gpu_util import to_device, f32, assert_attention_close, oracle_attention_slice, oracle_visibility, ATTN_ATOL
 
 pytestmark = pytest.mark.gpu
 
 
 def gpu_attention(case, layer=0, simt=False):
-    """case: device tensors.  Returns (out, lse, anc_bits, dense) for one layer."""
+    """case: device tensors.  Returns (out, lse, anc_bits, dense) for one layer; `dense` is the ORACLE's
+    mask of the same trees (the CUDA mask is checked equal to it here and then dropped), so that every
+    expected value below comes from the oracle alone."""
     L, B, N, Hq, d = case["q"].shape
     Hkv, Scap = case["k_cache"].shape[2], case["k_cache"].shape[3]
     dev = case["q"].device
@@ -40,6 +42,7 @@ def gpu_attention(case, layer=0, simt=False):
                             case["n_nodes"], bits, scale, out, ws, status, lse=lse)
     torch.cuda.synchronize()
     assert (status.cpu().numpy() == 0).all(), f"status {status.cpu().numpy()}"
+    dense = torch.from_numpy(oracle_visibility(case["parent"], case["n_nodes"], dense_gpu=dense, bits_gpu=bits))
     return out, lse, bits, dense
 
 
@@ -162,6 +165,44 @@ def test_leak_canary_one_hot_values(S):
     for h in range(2):
         assert np.abs(got[:, h] - want).max() <= 0.26      # 100/k rounded to bf16: half-ulp of 64..128 is 0.25
     # a leak of one key would shift some entry by >= 100/(S+8) > 4
+
+
+MOVES = [
+    # name, S, N, index of the dominant key (prefix row, or S + tree node)
+    ("ragged_prefix_tile_second_half", 242, 8, 200),
+    ("first_tile_of_the_item_second_half", 100, 8, 80),
+    ("tree_tile_second_half", 40, 128, 40 + 100),
+    ("whole_tile_then_ragged_tile", 370, 8, 340),
+]
+
+
+@pytest.mark.parametrize("name,S,N,big", MOVES, ids=[m[0] for m in MOVES])
+@pytest.mark.parametrize("d", [64, 128])
+def test_reference_maximum_moving_inside_a_masked_tile(name, S, N, big, d):
+    """The softmax keeps a lazy reference maximum and rescales only when the maximum grows by more than 2^8.
+    Masked key tiles are worked through in two halves of 64 keys; here one key in the SECOND half of such a
+    tile scores 2^12 above everything before it, so the reference moves after the first half has already
+    produced its probabilities: they have to move with it.  All other scores are 0, so every visible key
+    before the dominant one has weight 1 and that one 2^12.2: the output is a known mixture."""
+    parent = chain_tree(N)                          # node i sees nodes 0..i: tree key j is visible to rows >= j
+    case = _tree_case(parent, S, 2, 1, d, 384, seed=S + N)
+    case["k_cache"].zero_()
+    case["k_tree"].zero_()
+    case["q"].fill_(1.0)
+    amp = 0.75 * (128 / d) ** 0.5                   # score = d * amp / sqrt(d); 12.24 in log2 units for both head dims
+    if big < S:
+        case["k_cache"][0, 0, 0, big] = amp
+    else:
+        case["k_tree"][0, 0, big - S, 0] = amp
+    out, lse, bits, dense = gpu_attention(to_device(case))
+    ref_out, ref_lse = oracle_attention(case_to_numpy(case), dense.cpu().numpy())
+    assert_attention_close(out, lse, ref_out, ref_lse, name)
+    # the oracle's rows that see the dominant key are that key's V row up to the 2^-12 share of the others
+    cn = case_to_numpy(case)
+    vbig = orc.decode_bf16(cn["v_cache"][0][0, 0, big] if big < S else cn["v_tree"][0][0, big - S, 0])
+    rows = range(N) if big < S else range(big - S, N)
+    for i in rows:
+        assert np.abs(ref_out[0, i, 0] - vbig).max() < 0.5      # the other keys share less than 0.1 of the weight
 
 
 def test_non_ancestor_perturbation_leaves_rows_bit_identical():

@@ -8,7 +8,7 @@ import torch
 import paper_2603_08088_b200 as tv
 from oracle import tree_verify_oracle as orc
 from workloads import CONFIGS, make_case, case_to_numpy
-from gpu_util import to_device, i32, assert_attention_close
+from gpu_util import to_device, i32, assert_attention_close, oracle_visibility
 
 pytestmark = pytest.mark.gpu
 
@@ -76,9 +76,10 @@ def test_random_shape_three_layouts(seed):
     torch.cuda.synchronize()
     assert (i32(status) == 0).all(), f"{cfg}: status {i32(status)}"
     case_np = case_to_numpy(case)
+    vis = oracle_visibility(case["parent"], case["n_nodes"], dense_gpu=dense, bits_gpu=bits)   # the oracle's own mask
     ref_out, ref_lse = orc.tree_attention(case_np["q"][0], case_np["k_cache"][0], case_np["v_cache"][0],
                                           case_np["k_tree"][0], case_np["v_tree"][0], case_np["prefix_len"],
-                                          case_np["n_nodes"], i32(dense)[:, 0], scale)
+                                          case_np["n_nodes"], vis[:, 0], scale)
     assert_attention_close(outs[0][0], outs[0][1], ref_out, ref_lse, str(cfg))
     for o, l in outs[1:]:
         assert torch.equal(o.view(torch.int16), outs[0][0].view(torch.int16)) and torch.equal(l, outs[0][1]), str(cfg)

@@ -10,13 +10,14 @@ import paper_2603_08088_b200 as tv
 from paper_2603_08088_b200 import dist as tvd
 from oracle import tree_verify_oracle as orc
 from workloads import CONFIGS, make_case, case_to_numpy, bf16_bits
-from gpu_util import f32, ATTN_ATOL
+from gpu_util import f32, ATTN_ATOL, oracle_visibility
 
 pytestmark = pytest.mark.gpu
 
 
 def run_split(case, R):
-    """Returns o_parts[R,B,N,Hq,d] bf16, lse_parts[R,B,Hq,N] fp32 (device) and the dense mask (numpy)."""
+    """Returns o_parts[R,B,N,Hq,d] bf16, lse_parts[R,B,Hq,N] fp32 (device) and the oracle's dense mask of the same trees (numpy; the CUDA mask
+    is checked equal to it)."""
     L, B, N, Hq, d = case["q"].shape
     Hkv, Scap = case["k_cache"].shape[2], case["k_cache"].shape[3]
     dev = case["q"].device
@@ -44,7 +45,8 @@ def run_split(case, R):
         o_parts.append(out)
         l_parts.append(lse)
     assert (status.cpu().numpy() == 0).all()
-    return torch.stack(o_parts), torch.stack(l_parts), dense.cpu().numpy()
+    return (torch.stack(o_parts), torch.stack(l_parts),
+            oracle_visibility(case["parent"], case["n_nodes"], dense_gpu=dense, bits_gpu=bits))
 
 
 @pytest.mark.parametrize("ci,over,R", [(0, dict(B=3, S_lo=0, S_hi=300, Scap=320), 2),

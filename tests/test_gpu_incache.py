@@ -8,7 +8,7 @@ import torch
 import paper_2603_08088_b200 as tv
 from oracle import tree_verify_oracle as orc
 from workloads import CONFIGS, make_case, case_to_numpy
-from gpu_util import to_device, i32, assert_attention_close
+from gpu_util import to_device, i32, assert_attention_close, oracle_visibility
 
 pytestmark = pytest.mark.gpu
 
@@ -61,9 +61,10 @@ def test_incache_attention_matches_oracle_and_separate_buffers(name, ci, over):
     assert (i32(status) == 0).all()
     # the oracle sees the definition: separate tree buffers
     case_np = case_to_numpy(case)
+    vis = oracle_visibility(case["parent"], case["n_nodes"], dense_gpu=dense, bits_gpu=bits)    # the oracle's own mask
     ref_out, ref_lse = orc.tree_attention(case_np["q"][0], case_np["k_cache"][0], case_np["v_cache"][0],
                                           case_np["k_tree"][0], case_np["v_tree"][0], case_np["prefix_len"],
-                                          case_np["n_nodes"], i32(dense)[:, 0], d ** -0.5)
+                                          case_np["n_nodes"], vis[:, 0], d ** -0.5)
     assert_attention_close(out, lse, ref_out, ref_lse, name)
     # and the two layouts of the same kernel agree bit for bit (same tiles, same arithmetic)
     out2 = torch.zeros_like(out)

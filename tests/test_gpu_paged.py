@@ -8,7 +8,7 @@ import torch
 import paper_2603_08088_b200 as tv
 from oracle import tree_verify_oracle as orc
 from workloads import CONFIGS, make_case, case_to_numpy
-from gpu_util import to_device, i32, assert_attention_close
+from gpu_util import to_device, i32, assert_attention_close, oracle_visibility
 
 pytestmark = pytest.mark.gpu
 R = 128
@@ -74,9 +74,10 @@ def test_paged_attention_matches_oracle_and_contiguous_layout(name, ci, over):
     torch.cuda.synchronize()
     assert (i32(status) == 0).all()
     case_np = case_to_numpy(case)
+    vis = oracle_visibility(case["parent"], case["n_nodes"], dense_gpu=dense, bits_gpu=bits)    # the oracle's own mask
     ref_out, ref_lse = orc.tree_attention(case_np["q"][0], case_np["k_cache"][0], case_np["v_cache"][0],
                                           case_np["k_tree"][0], case_np["v_tree"][0], case_np["prefix_len"],
-                                          case_np["n_nodes"], i32(dense)[:, 0], d ** -0.5)
+                                          case_np["n_nodes"], vis[:, 0], d ** -0.5)
     assert_attention_close(out, lse, ref_out, ref_lse, name)
     out2, lse2 = torch.zeros_like(out), torch.zeros_like(lse)
     tv.tree_verify_attn(g["q"][0], kc.to(dev), vc.to(dev), g["k_tree"][0], g["v_tree"][0], g["prefix_len"], g["n_nodes"],

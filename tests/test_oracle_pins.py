@@ -65,6 +65,11 @@ def test_golden_hand_worked_mask_and_accept():
     assert acc["best_path"][0] == g["best_path"]
     assert acc["accepted_nodes"][0].tolist() == g["accepted_nodes"]
     assert acc["next_token"][0] == g["next_token"]
+    # accepted length of every candidate row on its own: the rule applied to a one-row table
+    toks = np.array([g["tokens"]], dtype=np.int32)
+    per_path = [int(orc.greedy_accept(mk["retrieve"][:, p:p + 1], toks, n, am)["accept_len"][0]) for p in range(3)]
+    assert per_path == g["per_path_accept"]
+    assert max(per_path) == g["accept_len"] and per_path.index(max(per_path)) == g["best_path"]
 
 
 def test_mask_equals_parent_walk_and_invariants():
