@@ -231,10 +231,10 @@ def run_ours(args, cfg):
                            buf.status, retrieve_indices=None if given_rows else buf.retrieve, n_paths=buf.n_paths)
         if marks is not None:
             marks[1].record()
-        for l in range(cfg.L):
-            tv.tree_verify_attn(case["q"][l], case["k_cache"][l], case["v_cache"][l], case["k_tree"][l],
-                                case["v_tree"][l], case["prefix_len"], case["n_nodes"], buf.anc_bits, scale,
-                                buf.out[l], buf.attn_ws, buf.status)
+        # all layers in one call; the mask kernel in front writes none of the attention's early inputs
+        tv.tree_verify_attn_layers(case["q"], case["k_cache"], case["v_cache"], case["k_tree"], case["v_tree"],
+                                   case["prefix_len"], case["n_nodes"], buf.anc_bits, scale, buf.out, buf.attn_ws,
+                                   buf.status, flags=tv.TV_ATTN_STABLE_INPUTS)
         if marks is not None:
             marks[2].record()
         if has_accept:

@@ -148,7 +148,6 @@ TV_API size_t tv_attn_workspace_bytes(int B, int Nmax, int Hq, int Hkv, int d, i
  * Limits: d in {64,128}; Nmax <= 256 (the node budgets of the paper's sweep);
  * Hq % Hkv == 0, Hq / Hkv <= 128; B <= 512; all tensors 16-byte aligned;
  * 0 <= prefix_len[b] <= Scap; scale > 0.
- * B > 192 is served by several launches over consecutive ranges of sequences.
  * CUDA graphs: every call of this header only launches on the given stream, so a
  * step can be captured into a CUDA graph and replayed; the split-KV counters in
  * the workspace are cleared by the piece that merges, so a replay (which

@@ -46,7 +46,7 @@ TV_API int tv_debug_attn_expire(const tv_bf16* q, const tv_bf16* k_cache, const 
 
 /*
  * Live only in a library built with -DTV_TRACE: while a device buffer of
- * 160 * 5 * 256 uint64 is registered here, every tree_verify_attn launch
+ * 160 * 4 * 256 uint64 is registered here, every tree_verify_attn launch
  * records a per-CTA, per-role timeline (tag << 48 | globaltimer ns) into it.
  * NULL switches it off.
  */

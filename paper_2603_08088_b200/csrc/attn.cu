@@ -6,7 +6,7 @@
 // 128/G nodes; a CTA owns MT (1 or 2) row tiles and streams 128-key tiles of
 // the committed prefix, then one tile of the tree's own keys.
 //
-// Pipeline (one CTA per SM, 16 warps):
+// Pipeline (one CTA per SM, 12 warps):
 //   warp 0      TMA producer: Q tiles once per work item, then K and V tiles
 //               through a 5-slot shared-memory ring (128-byte swizzled boxes).
 //   warp 1      tcgen05.mma issuer (one thread): S = Q K^T for a whole 128-key
@@ -18,14 +18,7 @@
 //   warps 4-7   softmax warpgroup for row tile 0: one thread per row, online
 //   warps 8-11  softmax with lazy rescale; tile 1 likewise.  The ancestor
 //               bitmask of the row is applied only on the tree tile(s), the
-//               prefix length only on the ragged last prefix tile.  At the end
-//               of an item a softmax thread leaves (m, l) of its row in shared
-//               memory and goes straight on to the next item.
-//   warps 12-15 epilogue warpgroup: takes O of a finished item out of TMEM,
-//               normalises it and stores the output rows (or, for a piece of a
-//               cut unit, the partial), releases O to the MMA issuer, and runs
-//               the merge of a cut unit - all while the other warps already
-//               work on the next item.
+//               prefix length only on the ragged last prefix tile.
 // TMEM: S0 | S1 | O0 | O1, 128 columns each; P (bf16) overlays the first 64
 // columns of its S.  With one row tile the two S buffers alternate by key tile.
 //
@@ -37,15 +30,9 @@
 // Work split.  All key tiles of all (b, hk) units form one linear space that
 // is cut evenly over the CTA groups (a group = the CTAs that hold the row
 // tiles of the same unit and walk the same keys together, so the second reader
-// hits L2).  A unit cut in pieces leaves partials (normalised O in bf16, m, l)
-// in the workspace, every piece one; each piece then bumps the unit's counter,
-// and the piece that brings it to the number of pieces merges them all (they
-// are published by then: nothing is waited for).  Counters carry a per-call
-// epoch, so the workspace needs no initialisation.  A CTA takes the pieces of
-// its range first (the end of a unit begun by the group in front, then the
-// start of the unit that the group behind finishes) and its whole units after
-// them, so that the two halves of a cut unit are done early in the launch and
-// the merge runs behind the whole units instead of at the end of the kernel.
+// hits L2).  A unit cut in pieces leaves partials (normalised O in bf16, m, l) in the
+// workspace; the piece that draws the last ticket on the unit's counter merges them.
+// Counters carry a per-call epoch, so the workspace needs no initialisation.
 //
 // Every wait on an mbarrier is bounded: on expiry the CTA raises
 // TV_ST_TIMEOUT for all sequences, all roles leave their loops, outstanding
@@ -64,9 +51,8 @@ namespace {
 constexpr int kTileN = 128;        // keys per tile
 constexpr int kTileM = 128;        // rows per row tile
 constexpr int kSlots = 5;          // K/V ring slots
-constexpr int kThreads = 512;
-constexpr int kEpiThread0 = 384;   // first thread of the epilogue warpgroup
-constexpr int kMaxB = 192;         // sequences per launch: the schedule table lives in shared memory (larger batches are launched in parts)
+constexpr int kThreads = 384;
+constexpr int kMaxB = 512;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kRescaleThreshold = 8.0f;            // in log2 units
 constexpr float kMaxFastSum = 16384.0f;               // 64 keys x 2^threshold: largest row sum the fast path accepts
@@ -77,7 +63,8 @@ constexpr float kMaxFastSum = 16384.0f;               // 64 keys x 2^threshold: 
 #define TV_POLY_SEL(i) ((((i) & 7) == 3) || (((i) & 15) == 7))
 #endif
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
-// virtual tiles charged per unit by the scheduler
+// virtual tiles charged per unit by the scheduler (32-layer shape, five seeds: 2 is 0.2-2 % faster than 4,
+// 0 and 1 are slower)
 #ifndef TV_SETUP_COST
 #define TV_SETUP_COST 2
 #endif
@@ -89,27 +76,6 @@ constexpr int kMaxGroups = 160;
 #define TV_MIN_VT 6
 #endif
 constexpr int kMinVirtualTilesPerGroup = TV_MIN_VT;
-// pieces of cut units first, whole units after them (0: the items of a range in their natural order)
-#ifndef TV_PIECES_FIRST
-#define TV_PIECES_FIRST 1
-#endif
-// register budget per thread after the split (setmaxnreg): producer / MMA warpgroup, softmax warpgroups, epilogue
-// warpgroup.  The CTA starts with 128 registers per thread (512 threads); 4 * kRegsLow + 8 * kRegsSoftmax +
-// 4 * kRegsEpi must not exceed 2048, or the increase never completes.
-#ifndef TV_REGS_LOW
-#define TV_REGS_LOW 48
-#endif
-#ifndef TV_REGS_SOFTMAX
-#define TV_REGS_SOFTMAX 192
-#endif
-#ifndef TV_REGS_EPI
-#define TV_REGS_EPI 80
-#endif
-static_assert(4 * TV_REGS_LOW + 8 * TV_REGS_SOFTMAX + 4 * TV_REGS_EPI <= 2048, "register split exceeds the register file");
-static_assert(TV_REGS_LOW % 8 == 0 && TV_REGS_SOFTMAX % 8 == 0 && TV_REGS_EPI % 8 == 0, "setmaxnreg takes multiples of 8");
-#define TV_STR2(x) #x
-#define TV_STR(x) TV_STR2(x)
-constexpr int kTraceRoles = 5;     // producer, MMA issuer, softmax 0, softmax 1, epilogue
 constexpr int kTraceCap = 256;     // events per (CTA, role) kept by the optional trace
 
 // ---------------------------------------------------------------- PTX helpers
@@ -277,7 +243,7 @@ struct Tracer {
   unsigned long long* base;
   int n;
   __device__ __forceinline__ void init(unsigned long long* trace, int role) {
-    base = trace ? trace + ((size_t)blockIdx.x * kTraceRoles + role) * kTraceCap : nullptr;
+    base = trace ? trace + ((size_t)blockIdx.x * 4 + role) * kTraceCap : nullptr;
     n = 0;
   }
   __device__ __forceinline__ void mark(uint32_t tag) {
@@ -345,12 +311,12 @@ struct AttnParams {
   int32_t* status;
   tv_bf16* part_o;               // [slots][D/8][MT*128][8] bf16 normalised outputs, column-group major
   float* part_ml;                // [slots][2][MT*128]  (m in log2 units, then l)
-  unsigned long long* counters;  // [B*Hkv*NP]: pieces of the unit that have published (epoch-tagged)
+  unsigned long long* counters;  // [B*Hkv*NP][2]: tickets claimed, partials ready (epoch-tagged)
   unsigned long long epoch;      // 48-bit tag of this call
   int B, Nmax, Hq, Hkv, Scap, G, NPT, NP, W, groups;
   int TT;                        // key tiles of the tree's own K/V: ceil(Nmax / 128), 1 or 2
-  uint32_t q_box_bytes;          // bytes of one Q box {64, G, NPT}: 16 KB when G divides 128
-  unsigned long long* trace;     // optional event trace [cta][role][kTraceCap] of (tag << 48 | ns), or NULL
+  uint32_t q_box_bytes;
+  unsigned long long* trace;     // optional event trace [cta][role 0..3][kTraceCap] of (tag << 48 | ns), or NULL          // bytes of one Q box {64, G, NPT}: 16 KB when G divides 128
   int tree_in_cache;             // the tree's K/V rows live in the cache behind the prefix (rows S_b + node)
   const int32_t* block_table;    // paged cache: page of key tile j of sequence b at [b * max_blocks + j]; else nullptr
   int max_blocks, n_pages;
@@ -367,21 +333,17 @@ struct Item {
   int b, hk, j0, j1, len, S, n;
 };
 
-// Shared bookkeeping of the linear tile space: cum[b] = sum over b' < b of (len_b' + kSetupCost), len_b =
-// ceil(S_b/128) + TT.  The schedule works in a "virtual" tile space: every (sequence, KV head) unit is charged
-// kSetupCost virtual tiles in front of its real key tiles, the price of starting a unit (Q load, pipeline
-// refill).  Cutting that space evenly gives CTAs that start more units fewer real tiles, and a cut that falls
-// into a unit's setup region snaps to the unit boundary, which saves a split.
+// Shared bookkeeping of the linear tile space: cum[b] = sum of len over b' < b, len_b = ceil(S_b/128) + 1.
+// The schedule works in a "virtual" tile space: every (sequence, KV head) unit is charged kSetupCost
+// virtual tiles in front of its real key tiles, the price of starting a unit (Q load, pipeline refill,
+// epilogue).  Cutting that space evenly gives CTAs that start more units fewer real tiles, and a cut that
+// falls into a unit's setup region snaps to the unit boundary, which saves a split.
 struct Sched {
-  const int* cum;
+  const int* cum;    // cum[b] = sum over b' < b of (len_b' + kSetupCost)
+  const int* gs;     // gs[k] = first virtual tile of CTA group k, gs[groups] = total
   int B, Hkv;
   int total;         // Hkv * cum[B]; the host refuses problems whose tile count does not fit 31 bits
-  int groups;        // CTA groups in use
-  unsigned q, r;     // total = q * groups + r
-  // first virtual tile of CTA group k: floor(total * k / groups) in 32-bit arithmetic
-  __device__ __forceinline__ int group_start(int k) const {
-    return k < groups ? (int)((unsigned)k * q + ((unsigned)k * r) / (unsigned)groups) : total;
-  }
+  __device__ __forceinline__ int group_start(int k, int) const { return gs[k]; }
   __device__ __forceinline__ int find_b(int g) const {
     int lo = 0, hi = B - 1;   // largest b with Hkv*cum[b] <= g
     while (lo < hi) {
@@ -401,13 +363,12 @@ struct SmemLayout {
   static constexpr int kBars = kRing + kSlots * kTileBytes;
   // barrier indices (8 bytes each)
   static constexpr int Q_FULL = 0, Q_EMPTY = 1, KV_FULL = 2, KV_EMPTY = 2 + kSlots, S_FULL = 2 + 2 * kSlots,
-                       P_READY = S_FULL + 2, O_DONE = P_READY + 2, ITEM_DONE = O_DONE + 2, ML_READY = ITEM_DONE + 2,
-                       ML_FREE = ML_READY + 2, O_FREE = ML_FREE + 2, EPI = O_FREE + 2, NBARS = EPI + 1;
+                       P_READY = S_FULL + 2, O_DONE = P_READY + 2, ITEM_DONE = O_DONE + 2, EPI = ITEM_DONE + 2,
+                       NBARS = EPI + 1;
   static constexpr int kMisc = kBars + NBARS * 8;          // tmem ptr, abort flag, last flag
-  static constexpr int kHand = kMisc + 16;                 // (m, l) of every row, softmax -> epilogue
-  static constexpr int kCum = kHand + MT * 128 * 8;
-  static constexpr int kTotal = kCum + (kMaxB + 1) * 4;
-  static_assert(kTotal <= 232448, "shared memory of the attention kernel exceeds 227 KB");
+  static constexpr int kCum = kMisc + 16;
+  static constexpr int kGs = kCum + (kMaxB + 1) * 4;
+  static constexpr int kTotal = kGs + (kMaxGroups + 1) * 4;
 };
 
 // ---------------------------------------------------------------- the kernel
@@ -425,45 +386,17 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::kMisc + 4);
   volatile int* last_flag = reinterpret_cast<volatile int*>(smem + L::kMisc + 8);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + L::kMisc);
-  float2* hand = reinterpret_cast<float2*>(smem + L::kHand);
   int* cum = reinterpret_cast<int*>(smem + L::kCum);
+  int* gs = reinterpret_cast<int*>(smem + L::kGs);
   const unsigned long long wait_limit = prm.wait_limit_ns;
 
-  // ---- setup: barriers, TMEM, schedule table
+  // ---- setup: schedule table, barriers, TMEM
   if (threadIdx.x == 64) {     // fetch the five TMA descriptors while the rest of the set-up runs
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_q) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_kc) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_vc) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_kt) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_vt) : "memory");
-  }
-  if (threadIdx.x == 32) {
-    mbar_init(bar(L::Q_FULL), 1);
-    mbar_init(bar(L::Q_EMPTY), 1);
-#pragma unroll 1
-    for (int s = 0; s < kSlots; ++s) {
-      mbar_init(bar(L::KV_FULL + s), 1);
-      mbar_init(bar(L::KV_EMPTY + s), 1);
-    }
-#pragma unroll 1
-    for (int s = 0; s < 2; ++s) {                // index = S buffer / row tile
-      mbar_init(bar(L::S_FULL + s), 1);
-      mbar_init(bar(L::P_READY + s), 128);
-      mbar_init(bar(L::O_DONE + s), 1);
-      mbar_init(bar(L::ITEM_DONE + s), 1);
-      mbar_init(bar(L::ML_READY + s), 128);
-      mbar_init(bar(L::ML_FREE + s), 128);
-      mbar_init(bar(L::O_FREE + s), 128);
-    }
-    mbar_init(bar(L::EPI), 128);
-    *abort_flag = ((sbase & 1023u) != 0) ? 1 : 0;   // swizzled tiles need a 1024-byte aligned base
-    *last_flag = 0;
-    fence_barrier_init();
-  }
-  if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32((const void*)tmem_slot))
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   // Without the caller's promise nothing of the problem is read before every earlier kernel of the stream has
   // finished (a kernel in front may still be writing prefix_len, and lines of it cached by an earlier launch on
@@ -491,17 +424,43 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     }
     if (lane == 0) cum[prm.B] = run;
   }
+  if (threadIdx.x == 32) {
+    mbar_init(bar(L::Q_FULL), 1);
+    mbar_init(bar(L::Q_EMPTY), 1);
+#pragma unroll 1
+    for (int s = 0; s < kSlots; ++s) {
+      mbar_init(bar(L::KV_FULL + s), 1);
+      mbar_init(bar(L::KV_EMPTY + s), 1);
+    }
+    for (int s = 0; s < 2; ++s) {                // index = S buffer
+      mbar_init(bar(L::S_FULL + s), 1);
+      mbar_init(bar(L::P_READY + s), 128);
+    }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(bar(L::O_DONE + s), 1);
+      mbar_init(bar(L::ITEM_DONE + s), 1);
+    }
+    mbar_init(bar(L::EPI), MT * 128);
+    *abort_flag = ((sbase & 1023u) != 0) ? 1 : 0;   // swizzled tiles need a 1024-byte aligned base
+    *last_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32((const void*)tmem_slot))
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   // Small problems use fewer CTA groups, so that a unit is cut into few pieces (each piece costs a partial
-  // write and a share of a merge) and every group still gets a worthwhile share of tiles.
-  Sched sch{cum, prm.B, prm.Hkv, prm.Hkv * cum[prm.B], 1, 0u, 0u};
+  // write and a merge) and every group still gets a worthwhile share of tiles.
+  int groups;
   {
-    const unsigned total = (unsigned)sch.total;
+    const unsigned total = (unsigned)(prm.Hkv * cum[prm.B]);
     const unsigned want = total / (unsigned)kMinVirtualTilesPerGroup;
-    int groups = want < 1u ? 1 : (want < (unsigned)prm.groups ? (int)want : prm.groups);
+    groups = want < 1u ? 1 : (want < (unsigned)prm.groups ? (int)want : prm.groups);
     // A group count just above a multiple of the unit count is rounded down to it: with units of equal length
     // (one sequence, all heads) every unit is then cut into the same number of equal pieces and no cut falls
     // just behind a unit boundary.  Not worth more than 1/16 of the groups.
@@ -509,25 +468,29 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       const int units = prm.B * prm.Hkv, over = groups % units;
       if (groups > units && over * 16 <= groups) groups -= over;
     }
-    sch.groups = groups;
-    sch.q = total / (unsigned)groups;
-    sch.r = total % (unsigned)groups;
+    // gs[k] = floor(total * k / groups) in 32-bit arithmetic: total = q * groups + r
+    const unsigned q = total / (unsigned)groups, r = total % (unsigned)groups;
+#pragma unroll 1
+    for (int k = threadIdx.x; k <= prm.groups; k += kThreads)
+      gs[k] = k <= groups ? (int)(k * q + (k * r) / (unsigned)groups) : (int)total;
   }
+  __syncthreads();
+
+  Sched sch{cum, gs, prm.B, prm.Hkv, prm.Hkv * cum[prm.B]};
   const int group = blockIdx.x / prm.NP;
   const int pair = blockIdx.x % prm.NP;
-  const int g_begin = sch.group_start(group);        // groups past the last used one get an empty range
-  const int g_end = sch.group_start(group + 1);
+  const int g_begin = sch.group_start(group, groups);        // groups past the last used one get an empty range
+  const int g_end = sch.group_start(group + 1, groups);
 
-  // ---- the items of this CTA's range, in the order every role takes them.
-  // walk(): the next item of [g, limit) in the natural order of the tile space.
-  auto walk = [&](int& g, int limit, Item& it) -> bool {
-    while (g < limit) {
+  // Walks the items of this CTA's range; identical in every role.
+  auto next_item = [&](int& g, Item& it) -> bool {
+    while (g < g_end) {
       const int b = sch.find_b(g);
       const int lenv = cum[b + 1] - cum[b];                       // setup region + real tiles
       const unsigned local = (unsigned)(g - prm.Hkv * cum[b]);
       const int hk = (int)(local / (unsigned)lenv);
       const int r0 = (int)(local - (unsigned)hk * (unsigned)lenv);
-      const int room = limit - g;
+      const int room = g_end - g;
       const int r1 = (lenv - r0) < room ? lenv : r0 + room;
       g += r1 - r0;
       const int j0 = r0 > kSetupCost ? r0 - kSetupCost : 0;
@@ -546,45 +509,6 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     }
     return false;
   };
-  // Order: the first item of the range, then - if the range ends inside a unit that the next group finishes (the
-  // start of a cut unit) - that piece, then everything in between.  walk_state: {g, end of the middle part, start
-  // of the piece at the end or -1, phase}.
-  struct Walk {
-    int g, mid_end, tail_g0, phase;
-  };
-  auto walk_init = [&]() -> Walk {
-    Walk w{g_begin, g_end, -1, 0};
-#if TV_PIECES_FIRST
-    if (g_end > g_begin) {
-      const int gl = g_end - 1;
-      const int b = sch.find_b(gl);
-      const int lenv = cum[b + 1] - cum[b];
-      const unsigned local = (unsigned)(gl - prm.Hkv * cum[b]);
-      const int r = (int)(local % (unsigned)lenv);                // place of the range's last virtual tile in its unit
-      const int ustart = gl - r;
-      // the unit goes on behind the range, real tiles of it lie inside, and it is not the range's first item
-      if (r + 1 < lenv && r + 1 > kSetupCost && ustart > g_begin) {
-        w.mid_end = ustart;
-        w.tail_g0 = ustart;
-      }
-    }
-#endif
-    return w;
-  };
-  auto next_item = [&](Walk& w, Item& it) -> bool {
-    if (w.phase == 0) {
-      w.phase = 1;
-      if (walk(w.g, w.mid_end, it)) return true;
-    }
-    if (w.phase == 1) {
-      w.phase = 2;
-      if (w.tail_g0 >= 0) {
-        int g2 = w.tail_g0;
-        if (walk(g2, g_end, it)) return true;
-      }
-    }
-    return walk(w.g, w.mid_end, it);
-  };
 
   constexpr uint32_t kIdescQK = instr_desc(kTileN, false);
   constexpr uint32_t kIdescPV = instr_desc(D, true);
@@ -592,9 +516,9 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 
   if (warp == 0) {
     // =========================================================== TMA producer
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 " TV_STR(TV_REGS_LOW) ";");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
     if (!*abort_flag && !(prm.debug & 1)) {        // the whole warp walks the items; one elected lane issues the copies
-      Walk wk = walk_init();
+      int g = g_begin;
       Item it;
       uint32_t item_idx = 0, fill = 0;
       bool ok = true;
@@ -603,11 +527,13 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       tr.mark(0);
       uint64_t kv_policy;      // the committed prefix is streamed once: first in line for eviction from L2
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(kv_policy));
-      // Overlap with the kernel in front (programmatic dependent launch).  With the caller's promise (prm.early)
+      // Overlap with the kernel in front (programmatic dependent launch): the committed prefix, prefix_len and
+      // n_nodes are not written by a tree_verify_attn call, the one kernel that lets this one start early, so
       // the first prefix tiles are requested at once; Q and the tree's K/V - what a preceding kernel may still
       // be producing - wait for that kernel to finish.  Only then may the next kernel be scheduled, so that at
-      // most two launches are in flight.  status[] may still be written by the kernel in front
-      // (tree_build_mask stores it last), so a flag found before the wait is kept and raised after it.
+      // most two launches are in flight and the two halves of the workspace suffice.
+      // status[] may still be written by the kernel in front (tree_build_mask stores it last), so a flag found
+      // before the wait is kept here and raised after it.
       bool synced = false;
       int bad_page_b = -1;
       auto sync_with_predecessor = [&]() {
@@ -631,7 +557,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         __syncwarp();
       };
       if (!prm.early) sync_with_predecessor();
-      while (ok && next_item(wk, it)) {
+      while (ok && next_item(g, it)) {
         ok = mbar_wait(bar(L::Q_EMPTY), (item_idx & 1) ^ 1, abort_flag, wait_limit);
         if (!ok) break;
         tr.mark(0x1000u | item_idx);
@@ -706,11 +632,9 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     //   two row tiles (buffer = row tile):  wait P_t -> O_t += P_t V -> S_t = Q_t K_next^T, t = 0, 1 in turn, so
     //     that the softmax of one row tile runs while the pipe works for the other one;
     //   one row tile (buffers alternate by key tile):  S_next = Q K_next^T -> wait P -> O += P V.
-    // The first PV of an item overwrites O: it waits until the epilogue warpgroup has taken the previous item's
-    // O out of TMEM.
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 " TV_STR(TV_REGS_LOW) ";");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
     if (!*abort_flag) {      // the whole warp walks the items; one elected lane issues
-      Walk wk = walk_init();
+      int g = g_begin;
       Item it;
       uint32_t item_idx = 0, fill = 0, tj = 0;
       bool ok = true;
@@ -750,7 +674,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
         __syncwarp();
       };
-      while (ok && next_item(wk, it)) {
+      while (ok && next_item(g, it)) {
         const int nt = it.j1 - it.j0;
         ok = mbar_wait(bar(L::Q_FULL), item_idx & 1, abort_flag, wait_limit);
         if (!ok) break;
@@ -783,10 +707,6 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 if (ok && more) ok = mbar_wait(bar(L::KV_FULL + kslot), (fk / kSlots) & 1, abort_flag, wait_limit);
                 if (!ok) break;
               }
-              if (jt == 0 && item_idx > 0) {          // O_t of the previous item must have left TMEM
-                ok = mbar_wait(bar(L::O_FREE + t), (item_idx - 1) & 1, abort_flag, wait_limit);
-                if (!ok) break;
-              }
               tc_fence_after();
               tr.mark(0x4000u | ((2 * tj + t) & 0xfffu));
               issue_pv(t, t, vslot, jt == 0);
@@ -805,7 +725,6 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             }
             ok = mbar_wait(bar(L::P_READY + buf), (tj >> 1) & 1, abort_flag, wait_limit);
             if (ok) ok = mbar_wait(bar(L::KV_FULL + vslot), (fv / kSlots) & 1, abort_flag, wait_limit);
-            if (ok && jt == 0 && item_idx > 0) ok = mbar_wait(bar(L::O_FREE), (item_idx - 1) & 1, abort_flag, wait_limit);
             if (!ok) break;
             tc_fence_after();
             tr.mark(0x4000u | (tj & 0xfffu));
@@ -824,45 +743,64 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         ++item_idx;
       }
     }
-  } else if (warp >= 4 && warp < 12) {
-    // =========================================================== softmax warpgroups
-    // Register budget: the CTA starts with 128 registers per thread; warps 0-3 and 12-15 give registers up and
-    // warps 4-11 take them.  The increase below can only complete once the others have released enough, so the
-    // three values have to satisfy the static_assert beside their definition or the kernel never gets past this
-    // instruction.
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 " TV_STR(TV_REGS_SOFTMAX) ";");
+  } else if (warp >= 4) {
+    // =========================================================== softmax / epilogue warpgroups
+    // Register budget: the CTA starts with 168 registers per thread; warps 0-3 give up 96 each (168 -> 72) and
+    // warps 4-11 take 48 each (168 -> 216).  4 x 96 = 8 x 48: the increase below can only complete once the
+    // other warpgroup has released enough, so any other split has to keep 4 (168 - low) >= 8 (high - 168) or the
+    // kernel never gets past this instruction.
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
     const int wg = (warp - 4) >> 2;                  // row tile of this warpgroup
     const int row = ((warp & 3) << 5) | lane;        // TMEM lane = row inside the tile
     const uint32_t lane_addr = (uint32_t)((warp & 3) << 5) << 16;
     const bool wg_active = wg < MT;
-    gdc_wait();      // anc_bits may belong to the kernel in front until it is done
+    gdc_wait();      // anc_bits, the workspace and the outputs may belong to the kernel in front until it is done
+    // in-cache layout: a tree that does not fit behind its prefix is reported, not read past the capacity (rows
+    // past Scap arrive as zeros and the sequence's output is unspecified).  Raised after the wait: status[] may
+    // be written by the kernel in front until then.
+    if (prm.tree_in_cache && blockIdx.x == 0)
+#pragma unroll 1
+      for (int b = threadIdx.x - 128; b < prm.B; b += kThreads - 128) {
+        int S = prm.prefix_len[b];
+        S = S < 0 ? 0 : (S > prm.Scap ? prm.Scap : S);
+        if (S + prm.n_nodes[b] > prm.Scap) atomicOr(prm.status + b, TV_ST_CAPACITY);
+      }
     if (wg_active && !*abort_flag) {
-      Walk wk = walk_init();
+      int g = g_begin;
       Item it;
-      uint32_t fill = 0, tj = 0, item_cnt = 0;   // tj: key tiles handled so far (all items)
+      uint32_t fill = 0, tj = 0, epi_phase = 0, item_cnt = 0;   // tj: key tiles handled so far (all items)
       bool ok = true;
       Tracer tr;
       tr.init((threadIdx.x & 127) == 0 ? prm.trace : nullptr, 2 + wg);
       tr.mark(0);
 #ifdef TV_PROF
       unsigned int prof[12] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u}, pc0 = 0, pc1 = 0, pc2 = 0, pend = 0;
-      // 0 wait S, 1 ld, 2 compute, 3 hand-over, 4 tiles, 5 between tiles, 6 start -> first S, 7 wait for the
-      // hand-over slot, 9 items, 10 first tile of an item: from item start to its S
+      // 0 wait S, 1 ld, 2 compute, 3 hand-over, 4 tiles, 5 between tiles, 6 start -> first S, 7 wait ITEM_DONE,
+      // 8 epilogue (whole or piece), 9 items, 10 first tile of an item: from item start to its S
       const unsigned int prof_start = clock();
       const long long prof_c0 = clock64();
-      const unsigned long long prof_g0 = globaltimer_ns();
+      const unsigned long long prof_g0 = globaltimer_ns();   // cycles: wait S, ld, compute, hand-over; tiles
 #endif
+      // Rendezvous of the softmax warpgroups through an mbarrier, so that it is bounded like every other wait.
       // All 32 lanes wait together and agree on the outcome, so that the warp-wide TMEM instructions
       // below are never executed by a part of a warp.
       auto wwait = [&](uint32_t b_, uint32_t parity) -> bool {
         return __all_sync(0xffffffffu, mbar_wait(b_, parity, abort_flag, wait_limit));
       };
-      while (ok && next_item(wk, it)) {
+      auto epi_sync = [&]() -> bool {
+        mbar_arrive(bar(L::EPI));
+        const bool r = wwait(bar(L::EPI), epi_phase & 1);
+        ++epi_phase;
+        return r;
+      };
+      while (ok && next_item(g, it)) {
 #ifdef TV_PROF
         const unsigned int pitem = clock();
+        unsigned int ep[6], ep_kind = 0, ep_others = 0, ep_own = 0;
 #endif
         const int nt = it.j1 - it.j0;
         const int node = (pair * MT + wg) * prm.NPT + row / prm.G;
+        const int gm = row % prm.G;
         const bool row_exists = row < prm.NPT * prm.G && node < prm.Nmax;
         const bool row_active = row_exists && node < it.n;
         uint32_t anc[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
@@ -873,6 +811,14 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
         float m_used = -INFINITY;      // running reference maximum, in log2 units (score * scale * log2e)
         float l_sum = 0.f;
+        // A piece of a cut unit draws its ticket early (thread 128 only): the counter is read at the start of
+        // the item and the compare-and-swap is issued when the last key tile begins, so that both round trips
+        // are hidden behind the softmax of that tile; the outcome is looked at in the epilogue.
+        const bool piece = !(it.j0 == 0 && it.j1 == it.len);
+        unsigned long long* claim_ctr = prm.counters + (((size_t)it.b * prm.Hkv + it.hk) * prm.NP + pair) * 2;
+        unsigned long long claim_assumed = 0, claim_ret = 1;
+        int claim_cnt = 0;
+        if (piece && threadIdx.x == 128) claim_assumed = *reinterpret_cast<volatile unsigned long long*>(claim_ctr);
         const uint32_t o_addr_loop = tmem + lane_addr + kTmemO0 + wg * 128;
         // key tiles below this index are full tiles of the committed prefix (no mask of any kind)
         const int j_full = min(it.S / kTileN, it.len - prm.TT);
@@ -885,6 +831,10 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             valid_keys = tt >= 0 ? max(0, min(kTileN, it.n - tt * kTileN)) : min(kTileN, it.S - j * kTileN);
           }
           const bool tree = tt >= 0;
+          if (piece && threadIdx.x == 128 && jt == nt - 1) {
+            claim_cnt = ((claim_assumed >> 16) == prm.epoch) ? (int)(claim_assumed & 0xffffu) : 0;
+            claim_ret = atomicCAS(claim_ctr, claim_assumed, (prm.epoch << 16) | (unsigned long long)(claim_cnt + 1));
+          }
           // ---- V rows past the valid keys may hold anything (stale cache rows, padded tree slots): zero
           // them so that 0 * NaN never reaches O.  Idempotent, so both warpgroups may do it.  Rows that lie
           // outside the tensor arrive as zeros from the copy itself: a tree tile whose tree is full (the
@@ -1101,23 +1051,282 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           tr.mark(0x2000u | (tj & 0xfffu));
         }
         if (!ok) break;
-        // ---- hand (m, l) of the row to the epilogue warpgroup (which waits for the item's last PV, normalises
-        // and stores) and go on with the next item at once.  The slot is free once the epilogue has read the
-        // previous item's pair.
-        TV_PROF_T(pc0);
-        if (item_cnt > 0) {
-          ok = wwait(bar(L::ML_FREE + wg), (item_cnt - 1) & 1);
+        // ---- epilogue of the item: wait for the last PV into this O buffer
+        {
+          // Wait for every MMA of the item.  This barrier completes once per item, so its phase is never
+          // more than one away from the one waited for (a parity wait cannot tell phases two apart, which
+          // is why the per-PV barrier O_DONE is not used here: both last PVs may or may not be done yet).
+          TV_PROF_T(pc0);
+          ok = wwait(bar(L::ITEM_DONE + wg), item_cnt & 1);
+          ++item_cnt;
           if (!ok) break;
-        }
-        hand[wg * 128 + row] = make_float2(row_active ? m_used : -INFINITY, row_active ? l_sum : 0.f);
-        mbar_arrive(bar(L::ML_READY + wg));
-        ++item_cnt;
-        TV_PROF_T(pc1);
+          tc_fence_after();
+          TV_PROF_T(pc1);
 #ifdef TV_PROF
-        prof[7] += pc1 - pc0;
+          prof[7] += pc1 - pc0;
+#endif
+          tr.mark(0x5000u);
+#ifdef TV_PROF
+          for (int i = 0; i < 6; ++i) ep[i] = pc1;
+#endif
+          const uint32_t o_addr = o_addr_loop;
+          const bool whole = (it.j0 == 0 && it.j1 == it.len);
+          const int h = it.hk * prm.G + gm;
+          tv_bf16* orow = prm.out + (((size_t)it.b * prm.Nmax + node) * prm.Hq + h) * D;
+          float* lse_p = prm.lse ? prm.lse + ((size_t)it.b * prm.Hq + h) * prm.Nmax + node : nullptr;
+          // Normalised bf16 output of this row, 32 columns at a time (one copy of the loop for every use: the
+          // epilogue is cold code, fetched while the other CTAs still stream K/V).
+          auto store_rows = [&](uint4* dst, size_t stride_u4, float inv, bool do_store, bool zero) {
+#pragma unroll 1
+            for (int q = 0; q < D / 32; ++q) {
+              uint32_t o[32];
+              tmem_ld32(o_addr + q * 32, o);
+              tmem_wait_ld();
+              if (do_store) {
+                uint4 v[4];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                  v[c].x = pack_bf16(__uint_as_float(o[8 * c + 0]) * inv, __uint_as_float(o[8 * c + 1]) * inv);
+                  v[c].y = pack_bf16(__uint_as_float(o[8 * c + 2]) * inv, __uint_as_float(o[8 * c + 3]) * inv);
+                  v[c].z = pack_bf16(__uint_as_float(o[8 * c + 4]) * inv, __uint_as_float(o[8 * c + 5]) * inv);
+                  v[c].w = pack_bf16(__uint_as_float(o[8 * c + 6]) * inv, __uint_as_float(o[8 * c + 7]) * inv);
+                  if (zero) v[c] = make_uint4(0, 0, 0, 0);       // rows of padded nodes: O may hold anything
+                }
+                if (stride_u4 == 1 && prm.out_al32) {     // a row of the output: whole 32-byte sectors per store
+                  st_global_32B(dst + q * 4, v[0], v[1]);
+                  st_global_32B(dst + q * 4 + 2, v[2], v[3]);
+                } else {
+#pragma unroll
+                  for (int c = 0; c < 4; ++c) dst[(size_t)(q * 4 + c) * stride_u4] = v[c];
+                }
+              }
+            }
+          };
+          if (whole) {
+            const float inv = (row_active && l_sum > 0.f) ? 1.f / l_sum : 0.f;
+            store_rows(reinterpret_cast<uint4*>(orow), 1, inv, row_exists, !row_active);
+            if (row_exists && lse_p)
+              *lse_p = (row_active && l_sum > 0.f) ? (m_used + log2f(l_sum)) / kLog2e : -INFINITY;
+            tc_fence_before();
+          } else {
+            // ---- a piece of a unit.  The pieces of a unit draw tickets on the unit's "claimed" counter (the
+            // draw was started while the last key tile was still being processed): the piece with the last
+            // ticket becomes the merger and keeps its O in TMEM; every other piece leaves its normalised
+            // output O/l (bf16) and (m, l) in its CTA's slot and then bumps the unit's "ready" counter.  The
+            // merger waits (bounded) until all other pieces are ready - they hold tickets, so they are in
+            // their epilogue - and combines out = sum_p w_p O_p / sum_p w_p with w_p = l_p 2^(m_p - max m).
+            // Every piece enters the sum as its bf16-rounded normalised output, the merger's own included,
+            // and the sum runs in piece order with one fused multiply-add per piece, so the result does not
+            // depend on which piece merges.  Both counters carry the call's epoch: no initialisation needed.
+            // Partial outputs are stored column-group major, [slot][D/8][MT*128 rows][8 bf16]: a warp writes
+            // and reads 512 contiguous bytes per instruction.
+            constexpr int kRows = MT * 128;
+            const int rr = wg * 128 + row;
+            // The unit's real tiles occupy [real0, uend) of the virtual tile space.  CTA groups k_first..k_last
+            // hold them, one piece each (a group between the two lies wholly inside the unit), and this CTA's
+            // group is one of them: two short walks over the cut table find both ends.
+            const int real0 = prm.Hkv * cum[it.b] + it.hk * (it.len + kSetupCost) + kSetupCost;
+            const int uend = real0 + it.len;
+            int k_first = group, k_last = group;
+            while (gs[k_first] > real0) --k_first;
+            while (gs[k_last + 1] < uend) ++k_last;
+            const int n_frag = k_last - k_first + 1;
+            // slot of the piece CTA group k holds: slot 1 of its CTA if the unit starts in that group, else slot 0
+            auto piece_slot = [&](int k) -> int { return (k * prm.NP + pair) * 2 + (k == k_first ? 1 : 0); };
+            const int my_slot = piece_slot(group);
+            unsigned long long* ctr = prm.counters + (((size_t)it.b * prm.Hkv + it.hk) * prm.NP + pair) * 2;
+            TV_PROF_T(ep[1]);
+            if (threadIdx.x == 128) {
+              int ticket;
+              if (claim_ret == claim_assumed) {
+                ticket = claim_cnt + 1;                      // the early draw went through
+              } else {
+                ticket = bump_counter(ctr, claim_ret, prm.epoch);
+              }
+              const int merger = (ticket == n_frag) ? 1 : 0;
+              if (merger) {
+                // wait until the other n_frag - 1 pieces have published their partials
+                const unsigned long long t0 = globaltimer_ns();
+                while (true) {
+                  const unsigned long long v = *reinterpret_cast<volatile unsigned long long*>(ctr + 1);
+                  const int ready = ((v >> 16) == prm.epoch) ? (int)(v & 0xffffu) : 0;
+                  if (ready >= n_frag - 1) break;
+                  if (*abort_flag || globaltimer_ns() - t0 > wait_limit) {
+                    *abort_flag = 1;
+                    break;
+                  }
+                }
+                __threadfence();
+                // every piece has drawn its ticket and published: nobody touches the two counters again in
+                // this launch.  Clearing them lets the same launch be replayed with the same epoch (a captured
+                // CUDA graph) and find them unused.
+                *reinterpret_cast<volatile unsigned long long*>(ctr) = 0ull;
+                *reinterpret_cast<volatile unsigned long long*>(ctr + 1) = 0ull;
+              }
+              *last_flag = merger;
+            }
+            ok = epi_sync();
+            if (!ok || *abort_flag) { ok = false; break; }
+            tr.mark(0x7000u | (*last_flag ? 1u : 0u));
+            TV_PROF_T(ep[2]);
+#ifdef TV_PROF
+            ep_kind = (*last_flag ? 2u : 1u) | ((unsigned)n_frag << 4);
+#endif
+            const float inv_own = (row_active && l_sum > 0.f) ? 1.f / l_sum : 0.f;
+            if (!*last_flag) {
+              uint4* po = reinterpret_cast<uint4*>(prm.part_o) + (size_t)my_slot * (D / 8) * kRows;
+              float* pml = prm.part_ml + (size_t)my_slot * 2 * kRows;
+              store_rows(po + rr, kRows, inv_own, row_active, false);
+              if (row_active) {
+                pml[rr] = m_used;
+                pml[kRows + rr] = l_sum;
+              }
+              tc_fence_before();
+              TV_PROF_T(ep[3]);
+              __threadfence();
+              TV_PROF_T(ep[4]);
+              tr.mark(0x6000u);
+              ok = epi_sync();
+              if (!ok) break;
+              TV_PROF_T(ep[5]);
+              if (threadIdx.x == 128) {
+                const unsigned long long seen = *reinterpret_cast<volatile unsigned long long*>(ctr + 1);
+                bump_counter(ctr + 1, seen, prm.epoch);
+              }
+            } else {
+              // ---- pass 1: reference maximum and total weight of the row.  (m, l) of the first four pieces
+              // are fetched together (one round trip; a unit rarely has more), the rest one by one.  Loads are
+              // issued by every thread (row rr always lies inside a slot; rows that are not active read stale
+              // bytes and are masked by selects): no thread-divergent branch sits between the warp-wide TMEM ops.
+              float pm[4], w4[4];
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const int k = k_first + i;
+                const bool other = k <= k_last && k != group;
+                const float* q_ml = prm.part_ml + (size_t)piece_slot(other ? k : group) * 2 * kRows;
+                const float m_k = __ldcg(q_ml + rr), l_k = __ldcg(q_ml + kRows + rr);
+                pm[i] = other ? m_k : (k == group ? m_used : -INFINITY);
+                w4[i] = other ? l_k : (k == group ? l_sum : 0.f);
+              }
+              float mm = fmaxf(fmaxf(pm[0], pm[1]), fmaxf(pm[2], pm[3]));
+#pragma unroll 1
+              for (int k = k_first + 4; k <= k_last; ++k)
+                mm = fmaxf(mm, k == group ? m_used : __ldcg(prm.part_ml + (size_t)piece_slot(k) * 2 * kRows + rr));
+              float lt = 0.f;
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {       // weights w_p = l_p 2^(m_p - mm), summed in piece order
+                w4[i] *= fast_exp2(pm[i] - mm);
+                lt += w4[i];
+              }
+              auto late_weight = [&](int k) -> float {     // pieces past the fourth
+                if (k == group) return l_sum * fast_exp2(m_used - mm);
+                const float* q_ml = prm.part_ml + (size_t)piece_slot(k) * 2 * kRows;
+                return __ldcg(q_ml + kRows + rr) * fast_exp2(__ldcg(q_ml + rr) - mm);
+              };
+#pragma unroll 1
+              for (int k = k_first + 4; k <= k_last; ++k) lt += late_weight(k);
+              if (!row_active) lt = 0.f;
+              const float inv = (row_active && lt > 0.f) ? 1.f / lt : 0.f;
+              TV_PROF_USE(__float_as_uint(inv));
+              TV_PROF_T(ep[3]);
+              // ---- pass 2: 64 output columns at a time, pieces in order (one fused multiply-add per piece and
+              // element, two elements per instruction); the own piece comes from TMEM and enters as its
+              // bf16-rounded normalised output, like every other piece
+              const float2 inv_own2 = make_float2(inv_own, inv_own), inv2 = make_float2(inv, inv);
+#pragma unroll 1
+              for (int hq = 0; hq < D / 64; ++hq) {
+                float2 acc[32];
+#pragma unroll
+                for (int c = 0; c < 32; ++c) acc[c] = make_float2(0.f, 0.f);
+#pragma unroll 1
+                for (int k = k_first; k <= k_last; ++k) {
+                  const int i = k - k_first;
+                  float w = i == 0 ? w4[0] : (i == 1 ? w4[1] : (i == 2 ? w4[2] : w4[3]));
+                  if (i >= 4) w = late_weight(k);
+                  const float2 w2 = make_float2(w, w);
+                  if (k == group) {
+                    TV_PROF_T(pc0);
+#pragma unroll
+                    for (int q = 0; q < 2; ++q) {
+                      uint32_t o[32];
+                      tmem_ld32(o_addr + (hq * 2 + q) * 32, o);
+                      tmem_wait_ld();
+#pragma unroll
+                      for (int c = 0; c < 16; ++c) {
+                        const float2 t = __fmul2_rn(make_float2(__uint_as_float(o[2 * c]), __uint_as_float(o[2 * c + 1])), inv_own2);
+                        const uint32_t own = pack_bf16(t.x, t.y);
+                        acc[q * 16 + c] = ffma2(w2, make_float2(__uint_as_float(own << 16), __uint_as_float(own & 0xffff0000u)),
+                                                acc[q * 16 + c]);
+                      }
+                    }
+#ifdef TV_PROF
+                    TV_PROF_USE(__float_as_uint(acc[31].y));
+                    ep_own += clock() - pc0;
+#endif
+                    continue;
+                  }
+                  const uint4* q_o = reinterpret_cast<const uint4*>(prm.part_o) + (size_t)piece_slot(k) * (D / 8) * kRows;
+                  uint4 v[8];
+                  TV_PROF_T(pc0);
+#pragma unroll
+                  for (int c = 0; c < 8; ++c) v[c] = __ldcg(q_o + (size_t)(hq * 8 + c) * kRows + rr);
+#pragma unroll
+                  for (int c = 0; c < 8; ++c) {
+                    const uint32_t wv[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                      acc[4 * c + e] = ffma2(w2, make_float2(__uint_as_float(wv[e] << 16), __uint_as_float(wv[e] & 0xffff0000u)),
+                                             acc[4 * c + e]);
+                  }
+#ifdef TV_PROF
+                  TV_PROF_USE(__float_as_uint(acc[31].y));
+                  ep_others += clock() - pc0;
+#endif
+                }
+                if (row_exists) {
+#pragma unroll
+                  for (int c = 0; c < 8; c += 2) {
+                    uint4 v[2];
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                      float2 t[4];
+#pragma unroll
+                      for (int x = 0; x < 4; ++x) t[x] = __fmul2_rn(acc[4 * (c + e) + x], inv2);
+                      v[e].x = pack_bf16(t[0].x, t[0].y);
+                      v[e].y = pack_bf16(t[1].x, t[1].y);
+                      v[e].z = pack_bf16(t[2].x, t[2].y);
+                      v[e].w = pack_bf16(t[3].x, t[3].y);
+                      if (!row_active) v[e] = make_uint4(0, 0, 0, 0);
+                    }
+                    if (prm.out_al32) {
+                      st_global_32B(orow + hq * 64 + c * 8, v[0], v[1]);
+                    } else {
+                      *reinterpret_cast<uint4*>(orow + hq * 64 + c * 8) = v[0];
+                      *reinterpret_cast<uint4*>(orow + hq * 64 + c * 8 + 8) = v[1];
+                    }
+                  }
+                }
+              }
+              if (row_exists && lse_p) *lse_p = (row_active && lt > 0.f) ? (mm + log2f(lt)) / kLog2e : -INFINITY;
+              tc_fence_before();
+              TV_PROF_T(ep[4]);
+              ok = epi_sync();   // keeps the two warpgroups' barrier phases in step with the other branch
+              if (!ok) break;
+              TV_PROF_T(ep[5]);
+            }
+          }
+        }
+        tr.mark(0x8000u);
+#ifdef TV_PROF
+        prof[8] += clock() - pc1;
+        if (tr.base && prof[9] < 24) {
+          unsigned long long* e = tr.base + prof[9] * 8;
+          e[0] = ep_kind; e[1] = ep_own;
+          for (int i = 1; i < 6; ++i) e[1 + i] = ep[i] - ep[i - 1];
+          e[7] = ep_others;      // pass 2: cycles from the loads of the other pieces to the end of their sums
+        }
         prof[9] += 1;
 #endif
-        tr.mark(0x8000u);
         fill += 2 * nt;
       }
 #ifdef TV_PROF
@@ -1129,243 +1338,8 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       }
 #endif
     }
-  } else if (warp >= 12) {
-    // =========================================================== epilogue warpgroup
-    // One thread per row, row tiles in turn.  For every item: (m, l) of the row from shared memory, O out of TMEM
-    // once the item's last PV has completed, normalised and rounded to bf16; a whole unit writes its output rows,
-    // a piece of a cut unit writes its partial and (m, l) to its CTA's slot of the workspace.  The pieces of a unit
-    // then count themselves on the unit's epoch-tagged counter (after a fence, so whoever reads the count also
-    // sees the partials); the piece that completes the count combines them all, its own included:
-    //   out = sum_p w_p O_p / sum_p w_p,  w_p = l_p 2^(m_p - max m),
-    // every piece entering as its bf16-rounded normalised output, in piece order, one fused multiply-add per
-    // piece: the result does not depend on which piece merges.  Partial outputs are stored column-group major,
-    // [slot][D/8][MT*128 rows][8 bf16]: a warp writes and reads 512 contiguous bytes per instruction.
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 " TV_STR(TV_REGS_EPI) ";");
-    const int row = threadIdx.x - kEpiThread0;       // TMEM lane = row inside a tile (warp 12 + i owns lanes 32 i ..)
-    const uint32_t lane_addr = (uint32_t)((warp & 3) << 5) << 16;
-    gdc_wait();      // the workspace and the outputs may belong to the kernel in front until it is done
-    // in-cache layout: a tree that does not fit behind its prefix is reported, not read past the capacity (rows
-    // past Scap arrive as zeros and the sequence's output is unspecified).  Raised after the wait: status[] may
-    // be written by the kernel in front until then.
-    if (prm.tree_in_cache && blockIdx.x == 0)
-#pragma unroll 1
-      for (int b = row; b < prm.B; b += 128) {
-        int S = prm.prefix_len[b];
-        S = S < 0 ? 0 : (S > prm.Scap ? prm.Scap : S);
-        if (S + prm.n_nodes[b] > prm.Scap) atomicOr(prm.status + b, TV_ST_CAPACITY);
-      }
-    if (!*abort_flag) {
-      Walk wk = walk_init();
-      Item it;
-      uint32_t item_cnt = 0, epi_phase = 0;
-      bool ok = true;
-      Tracer tr;
-      tr.init(row == 0 ? prm.trace : nullptr, 4);
-      tr.mark(0);
-      auto wwait = [&](uint32_t b_, uint32_t parity) -> bool {
-        return __all_sync(0xffffffffu, mbar_wait(b_, parity, abort_flag, wait_limit));
-      };
-      // rendezvous of the four epilogue warps, through an mbarrier so that it is bounded like every other wait
-      auto epi_sync = [&]() -> bool {
-        mbar_arrive(bar(L::EPI));
-        const bool r = wwait(bar(L::EPI), epi_phase & 1);
-        ++epi_phase;
-        return r;
-      };
-      constexpr int kRows = MT * 128;
-      while (ok && next_item(wk, it)) {
-        tr.mark(0x1000u | (item_cnt & 0xfffu));
-        const bool whole = (it.j0 == 0 && it.j1 == it.len);
-        // A piece: the unit's real tiles occupy [real0, uend) of the virtual tile space.  CTA groups
-        // k_first..k_last hold them, one piece each (a group between the two lies wholly inside the unit), and
-        // this CTA's group is one of them: two short walks over the cuts find both ends.  The piece of group k
-        // sits in slot 1 of its CTA if the unit starts in that group, else in slot 0 (a CTA holds at most the
-        // end of one unit and the start of another).
-        int k_first = group, k_last = group;
-        if (!whole) {
-          const int real0 = prm.Hkv * cum[it.b] + it.hk * (it.len + kSetupCost) + kSetupCost;
-          const int uend = real0 + it.len;
-          while (sch.group_start(k_first) > real0) --k_first;
-          while (sch.group_start(k_last + 1) < uend) ++k_last;
-        }
-        auto piece_slot = [&](int k) -> int { return (k * prm.NP + pair) * 2 + (k == k_first ? 1 : 0); };
-        const int my_slot = piece_slot(group);
-#pragma unroll 1
-        for (int t = 0; t < MT && ok; ++t) {
-          const int node = (pair * MT + t) * prm.NPT + row / prm.G;
-          const int gm = row % prm.G;
-          const bool row_exists = row < prm.NPT * prm.G && node < prm.Nmax;
-          const bool row_active = row_exists && node < it.n;
-          const int rr = t * 128 + row;
-          ok = wwait(bar(L::ML_READY + t), item_cnt & 1);
-          if (!ok) break;
-          const float2 ml = hand[rr];
-          mbar_arrive(bar(L::ML_FREE + t));
-          // every MMA of the item into this row tile's O (the barrier completes once per item)
-          ok = wwait(bar(L::ITEM_DONE + t), item_cnt & 1);
-          if (!ok) break;
-          tc_fence_after();
-          tr.mark(0x5000u | t);
-          const float inv = (row_active && ml.y > 0.f) ? 1.f / ml.y : 0.f;
-          const uint32_t o_addr = tmem + lane_addr + kTmemO0 + t * 128;
-          const int h = it.hk * prm.G + gm;
-          uint4* dst;
-          size_t stride_u4;
-          bool do_store;
-          if (whole) {
-            dst = reinterpret_cast<uint4*>(prm.out + (((size_t)it.b * prm.Nmax + node) * prm.Hq + h) * D);
-            stride_u4 = 1;
-            do_store = row_exists;
-          } else {
-            dst = reinterpret_cast<uint4*>(prm.part_o) + (size_t)my_slot * (D / 8) * kRows + rr;
-            stride_u4 = kRows;
-            do_store = row_active;
-          }
-          // normalised bf16 output of this row, 32 columns at a time
-#pragma unroll 1
-          for (int q = 0; q < D / 32; ++q) {
-            uint32_t o[32];
-            tmem_ld32(o_addr + q * 32, o);
-            tmem_wait_ld();
-            if (do_store) {
-              uint4 v[4];
-#pragma unroll
-              for (int c = 0; c < 4; ++c) {
-                v[c].x = pack_bf16(__uint_as_float(o[8 * c + 0]) * inv, __uint_as_float(o[8 * c + 1]) * inv);
-                v[c].y = pack_bf16(__uint_as_float(o[8 * c + 2]) * inv, __uint_as_float(o[8 * c + 3]) * inv);
-                v[c].z = pack_bf16(__uint_as_float(o[8 * c + 4]) * inv, __uint_as_float(o[8 * c + 5]) * inv);
-                v[c].w = pack_bf16(__uint_as_float(o[8 * c + 6]) * inv, __uint_as_float(o[8 * c + 7]) * inv);
-                if (!row_active) v[c] = make_uint4(0, 0, 0, 0);       // rows of padded nodes: O may hold anything
-              }
-              if (stride_u4 == 1 && prm.out_al32) {     // a row of the output: whole 32-byte sectors per store
-                st_global_32B(dst + q * 4, v[0], v[1]);
-                st_global_32B(dst + q * 4 + 2, v[2], v[3]);
-              } else {
-#pragma unroll
-                for (int c = 0; c < 4; ++c) dst[(size_t)(q * 4 + c) * stride_u4] = v[c];
-              }
-            }
-          }
-          // O_t is in registers / on its way to memory: the MMA issuer may overwrite it
-          tc_fence_before();
-          mbar_arrive(bar(L::O_FREE + t));
-          tr.mark(0x6000u | t);
-          if (whole) {
-            if (row_exists && prm.lse)
-              prm.lse[((size_t)it.b * prm.Hq + h) * prm.Nmax + node] =
-                  (row_active && ml.y > 0.f) ? (ml.x + log2f(ml.y)) / kLog2e : -INFINITY;
-          } else if (row_active) {
-            float* pml = prm.part_ml + (size_t)my_slot * 2 * kRows;
-            pml[rr] = ml.x;
-            pml[kRows + rr] = ml.y;
-          }
-        }
-        if (!ok) break;
-        ++item_cnt;
-        if (whole) continue;
-        // ---- publish the piece; the piece that completes the unit's count merges
-        const int n_frag = k_last - k_first + 1;
-        __threadfence();
-        ok = epi_sync();
-        if (!ok) break;
-        if (row == 0) {
-          unsigned long long* ctr = prm.counters + ((size_t)it.b * prm.Hkv + it.hk) * prm.NP + pair;
-          const unsigned long long seen = *reinterpret_cast<volatile unsigned long long*>(ctr);
-          const int cnt = bump_counter(ctr, seen, prm.epoch);
-          const int merger = (cnt == n_frag) ? 1 : 0;
-          // every piece has counted itself: nobody touches the counter again in this launch.  Clearing it lets the
-          // same launch be replayed with the same epoch (a captured CUDA graph) and find it unused.
-          if (merger) *reinterpret_cast<volatile unsigned long long*>(ctr) = 0ull;
-          __threadfence();
-          *last_flag = merger;
-        }
-        ok = epi_sync();
-        if (!ok) break;
-        const bool merges = *last_flag != 0;
-        ok = epi_sync();            // last_flag may be rewritten only after everybody has read it
-        if (!ok) break;
-        tr.mark(0x7000u | (merges ? 1u : 0u));
-        if (!merges) continue;
-        __threadfence();
-#pragma unroll 1
-        for (int t = 0; t < MT; ++t) {
-          const int node = (pair * MT + t) * prm.NPT + row / prm.G;
-          const int gm = row % prm.G;
-          const bool row_exists = row < prm.NPT * prm.G && node < prm.Nmax;
-          const bool row_active = row_exists && node < it.n;
-          const int rr = t * 128 + row;
-          const int h = it.hk * prm.G + gm;
-          tv_bf16* orow = prm.out + (((size_t)it.b * prm.Nmax + node) * prm.Hq + h) * D;
-          // pass 1: reference maximum and total weight of the row.  Every thread loads (row rr always lies inside
-          // a slot); rows that are not active read stale bytes and are masked by selects.
-          float mm = -INFINITY;
-#pragma unroll 1
-          for (int k = k_first; k <= k_last; ++k)
-            mm = fmaxf(mm, __ldcg(prm.part_ml + (size_t)piece_slot(k) * 2 * kRows + rr));
-          auto weight = [&](int k) -> float {     // w_p = l_p 2^(m_p - mm)
-            const float* q_ml = prm.part_ml + (size_t)piece_slot(k) * 2 * kRows;
-            return __ldcg(q_ml + kRows + rr) * fast_exp2(__ldcg(q_ml + rr) - mm);
-          };
-          float lt = 0.f;
-#pragma unroll 1
-          for (int k = k_first; k <= k_last; ++k) lt += weight(k);
-          if (!row_active) lt = 0.f;
-          const float inv = (row_active && lt > 0.f) ? 1.f / lt : 0.f;
-          const float2 inv2 = make_float2(inv, inv);
-          // pass 2: 32 output columns at a time, pieces in order, two elements per instruction
-#pragma unroll 1
-          for (int q = 0; q < D / 32; ++q) {
-            float2 acc[16];
-#pragma unroll
-            for (int c = 0; c < 16; ++c) acc[c] = make_float2(0.f, 0.f);
-#pragma unroll 1
-            for (int k = k_first; k <= k_last; ++k) {
-              const float w = weight(k);
-              const float2 w2 = make_float2(w, w);
-              const uint4* q_o = reinterpret_cast<const uint4*>(prm.part_o) + (size_t)piece_slot(k) * (D / 8) * kRows;
-              uint4 v[4];
-#pragma unroll
-              for (int c = 0; c < 4; ++c) v[c] = __ldcg(q_o + (size_t)(q * 4 + c) * kRows + rr);
-#pragma unroll
-              for (int c = 0; c < 4; ++c) {
-                const uint32_t wv[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                  acc[4 * c + e] = ffma2(w2, make_float2(__uint_as_float(wv[e] << 16), __uint_as_float(wv[e] & 0xffff0000u)),
-                                         acc[4 * c + e]);
-              }
-            }
-            if (row_exists) {
-              uint4 v[4];
-#pragma unroll
-              for (int c = 0; c < 4; ++c) {
-                float2 x[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) x[e] = __fmul2_rn(acc[4 * c + e], inv2);
-                v[c].x = pack_bf16(x[0].x, x[0].y);
-                v[c].y = pack_bf16(x[1].x, x[1].y);
-                v[c].z = pack_bf16(x[2].x, x[2].y);
-                v[c].w = pack_bf16(x[3].x, x[3].y);
-                if (!row_active) v[c] = make_uint4(0, 0, 0, 0);
-              }
-              if (prm.out_al32) {
-                st_global_32B(orow + q * 32, v[0], v[1]);
-                st_global_32B(orow + q * 32 + 16, v[2], v[3]);
-              } else {
-#pragma unroll
-                for (int c = 0; c < 4; ++c) *reinterpret_cast<uint4*>(orow + q * 32 + c * 8) = v[c];
-              }
-            }
-          }
-          if (row_exists && prm.lse)
-            prm.lse[((size_t)it.b * prm.Hq + h) * prm.Nmax + node] =
-                (row_active && lt > 0.f) ? (mm + log2f(lt)) / kLog2e : -INFINITY;
-        }
-        tr.mark(0x8000u);
-      }
-    }
   } else {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 " TV_STR(TV_REGS_LOW) ";");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
   }
 
   // ---- teardown
@@ -1442,7 +1416,7 @@ Geometry geometry(int B, int Nmax, int Hq, int Hkv, int d, bool query_device) {
   // workspace: counters, then (m,l) pairs, then partial O, sized for 160 SMs so the size does not depend on the device
   const size_t max_ctas = 160 > g.grid ? 160 : g.grid;
   g.counters_off = 0;
-  size_t off = (size_t)B * Hkv * g.NP * sizeof(unsigned long long);
+  size_t off = (size_t)B * Hkv * g.NP * 2 * sizeof(unsigned long long);
   off = (off + 255) & ~size_t(255);
   g.ml_off = off;
   off += max_ctas * 2 * (size_t)g.MT * 128 * 2 * sizeof(float);
@@ -1620,7 +1594,7 @@ int attn_entry(const tv_bf16* q,
 
 }  // namespace
 
-// Tuning aid, live only in a library built with -DTV_TRACE: while a device buffer of 160 * 5 * 256 u64 is
+// Tuning aid, live only in a library built with -DTV_TRACE: while a device buffer of 160 * 4 * 256 u64 is
 // registered here, every tree_verify_attn launch records a per-CTA, per-role timeline (tag << 48 |
 // globaltimer ns) into it.  NULL switches it off.
 extern "C" TV_API void tv_debug_set_attn_trace(unsigned long long* device_buffer) {
