@@ -119,6 +119,7 @@ def oracle_sample_seconds(cfg, seed):
     from workloads import case_to_numpy
     cn = case_to_numpy(case)
     Dp1 = cn["retrieve"].shape[2]
+    wall_0, cpu_0 = time.perf_counter(), time.process_time()
     t0 = time.perf_counter()
     mk = orc.build_mask(cn["parent"], cn["n_nodes"], Dp1 - 1, cn["retrieve"].shape[1])
     t_mask = time.perf_counter() - t0
@@ -149,12 +150,17 @@ def oracle_sample_seconds(cfg, seed):
         t_com = time.perf_counter() - t0
         est += t_arg * (cfg.B * cfg.V) / (small.B * small.V) + t_acc * cfg.B / small.B + t_com * cfg.B * cfg.L / small.B
         desc += f"; argmax over {small.V} of {cfg.V} logits per row; accept; commit of 1 layer"
+    # Threads the timed code actually used: CPU seconds of the process over wall seconds of the sample.  The oracle
+    # is Python loops on one core around numpy calls; only the per-head matmuls can fan out into numpy's BLAS pool.
+    wall, cpu = time.perf_counter() - wall_0, time.process_time() - cpu_0
+    used = cpu / max(wall, 1e-9)
     try:
         from threadpoolctl import threadpool_info
-        threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+        pool = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
     except Exception:
-        threads = os.cpu_count() or 1
-    return est, desc, threads
+        pool = os.cpu_count() or 1
+    desc += f"; CPU seconds / wall seconds of the sample = {used:.2f} (numpy BLAS pool: {pool} threads)"
+    return est, desc, max(1, int(round(used)))
 
 
 def run_reference(args, cfg):
@@ -356,6 +362,60 @@ def run_ours(args, cfg):
             graph_leg = {"error": f"{type(exc).__name__}: {exc}"[:200]}
             torch.cuda.synchronize()
 
+    # ---- the same step loop kept running for --sustain seconds (this rank's own clock): what the step costs once
+    # the board has reached its power limit, with the clocks seen over that region
+    sustained = None
+    if args.sustain > 0:
+        n_sus = max(args.steps, int(args.sustain / max(elapsed_ms / args.steps * 1e-3, 1e-6)) + 1)
+        every = max(1, n_sus // 64)                       # per-stage events on a subset of the steps
+        sm = {i: [ev() for _ in range(4)] for i in range(0, n_sus, every)}
+        sus_sampler = ClockSampler(local, period_s=0.02)
+        torch.cuda.synchronize()
+        sus_sampler.start()
+        s0, s1 = ev(), ev()
+        s0.record()
+        for i in range(n_sus):
+            one_step(sm.get(i))
+        s1.record()
+        torch.cuda.synchronize()
+        sus_clocks = sus_sampler.stop()
+        sus_ms = s0.elapsed_time(s1)
+        late = [m for i, m in sm.items() if i >= n_sus // 2]          # stages over the second half of the region
+        sustained = {"seconds": sus_ms * 1e-3, "steps": n_sus, "value": n_sus / (sus_ms * 1e-3), "unit": UNIT + " per GPU",
+                     "ms_per_step": sus_ms / n_sus,
+                     "attn_per_layer_us": sum(m[1].elapsed_time(m[2]) for m in late) / (len(late) * cfg.L) * 1e3,
+                     "accept_commit_us": sum(m[2].elapsed_time(m[3]) for m in late) / len(late) * 1e3,
+                     "clocks": sus_clocks}
+        if (buf.status.cpu().numpy() & 15).any():
+            raise SystemExit(f"bench.py: fatal status in the sustained run: {buf.status.cpu().numpy()}")
+
+    # ---- one-layer workloads: the attention launches alone, back to back on one stream (the step loop above is
+    # bound by the host's launch path when a step is a handful of short kernels); inputs cycle through the copies
+    attn_b2b = None
+    if cfg.L == 1:
+        n_b2b = 240
+        tv.tree_build_mask(case["parent"], case["n_nodes"], Dp1 - 1, buf.retrieve.shape[1], buf.anc_bits, buf.status,
+                           retrieve_indices=None if given_rows else buf.retrieve, n_paths=buf.n_paths)
+        for c in sets:
+            c["prefix_len"].copy_(prefix0)
+
+        def attn_only(i):
+            c = sets[i % n_sets]
+            tv.tree_verify_attn(c["q"][0], c["k_cache"][0], c["v_cache"][0], c["k_tree"][0], c["v_tree"][0],
+                                c["prefix_len"], c["n_nodes"], buf.anc_bits, scale, buf.out[0], buf.attn_ws, buf.status)
+
+        for i in range(8):
+            attn_only(i)
+        torch.cuda.synchronize()
+        b0, b1 = ev(), ev()
+        b0.record()
+        for i in range(n_b2b):
+            attn_only(i)
+        b1.record()
+        torch.cuda.synchronize()
+        b2b_us = b0.elapsed_time(b1) / n_b2b * 1e3
+        attn_b2b = {"launches": n_b2b, "us": b2b_us, "input_copies": n_sets}
+
     if rank != 0:
         return
     peak, peak_kind = measured_peaks()
@@ -384,6 +444,14 @@ def run_ours(args, cfg):
     }
     if graph_leg is not None:
         line["graph_replay"] = graph_leg
+    if sustained is not None:
+        sustained["attn_hbm_frac"] = alg_bytes / (sustained["attn_per_layer_us"] * 1e-6) / 1e9 / peak
+        line["sustained"] = sustained
+    if attn_b2b is not None:
+        attn_b2b["hbm_gbs"] = alg_bytes / (attn_b2b["us"] * 1e-6) / 1e9
+        attn_b2b["frac"] = attn_b2b["hbm_gbs"] / peak
+        attn_b2b["tensor_tflops"] = attn_flops(cfg, S_host) / (attn_b2b["us"] * 1e-6) / 1e12
+        line["attn_back_to_back"] = attn_b2b
     if args.budget_sweep:
         line["budget_sweep"] = budget_sweep(args.seed, dev)
     if args.in_cache and has_accept:
@@ -639,6 +707,8 @@ def main():
                     help="also time tree_verify_attn over the node budgets of the paper's sweep (extra key in the JSON line)")
     ap.add_argument("--in-cache", action="store_true",
                     help="also time the step with the tree's K/V inside the cache and the in-place commit")
+    ap.add_argument("--sustain", type=float, default=2.0,
+                    help="seconds the step loop is kept running after the headline for the power-capped figure (0: skip)")
     ap.add_argument("--no-graph", dest="graph", action="store_false",
                     help="skip the extra leg that times the step replayed from a captured CUDA graph")
     ap.add_argument("--sample-accept", action="store_true",
