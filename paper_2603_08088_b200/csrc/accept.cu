@@ -43,90 +43,116 @@ __device__ __forceinline__ float vec8_max(const uint4& u) {
   return r == r ? r : -INFINITY;                            // an all-NaN vector can never win
 }
 
-__global__ void __launch_bounds__(kScanThreads)
+// Persistent scan: the (row, vocabulary chunk) items are dealt round-robin to a grid of a few CTAs per SM, and a
+// CTA requests the vectors of its next item before it reduces the ones it holds, so the memory pipe never drains
+// at an item boundary.
+__global__ void __launch_bounds__(kScanThreads, 3)
 argmax_scan_kernel(const tv_bf16* __restrict__ logits, const int32_t* __restrict__ n_nodes,
-                   int Nmax, int V, int n_chunks, ArgPair* __restrict__ partial) {
+                   int Nmax, int V, int n_chunks, int n_items, ArgPair* __restrict__ partial) {
   tv::pdl_enter();
-  const int row = blockIdx.y;            // b * Nmax + i
-  const int b = row / Nmax, i = row - b * Nmax;
-  if (i >= n_nodes[b]) return;           // padded row: never read
-  const int chunk = blockIdx.x;
-  const int c0 = chunk * kChunkElems;
-  const int c1 = min(V, c0 + kChunkElems);
-  const tv_bf16* base = logits + (size_t)row * V;
   const int tid = threadIdx.x;
-
-  float best = -INFINITY;
-  int best_i = 0x7fffffff;
-
   const bool vec_ok = ((V & 7) == 0) && ((reinterpret_cast<uintptr_t>(logits) & 15u) == 0);
-  if (vec_ok) {
-    const uint4* vbase = reinterpret_cast<const uint4*>(base);
-    const int v0 = c0 >> 3, v1 = c1 >> 3;      // vector range of this chunk
-    uint4 u[kVecPerThread];
-    int vi[kVecPerThread];
-#pragma unroll
-    for (int k = 0; k < kVecPerThread; ++k) {
-      vi[k] = v0 + k * kScanThreads + tid;
-      u[k] = vi[k] < v1 ? __ldcs(vbase + vi[k]) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
-    }
-    int best_vec = -1;
-#pragma unroll
-    for (int k = 0; k < kVecPerThread; ++k) {
-      const float m = vec8_max(u[k]);
-      if (vi[k] < v1 && (m > best || best_vec < 0)) {   // increasing index order: strict > keeps the first
-        best = m;
-        best_vec = k;
-      }
-    }
-    if (best_vec >= 0) {
-      uint4 w = u[0];
-#pragma unroll
-      for (int k = 1; k < kVecPerThread; ++k) if (best_vec == k) w = u[k];
-      const uint32_t e[4] = {w.x, w.y, w.z, w.w};
-      float bv = -INFINITY;
-      int bi = 0x7fffffff;
-#pragma unroll
-      for (int t = 0; t < 8; ++t) {
-        const uint32_t bits = (t & 1) ? (e[t >> 1] >> 16) : (e[t >> 1] & 0xffffu);
-        float f = bf16_bits_to_float(bits);
-        f = f == f ? f : -INFINITY;
-        take_better(bv, bi, f, t);
-      }
-      int vsel = vi[0];
-#pragma unroll
-      for (int k = 1; k < kVecPerThread; ++k) if (best_vec == k) vsel = vi[k];
-      best = bv;
-      best_i = vsel * 8 + bi;
-    }
-  } else {
-    for (int v = c0 + tid; v < c1; v += kScanThreads) {
-      float f = bf16_bits_to_float(base[v]);
-      f = f == f ? f : -INFINITY;
-      take_better(best, best_i, f, v);
-    }
-  }
-
-  // warp, then block reduction with the same rule
-#pragma unroll
-  for (int off = 16; off > 0; off >>= 1) {
-    const float ov = __shfl_xor_sync(0xffffffffu, best, off);
-    const int oi = __shfl_xor_sync(0xffffffffu, best_i, off);
-    take_better(best, best_i, ov, oi);
-  }
   __shared__ float sv[kScanThreads / 32];
   __shared__ int si[kScanThreads / 32];
-  if ((tid & 31) == 0) {
-    sv[tid >> 5] = best;
-    si[tid >> 5] = best_i;
-  }
-  __syncthreads();
-  if (tid == 0) {
-    for (int w = 1; w < kScanThreads / 32; ++w) take_better(best, best_i, sv[w], si[w]);
-    ArgPair out;
-    out.val = best;
-    out.idx = best_i;
-    partial[(size_t)row * n_chunks + chunk] = out;
+  const uint4 kLowest = make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);     // bf16 -inf
+
+  // item -> (row, chunk, active); padded rows are never read
+  auto locate = [&](int item, int& row, int& chunk) -> bool {
+    if (item >= n_items) return false;
+    row = item / n_chunks;
+    chunk = item - row * n_chunks;
+    const int b = row / Nmax;
+    return row - b * Nmax < n_nodes[b];
+  };
+  auto fetch = [&](int row, int chunk, uint4* u) {
+    const uint4* vbase = reinterpret_cast<const uint4*>(logits + (size_t)row * V);
+    const int v0 = (chunk * kChunkElems) >> 3, v1 = min(V, (chunk + 1) * kChunkElems) >> 3;
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+      const int vi = v0 + k * kScanThreads + tid;
+      u[k] = vi < v1 ? __ldcs(vbase + vi) : kLowest;
+    }
+  };
+
+  int item = blockIdx.x;
+  int row = 0, chunk = 0;
+  bool active = locate(item, row, chunk);
+  uint4 u[kVecPerThread];
+  if (active && vec_ok) fetch(row, chunk, u);
+  while (item < n_items) {
+    const int nitem = item + gridDim.x;
+    int nrow = 0, nchunk = 0;
+    const bool nactive = locate(nitem, nrow, nchunk);
+    uint4 un[kVecPerThread];
+    if (nactive && vec_ok) fetch(nrow, nchunk, un);
+    if (active) {
+      const int c0 = chunk * kChunkElems;
+      const int c1 = min(V, c0 + kChunkElems);
+      float best = -INFINITY;
+      int best_i = 0x7fffffff;
+      if (vec_ok) {
+        const int v0 = c0 >> 3, v1 = c1 >> 3;      // vector range of this chunk
+        int best_vec = -1;
+#pragma unroll
+        for (int k = 0; k < kVecPerThread; ++k) {
+          const float m = vec8_max(u[k]);
+          if (v0 + k * kScanThreads + tid < v1 && (m > best || best_vec < 0)) {   // increasing index order: strict > keeps the first
+            best = m;
+            best_vec = k;
+          }
+        }
+        if (best_vec >= 0) {
+          uint4 w = u[0];
+#pragma unroll
+          for (int k = 1; k < kVecPerThread; ++k) if (best_vec == k) w = u[k];
+          const uint32_t e[4] = {w.x, w.y, w.z, w.w};
+          float bv = -INFINITY;
+          int bi = 0x7fffffff;
+#pragma unroll
+          for (int t = 0; t < 8; ++t) {
+            const uint32_t bits = (t & 1) ? (e[t >> 1] >> 16) : (e[t >> 1] & 0xffffu);
+            float f = bf16_bits_to_float(bits);
+            f = f == f ? f : -INFINITY;
+            take_better(bv, bi, f, t);
+          }
+          best = bv;
+          best_i = (v0 + best_vec * kScanThreads + tid) * 8 + bi;
+        }
+      } else {
+        const tv_bf16* base = logits + (size_t)row * V;
+        for (int v = c0 + tid; v < c1; v += kScanThreads) {
+          float f = bf16_bits_to_float(base[v]);
+          f = f == f ? f : -INFINITY;
+          take_better(best, best_i, f, v);
+        }
+      }
+      // warp, then block reduction with the same rule
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, best, off);
+        const int oi = __shfl_xor_sync(0xffffffffu, best_i, off);
+        take_better(best, best_i, ov, oi);
+      }
+      if ((tid & 31) == 0) {
+        sv[tid >> 5] = best;
+        si[tid >> 5] = best_i;
+      }
+      __syncthreads();
+      if (tid == 0) {
+        for (int w = 1; w < kScanThreads / 32; ++w) take_better(best, best_i, sv[w], si[w]);
+        ArgPair out;
+        out.val = best;
+        out.idx = best_i;
+        partial[(size_t)row * n_chunks + chunk] = out;
+      }
+      __syncthreads();       // sv / si are reused by the next item
+    }
+    item = nitem;
+    row = nrow;
+    chunk = nchunk;
+    active = nactive;
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) u[k] = un[k];
   }
 }
 
@@ -234,6 +260,17 @@ __global__ void node_scores_kernel(const tv_bf16* __restrict__ logits, const int
 
 int scan_chunks(int V) { return (V + kChunkElems - 1) / kChunkElems; }
 
+// CTAs of the persistent scan: three per SM (what its registers allow).
+int scan_ctas() {
+  static int n = [] {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148 * 3;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) return 148 * 3;
+    return sms * 3;
+  }();
+  return n;
+}
+
 // Scratch of tree_accept_noalloc: a fixed device array that lives in the library image, so that callers
 // who may not allocate device memory can still run the accept step.  Every GPU that loads the library
 // holds these 256 KiB until the process exits.
@@ -291,8 +328,11 @@ extern "C" int tree_accept(const tv_bf16* logits, const int32_t* tokens,
   const int n_chunks = scan_chunks(V);
   ArgPair* partial = static_cast<ArgPair*>(workspace);
   cudaStream_t s = (cudaStream_t)stream;
-  TV_CUDA_OK(tv::launch_pdl(argmax_scan_kernel, dim3(n_chunks, B * Nmax), dim3(kScanThreads), 0, s, logits, n_nodes, Nmax, V,
-                            n_chunks, partial));
+  const long long n_items = (long long)B * Nmax * n_chunks;
+  TV_REQUIRE(n_items < (1ll << 31), "tree_accept: B * Nmax * ceil(V / 16384) must stay below 2^31");
+  const int scan_grid = (int)(n_items < (long long)scan_ctas() ? n_items : scan_ctas());
+  TV_CUDA_OK(tv::launch_pdl(argmax_scan_kernel, dim3(scan_grid), dim3(kScanThreads), 0, s, logits, n_nodes, Nmax, V,
+                            n_chunks, (int)n_items, partial));
   TV_CUDA_OK(tv::launch_pdl(accept_kernel, dim3(B), dim3(256), Nmax * sizeof(int32_t), s, partial, n_chunks, tokens,
                             retrieve_indices, n_nodes, Nmax, P, Dp1, argmax_tok, safe_idx, candidates, accept_len, best_path,
                             accepted_nodes, next_token, status));

@@ -54,13 +54,26 @@ commit_copy_kernel(uint4* __restrict__ k_cache, uint4* __restrict__ v_cache,
   const size_t dst0 = (size_t)l * cache_layer_vec + (size_t)b * Hkv * Scap * dvec;      // [h, row, :]
   const int per = Hkv * dvec;                   // pieces of one node's row over all heads
   const int total = 2 * (A + 1) * per;
-  for (int t = threadIdx.x; t < total; t += kCopyThreads) {
-    const int kv = t >= (A + 1) * per;
-    const int u = kv ? t - (A + 1) * per : t;
-    const int j = u / per, w = u - j * per;
-    const int h = w / dvec, c = w - h * dvec;
-    const uint4 val = (kv ? v_tree : k_tree)[src0 + (size_t)s_nodes[j] * per + w];
-    (kv ? v_cache : k_cache)[dst0 + ((size_t)h * Scap + S + j) * dvec + c] = val;
+  // four pieces per thread and round: the loads of a round are all issued before the first store
+  for (int t0 = threadIdx.x; t0 < total; t0 += 4 * kCopyThreads) {
+    uint4 val[4];
+    uint4* dst[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int t = t0 + i * kCopyThreads;
+      dst[i] = nullptr;
+      if (t < total) {
+        const int kv = t >= (A + 1) * per;
+        const int u = kv ? t - (A + 1) * per : t;
+        const int j = u / per, w = u - j * per;
+        const int h = w / dvec, c = w - h * dvec;
+        val[i] = (kv ? v_tree : k_tree)[src0 + (size_t)s_nodes[j] * per + w];
+        dst[i] = (kv ? v_cache : k_cache) + dst0 + ((size_t)h * Scap + S + j) * dvec + c;
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      if (dst[i]) *dst[i] = val[i];
   }
 }
 
