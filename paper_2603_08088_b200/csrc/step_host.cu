@@ -105,6 +105,18 @@ extern "C" int tv_verify_step_host(const tv_step_host_args* a) {
   TV_REQUIRE(a->L >= 1 && a->B >= 1 && a->Nmax >= 1 && a->V >= 1 && a->P >= 1 && a->Dp1 >= 1 && a->Dp1 <= a->Nmax,
              "tv_verify_step_host: bad dimension");
   TV_REQUIRE((reinterpret_cast<uintptr_t>(a->staging) & 255u) == 0, "tv_verify_step_host: staging must be 256-byte aligned");
+  // Everything the four calls below would refuse is refused here, before the first copy is queued: a call that
+  // returns an error has then never touched the host buffers or the staging area.
+  TV_REQUIRE(a->B <= 512 && a->Nmax <= 256 && (long long)a->B * a->Nmax <= 65535,
+             "tv_verify_step_host: need B <= 512, Nmax <= 256, B * Nmax <= 65535");
+  TV_REQUIRE(a->d == 64 || a->d == 128, "tv_verify_step_host: d must be 64 or 128");
+  TV_REQUIRE(a->Hq >= 1 && a->Hkv >= 1 && a->Hq % a->Hkv == 0 && a->Hq / a->Hkv <= 128,
+             "tv_verify_step_host: need Hq %% Hkv == 0 and Hq / Hkv <= 128");
+  TV_REQUIRE(a->Scap >= 1 && a->scale > 0.f && a->L <= 65535 && a->Dp1 <= 1024,
+             "tv_verify_step_host: need Scap >= 1, scale > 0, L <= 65535, Dp1 <= 1024");
+  TV_REQUIRE((long long)a->B * a->Hkv * ((a->Scap + 127) / 128 + 8) < (1ll << 31),
+             "tv_verify_step_host: B * Hkv * Scap is too large for the attention's tile scheduler");
+  TV_REQUIRE(tv::aligned16(a->k_cache) && tv::aligned16(a->v_cache), "tv_verify_step_host: the caches must be 16-byte aligned");
   const int L = a->L, B = a->B, Nmax = a->Nmax, Hq = a->Hq, Hkv = a->Hkv, d = a->d, Scap = a->Scap, V = a->V,
             P = a->P, Dp1 = a->Dp1;
   const Staging s = layout(L, B, Nmax, Hq, Hkv, d, Scap, V, P, Dp1);
@@ -119,6 +131,9 @@ extern "C" int tv_verify_step_host(const tv_step_host_args* a) {
   TV_CUDA_OK(get_pipes(5 + 2 * L, &pp));
   cudaStream_t s_in = pp->in, s_out = pp->out;
   cudaEvent_t* ev = pp->events.data();
+  // From here on copies are in flight on the two private streams: if anything fails further down, the three
+  // streams are drained before the error is returned, so that the caller may free or reuse its buffers at once.
+  auto body = [&]() -> int {
   // work already queued on the caller's stream may still use the staging area and the host buffers
   TV_CUDA_OK(cudaEventRecord(ev[0], st));
   TV_CUDA_OK(cudaStreamWaitEvent(s_in, ev[0], 0));
@@ -187,4 +202,12 @@ extern "C" int tv_verify_step_host(const tv_step_host_args* a) {
   TV_CUDA_OK(cudaStreamWaitEvent(st, ev[4], 0));
   TV_CUDA_OK(cudaStreamSynchronize(st));
   return TV_OK;
+  };
+  const int rc_step = body();
+  if (rc_step != TV_OK) {
+    cudaStreamSynchronize(s_in);
+    cudaStreamSynchronize(s_out);
+    cudaStreamSynchronize(st);
+  }
+  return rc_step;
 }

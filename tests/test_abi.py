@@ -59,6 +59,23 @@ def test_null_and_bad_dims_are_rejected_without_a_launch(lib):
     assert rc == 1     # Nmax > 256
 
 
+def test_host_step_rejects_bad_dimensions_before_any_copy(lib):
+    """tv_verify_step_host checks everything its four calls would refuse before it queues a copy, so an error
+    return means the host buffers were never touched (no device is needed to see it: nothing is launched)."""
+    from paper_2603_08088_b200.binding import StepHostArgs
+    a = StepHostArgs()
+    for name, _ in StepHostArgs._fields_:
+        if name not in ("staging_bytes", "L", "B", "Nmax", "Hq", "Hkv", "d", "Scap", "V", "P", "Dp1", "scale", "stream"):
+            setattr(a, name, 0x1000)
+    a.staging_bytes = 1 << 40
+    a.L, a.B, a.Nmax, a.Hq, a.Hkv, a.d, a.Scap, a.V, a.P, a.Dp1, a.scale = 2, 2, 15, 4, 2, 32, 256, 1024, 8, 5, 0.125
+    assert lib.tv_verify_step_host(ctypes.byref(a)) == 1 and b"d must be 64 or 128" in lib.tv_last_error()
+    a.d, a.Hq = 64, 5
+    assert lib.tv_verify_step_host(ctypes.byref(a)) == 1 and b"Hq" in lib.tv_last_error()
+    a.Hq, a.Nmax = 4, 300
+    assert lib.tv_verify_step_host(ctypes.byref(a)) == 1 and b"Nmax" in lib.tv_last_error()
+
+
 def test_missing_library_fails_loudly(monkeypatch):
     from paper_2603_08088_b200 import binding
     monkeypatch.setattr(binding, "_lib", None)

@@ -617,6 +617,17 @@ def test_stochastic_accept_hand_worked_example():
     bad[0, 1] = 4
     r = orc.stochastic_accept(logits, bad, parent, n, np.array([[0.0, 0.0, 0.4, 0.9]]), np.array([0.1]), T, 4)
     assert r["status"].tolist() == [orc.ST_BAD_INDEX] and r["accepted_nodes"].tolist() == [[0, 2, 0, 0]]
+    # The flag is a property of the inputs, not of the walk: every valid non-root slot is checked, also one the walk
+    # never tries (node 3 hangs under node 2, which fails here) - the same rule as for the candidate rows of the
+    # greedy gather, where an out-of-range index in any slot is reported whether or not acceptance reaches it.
+    untried = tokens.copy()
+    untried[0, 3] = 99
+    r = orc.stochastic_accept(logits, untried, parent, n, np.array([[0.0, 0.3, 0.7, 0.1]]), np.array([0.4]), T, 4)
+    assert r["status"].tolist() == [orc.ST_BAD_INDEX]
+    assert r["accept_len"].tolist() == [0] and r["next_token"].tolist() == [2]       # the walk itself is unchanged
+    # a padded slot (here slot 3, with three active nodes) is not a proposal and raises nothing
+    r = orc.stochastic_accept(logits, untried, parent, np.array([3]), np.array([[0.0, 0.3, 0.7, 0.1]]), np.array([0.4]), T, 4)
+    assert r["status"].tolist() == [0]
 
 
 def test_stochastic_accept_becomes_greedy_at_low_temperature():

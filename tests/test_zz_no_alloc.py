@@ -1,7 +1,7 @@
 """tree_accept_noalloc: the accept step for callers that are not allowed to
 allocate device memory (its argmax scratch is a fixed array inside the
 library).  Checked through the C ABI against tree_accept with a caller
-workspace, bit for bit, on two calls in a row with different inputs, so that
+workspace and against the oracle, bit for bit, on two calls in a row with different inputs, so that
 whatever the first call left in the shared scratch cannot leak into the second.
 Collected last on purpose: a run that stops at the first failure has already
 run every other test."""
@@ -10,7 +10,8 @@ import pytest
 import torch
 
 import paper_2603_08088_b200 as tv
-from workloads import CONFIGS, make_case
+from oracle import tree_verify_oracle as orc
+from workloads import CONFIGS, make_case, bf16_bits
 
 pytestmark = pytest.mark.gpu
 
@@ -42,6 +43,14 @@ def _run_both(cfg, seed):
     for k in OUTS:
         assert torch.equal(a[k], b[k]), f"{k} differs between tree_accept and tree_accept_noalloc"
     assert torch.equal(st_a, st_b)
+    # and directly against the oracle, not only through the other entry point
+    n_nodes = case["n_nodes"].cpu().numpy()
+    am = orc.argmax_rows(bf16_bits(case["logits"]), n_nodes)
+    ref = orc.greedy_accept(case["retrieve"].cpu().numpy(), case["tokens"].cpu().numpy(), n_nodes, am)
+    assert np.array_equal(b["argmax_tok"].cpu().numpy(), am)
+    for k in ("accept_len", "best_path", "accepted_nodes", "next_token", "safe_idx", "candidates"):
+        assert np.array_equal(b[k].cpu().numpy(), ref[k]), f"{k} differs from the oracle"
+    assert np.array_equal(st_b.cpu().numpy(), ref["status"])
     return a
 
 
