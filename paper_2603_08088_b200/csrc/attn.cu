@@ -327,6 +327,9 @@ struct AttnParams {
                                  // table and the committed rows alone: they are read before the grid-dependency wait
   unsigned long long wait_limit_ns;   // limit of every bounded wait
   int debug;                     // bit 0: the producer issues no copy at all (exercises the expiry of the waits)
+  int chained;                   // the launch in front is a tree_verify_attn launch of the same call, on the other half
+                                 // of the workspace: nothing this launch reads or writes belongs to it, so no role
+                                 // waits for it; an idle warp does the wait that bounds the launches in flight to two
 };
 
 struct Item {
@@ -534,7 +537,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       // most two launches are in flight and the two halves of the workspace suffice.
       // status[] may still be written by the kernel in front (tree_build_mask stores it last), so a flag found
       // before the wait is kept here and raised after it.
-      bool synced = false;
+      bool synced = prm.chained != 0;          // chained: nothing to wait for, warp 2 releases the next launch
       int bad_page_b = -1;
       auto sync_with_predecessor = [&]() {
         gdc_wait();
@@ -619,7 +622,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
       }
       if (!synced) sync_with_predecessor();        // a CTA without work still has to let the next kernel go
-    } else {
+    } else if (!prm.chained) {
       gdc_wait();
       if (elect_one()) gdc_launch_dependents();
     }
@@ -754,7 +757,9 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const int row = ((warp & 3) << 5) | lane;        // TMEM lane = row inside the tile
     const uint32_t lane_addr = (uint32_t)((warp & 3) << 5) << 16;
     const bool wg_active = wg < MT;
-    gdc_wait();      // anc_bits, the workspace and the outputs may belong to the kernel in front until it is done
+    // anc_bits, the workspace and the outputs may belong to the kernel in front until it is done - unless that
+    // kernel is the previous layer of the same call
+    if (!prm.chained) gdc_wait();
     // in-cache layout: a tree that does not fit behind its prefix is reported, not read past the capacity (rows
     // past Scap arrive as zeros and the sequence's output is unspecified).  Raised after the wait: status[] may
     // be written by the kernel in front until then.
@@ -1340,6 +1345,12 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     }
   } else {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+    // Chained launch: the launch after this one takes the half of the workspace that the launch in front of
+    // this one is still using, so it may only be released once that launch has completed.
+    if (warp == 2 && prm.chained) {
+      gdc_wait();
+      if (elect_one()) gdc_launch_dependents();
+    }
   }
 
   // ---- teardown
@@ -1390,7 +1401,7 @@ bool encode_map(CUtensorMap* m, const void* base, int rank, const cuuint64_t* di
 
 struct Geometry {
   int G, NPT, n_row_tiles, MT, NP, sms, groups, grid;
-  size_t counters_off, ml_off, o_off, total;
+  size_t counters_off, ml_off, o_off, half, total;
 };
 
 int sm_count() {
@@ -1424,7 +1435,8 @@ Geometry geometry(int B, int Nmax, int Hq, int Hkv, int d, bool query_device) {
   g.o_off = off;
   off += max_ctas * 2 * (size_t)g.MT * 128 * d * sizeof(tv_bf16);
   off = (off + 255) & ~size_t(255);
-  g.total = off;
+  g.half = off;          // two such halves: the layers of one call overlap and take turns
+  g.total = 2 * off;
   return g;
 }
 
@@ -1467,11 +1479,13 @@ cudaError_t launch(const Geometry& g, const CUtensorMap* maps, const AttnParams&
 
 struct AttnOptions {
   bool early = false;                              // TV_ATTN_STABLE_INPUTS was promised
+  bool chained = false;                            // behind a launch of the same call that uses the other half
+  int half = 0;                                    // half of the workspace this launch uses
   unsigned long long wait_limit_ns = kWaitLimitNs;
   int debug = 0;
 };
 
-// One launch over sequences [0, B) of the given pointers, B <= kMaxB.  Both layouts of the committed cache:
+// The launch.  Both layouts of the committed cache:
 // contiguous [B,Hkv,Scap,d] (block_table == nullptr) or pages [n_pages,Hkv,128,d] named by
 // block_table[B,max_blocks] (then Scap = 128 * max_blocks).
 int attn_launch(const tv_bf16* q, const tv_bf16* k_cache, const tv_bf16* v_cache,
@@ -1508,9 +1522,10 @@ int attn_launch(const tv_bf16* q, const tv_bf16* k_cache, const tv_bf16* v_cache
   prm.out = out;
   prm.lse = lse;
   prm.status = status;
-  // Consecutive launches may share the workspace although they overlap on the device: a launch touches it only
-  // after its grid-dependency wait, that is after every earlier kernel of the stream has completed.
-  char* ws = static_cast<char*>(workspace);
+  // A launch that is not chained touches the workspace only after its grid-dependency wait, that is after every
+  // earlier kernel of the stream has completed; chained launches (the layers of one call) overlap and alternate
+  // between the two halves, and the launch after next is only released once the launch in front has completed.
+  char* ws = static_cast<char*>(workspace) + (opt.half ? g.half : 0);
   prm.counters = reinterpret_cast<unsigned long long*>(ws + g.counters_off);
   prm.part_ml = reinterpret_cast<float*>(ws + g.ml_off);
   prm.part_o = reinterpret_cast<tv_bf16*>(ws + g.o_off);
@@ -1527,7 +1542,8 @@ int attn_launch(const tv_bf16* q, const tv_bf16* k_cache, const tv_bf16* v_cache
   prm.q_box_bytes = 64u * (uint32_t)g.G * (uint32_t)g.NPT * 2u;
   prm.trace = g_trace.load(std::memory_order_relaxed);
   prm.scale_log2e = scale * kLog2e;
-  prm.early = opt.early ? 1 : 0;
+  prm.early = (opt.early || opt.chained) ? 1 : 0;
+  prm.chained = opt.chained ? 1 : 0;
   prm.wait_limit_ns = opt.wait_limit_ns;
   prm.debug = opt.debug;
   cudaError_t e;
@@ -1568,28 +1584,10 @@ int attn_entry(const tv_bf16* q,
   if (g.grid > 160) return tv::fail(TV_ERR_INVALID_ARG, "tree_verify_attn: device with more than 160 SMs is not supported");
   if (workspace_bytes < g.total)
     return tv::fail(TV_ERR_WORKSPACE, "tree_verify_attn: workspace of %zu bytes, need %zu", workspace_bytes, g.total);
-  // The schedule table of a launch holds kMaxB sequences: a larger batch goes out as several launches over
-  // consecutive ranges of sequences (every tensor has the sequence as its outermost index).  A launch behind
-  // another launch of the same call may always read its inputs early.
-  AttnOptions o = opt;
-  for (int b0 = 0; b0 < B; b0 += kMaxB) {
-    const int nb = B - b0 < kMaxB ? B - b0 : kMaxB;
-    const size_t qoff = (size_t)b0 * Nmax * Hq * d, toff = (size_t)b0 * Nmax * Hkv * d;
-    const size_t coff = block_table ? 0 : (size_t)b0 * Hkv * Scap * d;
-    const tv_bf16* kc = k_cache + coff;
-    const tv_bf16* vc = v_cache + coff;
-    // in-cache layout: the tree descriptors are never used by the kernel; they get the cache as a placeholder
-    const tv_bf16* kt = in_cache ? kc : k_tree + toff;
-    const tv_bf16* vt = in_cache ? vc : v_tree + toff;
-    const int rc = attn_launch(q + qoff, kc, vc, block_table ? block_table + (size_t)b0 * max_blocks : nullptr, n_pages,
-                               max_blocks, kt, vt, in_cache, prefix_len + b0, n_nodes + b0,
-                               anc_bits + (size_t)b0 * Nmax * ((Nmax + 31) / 32), nb, Nmax, Hq, Hkv, d, Scap, scale,
-                               out + qoff, lse ? lse + (size_t)b0 * Hq * Nmax : nullptr, workspace, status + b0, o,
-                               (cudaStream_t)stream);
-    if (rc != TV_OK) return rc;
-    o.early = true;
-  }
-  return TV_OK;
+  // in-cache layout: the tree descriptors are never used by the kernel; they get the cache as a placeholder
+  return attn_launch(q, k_cache, v_cache, block_table, n_pages, max_blocks, in_cache ? k_cache : k_tree,
+                     in_cache ? v_cache : v_tree, in_cache, prefix_len, n_nodes, anc_bits, B, Nmax, Hq, Hkv, d, Scap, scale,
+                     out, lse, workspace, status, opt, (cudaStream_t)stream);
 }
 
 }  // namespace
@@ -1679,7 +1677,11 @@ extern "C" int tree_verify_attn_layers(const tv_bf16* q,
                               lse ? lse + (size_t)l * B * Hq * Nmax : nullptr, workspace, workspace_bytes, status, opt,
                               stream);
     if (rc != TV_OK) return rc;
-    opt.early = true;      // behind a tree_verify_attn launch of this very call the inputs are stable
+    // Behind a tree_verify_attn launch of this very call the inputs are stable, and with the other half of the
+    // workspace nothing of that launch is touched at all: the next layer does not wait for it.
+    opt.early = true;
+    opt.chained = true;
+    opt.half ^= 1;
   }
   return TV_OK;
 }
