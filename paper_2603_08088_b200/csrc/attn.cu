@@ -149,20 +149,21 @@ __device__ __forceinline__ void st_global_32B(void* p, uint4 a, uint4 b) {
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// Tiled TMA loads.  The 3D one carries an L2 eviction-priority hint: the committed K/V prefix is read once per
+// Tiled TMA loads.  The one for the cache carries an L2 eviction-priority hint: the committed K/V prefix is read once per
 // launch, and letting it leave L2 first keeps Q, the partials and the kernel's own code resident.
-__device__ __forceinline__ void tma_load_3d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
-                                                 uint64_t policy) {
+// (The outermost coordinate of every tensor is the layer.)
+__device__ __forceinline__ void tma_load_4d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
+                                                 int c3, uint64_t policy) {
   asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5}], [%2], %6;"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "l"(policy)
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5, %6}], [%2], %7;"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(policy)
       : "memory");
 }
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
-                                            int c3) {
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
+                                            int c3, int c4) {
   asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
       : "memory");
 }
 
@@ -327,13 +328,12 @@ struct AttnParams {
                                  // table and the committed rows alone: they are read before the grid-dependency wait
   unsigned long long wait_limit_ns;   // limit of every bounded wait
   int debug;                     // bit 0: the producer issues no copy at all (exercises the expiry of the waits)
-  int chained;                   // the launch in front is a tree_verify_attn launch of the same call, on the other half
-                                 // of the workspace: nothing this launch reads or writes belongs to it, so no role
-                                 // waits for it; an idle warp does the wait that bounds the launches in flight to two
+  int L;                         // layers in this launch: their units form one tile space, layer after layer
+  long long out_layer_stride;    // elements between the outputs of two layers (lse is dense, [L,B,Hq,Nmax])
 };
 
 struct Item {
-  int b, hk, j0, j1, len, S, n;
+  int b, hk, j0, j1, len, S, n, layer;
 };
 
 // Shared bookkeeping of the linear tile space: cum[b] = sum of len over b' < b, len_b = ceil(S_b/128) + 1.
@@ -345,7 +345,8 @@ struct Sched {
   const int* cum;    // cum[b] = sum over b' < b of (len_b' + kSetupCost)
   const int* gs;     // gs[k] = first virtual tile of CTA group k, gs[groups] = total
   int B, Hkv;
-  int total;         // Hkv * cum[B]; the host refuses problems whose tile count does not fit 31 bits
+  int total;         // layers * Hkv * cum[B]; the host refuses problems whose tile count does not fit 31 bits
+  int per_layer;     // Hkv * cum[B]: the units of a layer tile one such stretch, layer after layer
   __device__ __forceinline__ int group_start(int k, int) const { return gs[k]; }
   __device__ __forceinline__ int find_b(int g) const {
     int lo = 0, hi = B - 1;   // largest b with Hkv*cum[b] <= g
@@ -461,14 +462,14 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   // write and a merge) and every group still gets a worthwhile share of tiles.
   int groups;
   {
-    const unsigned total = (unsigned)(prm.Hkv * cum[prm.B]);
+    const unsigned total = (unsigned)(prm.Hkv * cum[prm.B]) * (unsigned)prm.L;
     const unsigned want = total / (unsigned)kMinVirtualTilesPerGroup;
     groups = want < 1u ? 1 : (want < (unsigned)prm.groups ? (int)want : prm.groups);
     // A group count just above a multiple of the unit count is rounded down to it: with units of equal length
     // (one sequence, all heads) every unit is then cut into the same number of equal pieces and no cut falls
     // just behind a unit boundary.  Not worth more than 1/16 of the groups.
     {
-      const int units = prm.B * prm.Hkv, over = groups % units;
+      const int units = prm.B * prm.Hkv * prm.L, over = groups % units;
       if (groups > units && over * 16 <= groups) groups -= over;
     }
     // gs[k] = floor(total * k / groups) in 32-bit arithmetic: total = q * groups + r
@@ -479,7 +480,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   }
   __syncthreads();
 
-  Sched sch{cum, gs, prm.B, prm.Hkv, prm.Hkv * cum[prm.B]};
+  Sched sch{cum, gs, prm.B, prm.Hkv, prm.Hkv * cum[prm.B] * prm.L, prm.Hkv * cum[prm.B]};
   const int group = blockIdx.x / prm.NP;
   const int pair = blockIdx.x % prm.NP;
   const int g_begin = sch.group_start(group, groups);        // groups past the last used one get an empty range
@@ -488,9 +489,11 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   // Walks the items of this CTA's range; identical in every role.
   auto next_item = [&](int& g, Item& it) -> bool {
     while (g < g_end) {
-      const int b = sch.find_b(g);
+      const int layer = (int)((unsigned)g / (unsigned)sch.per_layer);
+      const int gl = g - layer * sch.per_layer;                   // place inside the layer
+      const int b = sch.find_b(gl);
       const int lenv = cum[b + 1] - cum[b];                       // setup region + real tiles
-      const unsigned local = (unsigned)(g - prm.Hkv * cum[b]);
+      const unsigned local = (unsigned)(gl - prm.Hkv * cum[b]);
       const int hk = (int)(local / (unsigned)lenv);
       const int r0 = (int)(local - (unsigned)hk * (unsigned)lenv);
       const int room = g_end - g;
@@ -501,6 +504,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       if (j1 <= j0) continue;                                     // only setup tiles of this unit fall in the range
       it.b = b;
       it.hk = hk;
+      it.layer = layer;
       it.j0 = j0;
       it.j1 = j1;
       it.len = lenv - kSetupCost;
@@ -537,7 +541,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       // most two launches are in flight and the two halves of the workspace suffice.
       // status[] may still be written by the kernel in front (tree_build_mask stores it last), so a flag found
       // before the wait is kept here and raised after it.
-      bool synced = prm.chained != 0;          // chained: nothing to wait for, warp 2 releases the next launch
+      bool synced = false;
       int bad_page_b = -1;
       auto sync_with_predecessor = [&]() {
         gdc_wait();
@@ -554,8 +558,8 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           for (int t = 0; t < MT; ++t)
 #pragma unroll
             for (int h = 0; h < D / 64; ++h)
-              tma_load_4d(sbase + L::kQ + t * L::kTileBytes + h * L::kHalf, &map_q, bar(L::Q_FULL), h * 64,
-                          it.hk * prm.G, (pair * MT + t) * prm.NPT, it.b);
+              tma_load_5d(sbase + L::kQ + t * L::kTileBytes + h * L::kHalf, &map_q, bar(L::Q_FULL), h * 64,
+                          it.hk * prm.G, (pair * MT + t) * prm.NPT, it.b, it.layer);
         }
         __syncwarp();
       };
@@ -603,13 +607,14 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 #pragma unroll
               for (int h = 0; h < D / 64; ++h) {
                 if (tree && prm.tree_in_cache)
-                  tma_load_3d_hint(dst + h * L::kHalf, kv ? &map_vc : &map_kc, bar(L::KV_FULL + slot), h * 64,
-                                   it.S + tt * kTileN, it.b * prm.Hkv + it.hk, kv_policy);
+                  tma_load_4d_hint(dst + h * L::kHalf, kv ? &map_vc : &map_kc, bar(L::KV_FULL + slot), h * 64,
+                                   it.S + tt * kTileN, it.b * prm.Hkv + it.hk, it.layer, kv_policy);
                 else if (tree)
-                  tma_load_4d(dst + h * L::kHalf, kv ? &map_vt : &map_kt, bar(L::KV_FULL + slot), h * 64, it.hk, tt * kTileN, it.b);
+                  tma_load_5d(dst + h * L::kHalf, kv ? &map_vt : &map_kt, bar(L::KV_FULL + slot), h * 64, it.hk, tt * kTileN, it.b,
+                              it.layer);
                 else
-                  tma_load_3d_hint(dst + h * L::kHalf, kv ? &map_vc : &map_kc, bar(L::KV_FULL + slot), h * 64, row0, slab,
-                                   kv_policy);
+                  tma_load_4d_hint(dst + h * L::kHalf, kv ? &map_vc : &map_kc, bar(L::KV_FULL + slot), h * 64, row0, slab,
+                                   it.layer, kv_policy);
               }
             }
             __syncwarp();
@@ -622,7 +627,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
       }
       if (!synced) sync_with_predecessor();        // a CTA without work still has to let the next kernel go
-    } else if (!prm.chained) {
+    } else {
       gdc_wait();
       if (elect_one()) gdc_launch_dependents();
     }
@@ -757,9 +762,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const int row = ((warp & 3) << 5) | lane;        // TMEM lane = row inside the tile
     const uint32_t lane_addr = (uint32_t)((warp & 3) << 5) << 16;
     const bool wg_active = wg < MT;
-    // anc_bits, the workspace and the outputs may belong to the kernel in front until it is done - unless that
-    // kernel is the previous layer of the same call
-    if (!prm.chained) gdc_wait();
+    gdc_wait();      // anc_bits, the workspace and the outputs may belong to the kernel in front until it is done
     // in-cache layout: a tree that does not fit behind its prefix is reported, not read past the capacity (rows
     // past Scap arrive as zeros and the sequence's output is unspecified).  Raised after the wait: status[] may
     // be written by the kernel in front until then.
@@ -820,7 +823,8 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         // the item and the compare-and-swap is issued when the last key tile begins, so that both round trips
         // are hidden behind the softmax of that tile; the outcome is looked at in the epilogue.
         const bool piece = !(it.j0 == 0 && it.j1 == it.len);
-        unsigned long long* claim_ctr = prm.counters + (((size_t)it.b * prm.Hkv + it.hk) * prm.NP + pair) * 2;
+        unsigned long long* claim_ctr =
+            prm.counters + ((((size_t)it.layer * prm.B + it.b) * prm.Hkv + it.hk) * prm.NP + pair) * 2;
         unsigned long long claim_assumed = 0, claim_ret = 1;
         int claim_cnt = 0;
         if (piece && threadIdx.x == 128) claim_assumed = *reinterpret_cast<volatile unsigned long long*>(claim_ctr);
@@ -1077,8 +1081,8 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           const uint32_t o_addr = o_addr_loop;
           const bool whole = (it.j0 == 0 && it.j1 == it.len);
           const int h = it.hk * prm.G + gm;
-          tv_bf16* orow = prm.out + (((size_t)it.b * prm.Nmax + node) * prm.Hq + h) * D;
-          float* lse_p = prm.lse ? prm.lse + ((size_t)it.b * prm.Hq + h) * prm.Nmax + node : nullptr;
+          tv_bf16* orow = prm.out + (size_t)it.layer * prm.out_layer_stride + (((size_t)it.b * prm.Nmax + node) * prm.Hq + h) * D;
+          float* lse_p = prm.lse ? prm.lse + (((size_t)it.layer * prm.B + it.b) * prm.Hq + h) * prm.Nmax + node : nullptr;
           // Normalised bf16 output of this row, 32 columns at a time (one copy of the loop for every use: the
           // epilogue is cold code, fetched while the other CTAs still stream K/V).
           auto store_rows = [&](uint4* dst, size_t stride_u4, float inv, bool do_store, bool zero) {
@@ -1130,7 +1134,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             // The unit's real tiles occupy [real0, uend) of the virtual tile space.  CTA groups k_first..k_last
             // hold them, one piece each (a group between the two lies wholly inside the unit), and this CTA's
             // group is one of them: two short walks over the cut table find both ends.
-            const int real0 = prm.Hkv * cum[it.b] + it.hk * (it.len + kSetupCost) + kSetupCost;
+            const int real0 = it.layer * sch.per_layer + prm.Hkv * cum[it.b] + it.hk * (it.len + kSetupCost) + kSetupCost;
             const int uend = real0 + it.len;
             int k_first = group, k_last = group;
             while (gs[k_first] > real0) --k_first;
@@ -1139,7 +1143,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             // slot of the piece CTA group k holds: slot 1 of its CTA if the unit starts in that group, else slot 0
             auto piece_slot = [&](int k) -> int { return (k * prm.NP + pair) * 2 + (k == k_first ? 1 : 0); };
             const int my_slot = piece_slot(group);
-            unsigned long long* ctr = prm.counters + (((size_t)it.b * prm.Hkv + it.hk) * prm.NP + pair) * 2;
+            unsigned long long* ctr = claim_ctr;
             TV_PROF_T(ep[1]);
             if (threadIdx.x == 128) {
               int ticket;
@@ -1345,12 +1349,6 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     }
   } else {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
-    // Chained launch: the launch after this one takes the half of the workspace that the launch in front of
-    // this one is still using, so it may only be released once that launch has completed.
-    if (warp == 2 && prm.chained) {
-      gdc_wait();
-      if (elect_one()) gdc_launch_dependents();
-    }
   }
 
   // ---- teardown
@@ -1401,7 +1399,7 @@ bool encode_map(CUtensorMap* m, const void* base, int rank, const cuuint64_t* di
 
 struct Geometry {
   int G, NPT, n_row_tiles, MT, NP, sms, groups, grid;
-  size_t counters_off, ml_off, o_off, half, total;
+  size_t ml_off, o_off, counters_off, counters_per_layer, total;
 };
 
 int sm_count() {
@@ -1414,6 +1412,8 @@ int sm_count() {
   return sms;
 }
 
+constexpr int kCounterLayers = 32;      // layers whose counters the workspace of tv_attn_workspace_bytes holds
+
 Geometry geometry(int B, int Nmax, int Hq, int Hkv, int d, bool query_device) {
   Geometry g{};
   g.G = Hq / Hkv;
@@ -1424,19 +1424,19 @@ Geometry geometry(int B, int Nmax, int Hq, int Hkv, int d, bool query_device) {
   g.sms = query_device ? sm_count() : 148;
   g.groups = g.sms / g.NP > 0 ? g.sms / g.NP : 1;
   g.grid = g.groups * g.NP;
-  // workspace: counters, then (m,l) pairs, then partial O, sized for 160 SMs so the size does not depend on the device
+  // workspace: (m,l) pairs, partial O (both sized for 160 SMs so the size does not depend on the device), then
+  // the units' counters, layer after layer: as many layers as fit behind the partials can share one launch
   const size_t max_ctas = 160 > g.grid ? 160 : g.grid;
-  g.counters_off = 0;
-  size_t off = (size_t)B * Hkv * g.NP * 2 * sizeof(unsigned long long);
-  off = (off + 255) & ~size_t(255);
+  size_t off = 0;
   g.ml_off = off;
   off += max_ctas * 2 * (size_t)g.MT * 128 * 2 * sizeof(float);
   off = (off + 255) & ~size_t(255);
   g.o_off = off;
   off += max_ctas * 2 * (size_t)g.MT * 128 * d * sizeof(tv_bf16);
   off = (off + 255) & ~size_t(255);
-  g.half = off;          // two such halves: the layers of one call overlap and take turns
-  g.total = 2 * off;
+  g.counters_off = off;
+  g.counters_per_layer = ((size_t)B * Hkv * g.NP * 2 * sizeof(unsigned long long) + 255) & ~size_t(255);
+  g.total = off + kCounterLayers * g.counters_per_layer;
   return g;
 }
 
@@ -1479,40 +1479,49 @@ cudaError_t launch(const Geometry& g, const CUtensorMap* maps, const AttnParams&
 
 struct AttnOptions {
   bool early = false;                              // TV_ATTN_STABLE_INPUTS was promised
-  bool chained = false;                            // behind a launch of the same call that uses the other half
-  int half = 0;                                    // half of the workspace this launch uses
   unsigned long long wait_limit_ns = kWaitLimitNs;
   int debug = 0;
 };
 
-// The launch.  Both layouts of the committed cache:
-// contiguous [B,Hkv,Scap,d] (block_table == nullptr) or pages [n_pages,Hkv,128,d] named by
-// block_table[B,max_blocks] (then Scap = 128 * max_blocks).
+// Layer strides of a call (elements); a single-layer call has L = 1 and strides that are never used.
+struct LayerStrides {
+  int64_t q = 0, cache = 0, tree = 0, out = 0;
+};
+
+// One launch over L layers.  Both layouts of the committed cache: contiguous [L,B,Hkv,Scap,d]
+// (block_table == nullptr) or, for one layer, pages [n_pages,Hkv,128,d] named by block_table[B,max_blocks]
+// (then Scap = 128 * max_blocks).  The layer is the outermost coordinate of every tensor map.
 int attn_launch(const tv_bf16* q, const tv_bf16* k_cache, const tv_bf16* v_cache,
                 const int32_t* block_table, int n_pages, int max_blocks,
                 const tv_bf16* k_tree, const tv_bf16* v_tree, bool in_cache,
                 const int32_t* prefix_len, const int32_t* n_nodes, const uint32_t* anc_bits,
-                int B, int Nmax, int Hq, int Hkv, int d, int Scap, float scale,
+                int L, const LayerStrides& ls, int B, int Nmax, int Hq, int Hkv, int d, int Scap, float scale,
                 tv_bf16* out, float* lse, void* workspace, int32_t* status, const AttnOptions& opt, cudaStream_t s) {
   const Geometry g = geometry(B, Nmax, Hq, Hkv, d, true);
   CUtensorMap maps[5];
   {
     const cuuint64_t e = 2;
-    cuuint64_t qd[4] = {(cuuint64_t)d, (cuuint64_t)Hq, (cuuint64_t)Nmax, (cuuint64_t)B};
-    cuuint64_t qs[3] = {(cuuint64_t)d * e, (cuuint64_t)Hq * d * e, (cuuint64_t)Nmax * Hq * d * e};
-    cuuint32_t qb[4] = {64, (cuuint32_t)g.G, (cuuint32_t)g.NPT, 1};
+    const cuuint64_t layers = (cuuint64_t)L;
+    // a stride of a dimension of extent 1 is never used, but has to be a valid one
+    const cuuint64_t q_ls = L > 1 ? (cuuint64_t)ls.q * e : (cuuint64_t)B * Nmax * Hq * d * e;
+    const cuuint64_t t_ls = L > 1 ? (cuuint64_t)ls.tree * e : (cuuint64_t)B * Nmax * Hkv * d * e;
+    cuuint64_t qd[5] = {(cuuint64_t)d, (cuuint64_t)Hq, (cuuint64_t)Nmax, (cuuint64_t)B, layers};
+    cuuint64_t qs[4] = {(cuuint64_t)d * e, (cuuint64_t)Hq * d * e, (cuuint64_t)Nmax * Hq * d * e, q_ls};
+    cuuint32_t qb[5] = {64, (cuuint32_t)g.G, (cuuint32_t)g.NPT, 1, 1};
     // rows of one (sequence, KV head) slab, or of one (page, KV head) slab of 128 rows
     const cuuint64_t slab_rows = block_table ? (cuuint64_t)kTileN : (cuuint64_t)Scap;
     const cuuint64_t slabs = block_table ? (cuuint64_t)n_pages * Hkv : (cuuint64_t)B * Hkv;
-    cuuint64_t cd[3] = {(cuuint64_t)d, slab_rows, slabs};
-    cuuint64_t cs[2] = {(cuuint64_t)d * e, slab_rows * d * e};
-    cuuint32_t cb[3] = {64, kTileN, 1};
-    cuuint64_t td[4] = {(cuuint64_t)d, (cuuint64_t)Hkv, (cuuint64_t)Nmax, (cuuint64_t)B};
-    cuuint64_t ts[3] = {(cuuint64_t)d * e, (cuuint64_t)Hkv * d * e, (cuuint64_t)Nmax * Hkv * d * e};
-    cuuint32_t tb[4] = {64, 1, kTileN, 1};
-    const bool ok = encode_map(&maps[0], q, 4, qd, qs, qb) && encode_map(&maps[1], k_cache, 3, cd, cs, cb) &&
-                    encode_map(&maps[2], v_cache, 3, cd, cs, cb) && encode_map(&maps[3], k_tree, 4, td, ts, tb) &&
-                    encode_map(&maps[4], v_tree, 4, td, ts, tb);
+    const cuuint64_t c_ls = L > 1 ? (cuuint64_t)ls.cache * e : slabs * slab_rows * d * e;
+    cuuint64_t cd[4] = {(cuuint64_t)d, slab_rows, slabs, layers};
+    cuuint64_t cs[3] = {(cuuint64_t)d * e, slab_rows * d * e, c_ls};
+    cuuint32_t cb[4] = {64, kTileN, 1, 1};
+    cuuint64_t td[5] = {(cuuint64_t)d, (cuuint64_t)Hkv, (cuuint64_t)Nmax, (cuuint64_t)B, layers};
+    cuuint64_t ts[4] = {(cuuint64_t)d * e, (cuuint64_t)Hkv * d * e, (cuuint64_t)Nmax * Hkv * d * e, t_ls};
+    cuuint32_t tb[5] = {64, 1, kTileN, 1, 1};
+    const bool ok = encode_map(&maps[0], q, 5, qd, qs, qb) && encode_map(&maps[1], k_cache, 4, cd, cs, cb) &&
+                    encode_map(&maps[2], v_cache, 4, cd, cs, cb) &&
+                    (in_cache ? (maps[3] = maps[1], maps[4] = maps[2], true)      // placeholders the kernel never uses
+                              : (encode_map(&maps[3], k_tree, 5, td, ts, tb) && encode_map(&maps[4], v_tree, 5, td, ts, tb)));
     if (!ok) return tv::fail(TV_ERR_CUDA, "tree_verify_attn: cuTensorMapEncodeTiled failed");
   }
   AttnParams prm{};
@@ -1522,10 +1531,9 @@ int attn_launch(const tv_bf16* q, const tv_bf16* k_cache, const tv_bf16* v_cache
   prm.out = out;
   prm.lse = lse;
   prm.status = status;
-  // A launch that is not chained touches the workspace only after its grid-dependency wait, that is after every
-  // earlier kernel of the stream has completed; chained launches (the layers of one call) overlap and alternate
-  // between the two halves, and the launch after next is only released once the launch in front has completed.
-  char* ws = static_cast<char*>(workspace) + (opt.half ? g.half : 0);
+  // The launch touches the workspace only after its grid-dependency wait, that is after every earlier kernel of
+  // the stream has completed: consecutive launches may share it although they overlap on the device.
+  char* ws = static_cast<char*>(workspace);
   prm.counters = reinterpret_cast<unsigned long long*>(ws + g.counters_off);
   prm.part_ml = reinterpret_cast<float*>(ws + g.ml_off);
   prm.part_o = reinterpret_cast<tv_bf16*>(ws + g.o_off);
@@ -1538,14 +1546,15 @@ int attn_launch(const tv_bf16* q, const tv_bf16* k_cache, const tv_bf16* v_cache
   prm.block_table = block_table;
   prm.max_blocks = max_blocks;
   prm.n_pages = n_pages;
-  prm.out_al32 = (reinterpret_cast<uintptr_t>(out) & 31u) == 0 ? 1 : 0;
+  prm.out_al32 = ((reinterpret_cast<uintptr_t>(out) & 31u) == 0 && (L == 1 || (ls.out * 2) % 32 == 0)) ? 1 : 0;
   prm.q_box_bytes = 64u * (uint32_t)g.G * (uint32_t)g.NPT * 2u;
   prm.trace = g_trace.load(std::memory_order_relaxed);
   prm.scale_log2e = scale * kLog2e;
-  prm.early = (opt.early || opt.chained) ? 1 : 0;
-  prm.chained = opt.chained ? 1 : 0;
+  prm.early = opt.early ? 1 : 0;
   prm.wait_limit_ns = opt.wait_limit_ns;
   prm.debug = opt.debug;
+  prm.L = L;
+  prm.out_layer_stride = ls.out;
   cudaError_t e;
   if (d == 128) e = g.MT == 2 ? launch<128, 2>(g, maps, prm, s) : launch<128, 1>(g, maps, prm, s);
   else e = g.MT == 2 ? launch<64, 2>(g, maps, prm, s) : launch<64, 1>(g, maps, prm, s);
@@ -1560,7 +1569,7 @@ int attn_entry(const tv_bf16* q,
                const tv_bf16* k_tree, const tv_bf16* v_tree,
                const int32_t* prefix_len, const int32_t* n_nodes,
                const uint32_t* anc_bits,
-               int B, int Nmax, int Hq, int Hkv, int d, int Scap, float scale,
+               int L, const LayerStrides& ls, int B, int Nmax, int Hq, int Hkv, int d, int Scap, float scale,
                tv_bf16* out, float* lse,
                void* workspace, size_t workspace_bytes,
                int32_t* status, const AttnOptions& opt, tv_stream stream) {
@@ -1568,7 +1577,7 @@ int attn_entry(const tv_bf16* q,
              "tree_verify_attn: NULL pointer");
   TV_REQUIRE((k_tree == nullptr) == (v_tree == nullptr), "tree_verify_attn: k_tree and v_tree must both be given or both be NULL");
   const bool in_cache = (k_tree == nullptr);       // the tree's K/V rows sit in the cache behind the prefix
-  TV_REQUIRE(B >= 0 && B <= 512, "tree_verify_attn: need 0 <= B <= 512");
+  TV_REQUIRE(B >= 0 && B <= kMaxB, "tree_verify_attn: need 0 <= B <= 512");
   TV_REQUIRE(Nmax >= 1 && Nmax <= 256, "tree_verify_attn: Nmax must be in 1..256");
   TV_REQUIRE(d == 64 || d == 128, "tree_verify_attn: d must be 64 or 128");
   TV_REQUIRE(Hq >= 1 && Hkv >= 1 && Hq % Hkv == 0 && Hq / Hkv <= kTileM, "tree_verify_attn: need Hq %% Hkv == 0 and Hq/Hkv <= 128");
@@ -1577,17 +1586,33 @@ int attn_entry(const tv_bf16* q,
                  tv::aligned16(v_tree) && tv::aligned16(out),
              "tree_verify_attn: tensors must be 16-byte aligned");
   TV_REQUIRE((reinterpret_cast<uintptr_t>(workspace) & 255u) == 0, "tree_verify_attn: workspace must be 256-byte aligned");
-  if (B == 0) return TV_OK;
+  if (B == 0 || L == 0) return TV_OK;
   const Geometry g = geometry(B, Nmax, Hq, Hkv, d, true);
-  TV_REQUIRE((long long)B * Hkv * ((Scap + kTileN - 1) / kTileN + 2 + kSetupCost) < (1ll << 31),
-             "tree_verify_attn: B * Hkv * Scap is too large for the tile scheduler");
+  const long long tiles_per_layer = (long long)B * Hkv * ((Scap + kTileN - 1) / kTileN + 2 + kSetupCost);
+  TV_REQUIRE(tiles_per_layer < (1ll << 31), "tree_verify_attn: B * Hkv * Scap is too large for the tile scheduler");
   if (g.grid > 160) return tv::fail(TV_ERR_INVALID_ARG, "tree_verify_attn: device with more than 160 SMs is not supported");
-  if (workspace_bytes < g.total)
-    return tv::fail(TV_ERR_WORKSPACE, "tree_verify_attn: workspace of %zu bytes, need %zu", workspace_bytes, g.total);
-  // in-cache layout: the tree descriptors are never used by the kernel; they get the cache as a placeholder
-  return attn_launch(q, k_cache, v_cache, block_table, n_pages, max_blocks, in_cache ? k_cache : k_tree,
-                     in_cache ? v_cache : v_tree, in_cache, prefix_len, n_nodes, anc_bits, B, Nmax, Hq, Hkv, d, Scap, scale,
-                     out, lse, workspace, status, opt, (cudaStream_t)stream);
+  if (workspace_bytes < g.counters_off + g.counters_per_layer)
+    return tv::fail(TV_ERR_WORKSPACE, "tree_verify_attn: workspace of %zu bytes, need %zu", workspace_bytes,
+                    g.counters_off + g.counters_per_layer);
+  // Layers that share a launch: as many as the workspace has counters for and as the 31-bit tile space holds.
+  long long per_launch = (long long)((workspace_bytes - g.counters_off) / g.counters_per_layer);
+  const long long by_tiles = ((1ll << 31) - 1) / tiles_per_layer;
+  if (per_launch > by_tiles) per_launch = by_tiles;
+  if (per_launch > 65535) per_launch = 65535;
+  AttnOptions o = opt;
+  for (int l0 = 0; l0 < L; l0 += (int)per_launch) {
+    const int nl = L - l0 < per_launch ? L - l0 : (int)per_launch;
+    const tv_bf16* kc = k_cache + (size_t)l0 * ls.cache;
+    const tv_bf16* vc = v_cache + (size_t)l0 * ls.cache;
+    const int rc = attn_launch(q + (size_t)l0 * ls.q, kc, vc, block_table, n_pages, max_blocks,
+                               in_cache ? kc : k_tree + (size_t)l0 * ls.tree, in_cache ? vc : v_tree + (size_t)l0 * ls.tree,
+                               in_cache, prefix_len, n_nodes, anc_bits, nl, ls, B, Nmax, Hq, Hkv, d, Scap, scale,
+                               out + (size_t)l0 * ls.out, lse ? lse + (size_t)l0 * B * Hq * Nmax : nullptr, workspace, status,
+                               o, (cudaStream_t)stream);
+    if (rc != TV_OK) return rc;
+    o.early = true;       // behind a tree_verify_attn launch of this very call the inputs are stable
+  }
+  return TV_OK;
 }
 
 }  // namespace
@@ -1611,8 +1636,8 @@ extern "C" TV_API int tv_debug_attn_expire(const tv_bf16* q, const tv_bf16* k_ca
   AttnOptions opt;
   opt.wait_limit_ns = wait_limit_ns;
   opt.debug = mode;
-  return attn_entry(q, k_cache, v_cache, nullptr, 0, 0, k_tree, v_tree, prefix_len, n_nodes, anc_bits, B, Nmax, Hq, Hkv,
-                    d, Scap, scale, out, lse, workspace, workspace_bytes, status, opt, stream);
+  return attn_entry(q, k_cache, v_cache, nullptr, 0, 0, k_tree, v_tree, prefix_len, n_nodes, anc_bits, 1, LayerStrides{}, B,
+                    Nmax, Hq, Hkv, d, Scap, scale, out, lse, workspace, workspace_bytes, status, opt, stream);
 }
 
 extern "C" size_t tv_attn_workspace_bytes(int B, int Nmax, int Hq, int Hkv, int d, int Scap) {
@@ -1630,8 +1655,8 @@ extern "C" int tree_verify_attn(const tv_bf16* q,
                                 tv_bf16* out, float* lse,
                                 void* workspace, size_t workspace_bytes,
                                 int32_t* status, tv_stream stream) {
-  return attn_entry(q, k_cache, v_cache, nullptr, 0, 0, k_tree, v_tree, prefix_len, n_nodes, anc_bits, B, Nmax, Hq, Hkv,
-                    d, Scap, scale, out, lse, workspace, workspace_bytes, status, AttnOptions{}, stream);
+  return attn_entry(q, k_cache, v_cache, nullptr, 0, 0, k_tree, v_tree, prefix_len, n_nodes, anc_bits, 1, LayerStrides{}, B,
+                    Nmax, Hq, Hkv, d, Scap, scale, out, lse, workspace, workspace_bytes, status, AttnOptions{}, stream);
 }
 
 extern "C" int tree_verify_attn_paged(const tv_bf16* q,
@@ -1648,8 +1673,8 @@ extern "C" int tree_verify_attn_paged(const tv_bf16* q,
   TV_REQUIRE(n_pages >= 1 && max_blocks >= 1 && max_blocks <= (1 << 20) && (long long)n_pages * Hkv < (1ll << 31),
              "tree_verify_attn_paged: need n_pages >= 1, 1 <= max_blocks <= 2^20, n_pages * Hkv < 2^31");
   return attn_entry(q, k_pages, v_pages, block_table, n_pages, max_blocks, k_tree, v_tree, prefix_len, n_nodes, anc_bits,
-                    B, Nmax, Hq, Hkv, d, max_blocks * kTileN, scale, out, lse, workspace, workspace_bytes, status,
-                    AttnOptions{}, stream);
+                    1, LayerStrides{}, B, Nmax, Hq, Hkv, d, max_blocks * kTileN, scale, out, lse, workspace, workspace_bytes,
+                    status, AttnOptions{}, stream);
 }
 
 extern "C" int tree_verify_attn_layers(const tv_bf16* q,
@@ -1668,20 +1693,11 @@ extern "C" int tree_verify_attn_layers(const tv_bf16* q,
   TV_REQUIRE((flags & ~(unsigned)TV_ATTN_STABLE_INPUTS) == 0, "tree_verify_attn_layers: unknown flag");
   AttnOptions opt;
   opt.early = (flags & TV_ATTN_STABLE_INPUTS) != 0;
-  for (int l = 0; l < L; ++l) {
-    const int rc = attn_entry(q + (size_t)l * q_layer_stride, k_cache + (size_t)l * cache_layer_stride,
-                              v_cache + (size_t)l * cache_layer_stride, nullptr, 0, 0,
-                              k_tree ? k_tree + (size_t)l * tree_layer_stride : nullptr,
-                              v_tree ? v_tree + (size_t)l * tree_layer_stride : nullptr, prefix_len, n_nodes, anc_bits, B,
-                              Nmax, Hq, Hkv, d, Scap, scale, out + (size_t)l * out_layer_stride,
-                              lse ? lse + (size_t)l * B * Hq * Nmax : nullptr, workspace, workspace_bytes, status, opt,
-                              stream);
-    if (rc != TV_OK) return rc;
-    // Behind a tree_verify_attn launch of this very call the inputs are stable, and with the other half of the
-    // workspace nothing of that launch is touched at all: the next layer does not wait for it.
-    opt.early = true;
-    opt.chained = true;
-    opt.half ^= 1;
-  }
-  return TV_OK;
+  LayerStrides ls;
+  ls.q = q_layer_stride;
+  ls.cache = cache_layer_stride;
+  ls.tree = tree_layer_stride;
+  ls.out = out_layer_stride;
+  return attn_entry(q, k_cache, v_cache, nullptr, 0, 0, k_tree, v_tree, prefix_len, n_nodes, anc_bits, L, ls, B, Nmax, Hq,
+                    Hkv, d, Scap, scale, out, lse, workspace, workspace_bytes, status, opt, stream);
 }
