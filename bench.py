@@ -389,6 +389,29 @@ def run_ours(args, cfg):
         if (buf.status.cpu().numpy() & 15).any():
             raise SystemExit(f"bench.py: fatal status in the sustained run: {buf.status.cpu().numpy()}")
 
+    # ---- multi-layer workloads: the same layers issued as L separate tree_verify_attn calls, back to back (what a
+    # caller whose layers depend on each other has to issue: every call is a launch of its own with its own pipeline
+    # fill, tail and merges, and reads nothing before the call in front has finished)
+    attn_single = None
+    if cfg.L > 1:
+        case["prefix_len"].copy_(prefix0)
+
+        def layer_by_layer():      # issued from C, so that the host's launch path does not bound the figure
+            tv.tree_verify_attn_layers(case["q"], case["k_cache"], case["v_cache"], case["k_tree"], case["v_tree"],
+                                       case["prefix_len"], case["n_nodes"], buf.anc_bits, scale, buf.out, buf.attn_ws,
+                                       buf.status, flags=tv.TV_ATTN_LAUNCH_PER_LAYER)
+
+        layer_by_layer()
+        torch.cuda.synchronize()
+        reps = 5
+        c0, c1 = ev(), ev()
+        c0.record()
+        for _ in range(reps):
+            layer_by_layer()
+        c1.record()
+        torch.cuda.synchronize()
+        attn_single = {"calls": reps * cfg.L, "us_per_layer": c0.elapsed_time(c1) / (reps * cfg.L) * 1e3}
+
     # ---- one-layer workloads: the attention launches alone, back to back on one stream (the step loop above is
     # bound by the host's launch path when a step is a handful of short kernels); inputs cycle through the copies
     attn_b2b = None
@@ -447,6 +470,10 @@ def run_ours(args, cfg):
     if sustained is not None:
         sustained["attn_hbm_frac"] = alg_bytes / (sustained["attn_per_layer_us"] * 1e-6) / 1e9 / peak
         line["sustained"] = sustained
+    if attn_single is not None:
+        attn_single["hbm_gbs"] = alg_bytes / (attn_single["us_per_layer"] * 1e-6) / 1e9
+        attn_single["frac"] = attn_single["hbm_gbs"] / peak
+        line["attn_single_call"] = attn_single
     if attn_b2b is not None:
         attn_b2b["hbm_gbs"] = alg_bytes / (attn_b2b["us"] * 1e-6) / 1e9
         attn_b2b["frac"] = attn_b2b["hbm_gbs"] / peak
@@ -544,9 +571,9 @@ def in_cache_step(cfg, case, buf, prefix0, scale, given_rows, steps, dev):
         tv.tree_build_mask(case["parent"], case["n_nodes"], cfg.D, buf.retrieve.shape[1], buf.anc_bits, buf.status,
                            retrieve_indices=None if given_rows else buf.retrieve, n_paths=buf.n_paths)
         m[1].record()
-        for l in range(cfg.L):
-            tv.tree_verify_attn(case["q"][l], case["k_cache"][l], case["v_cache"][l], None, None, case["prefix_len"],
-                                case["n_nodes"], buf.anc_bits, scale, buf.out[l], buf.attn_ws, buf.status)
+        tv.tree_verify_attn_layers(case["q"], case["k_cache"], case["v_cache"], None, None, case["prefix_len"],
+                                   case["n_nodes"], buf.anc_bits, scale, buf.out, buf.attn_ws, buf.status,
+                                   flags=tv.TV_ATTN_STABLE_INPUTS)
         m[2].record()
         tv.tree_accept(case["logits"], case["tokens"], case["retrieve"] if given_rows else buf.retrieve, case["n_nodes"],
                        buf.argmax_tok, buf.accept_len, buf.best_path, buf.accepted_nodes, buf.next_token, buf.accept_ws,
@@ -625,10 +652,9 @@ def paged_step(cfg, case, buf, prefix0, scale, given_rows, steps, dev, seed):
         tv.tree_build_mask(case["parent"], case["n_nodes"], cfg.D, buf.retrieve.shape[1], buf.anc_bits, buf.status,
                            retrieve_indices=None if given_rows else buf.retrieve, n_paths=buf.n_paths)
         m[1].record()
-        for l in range(L):
-            tv.tree_verify_attn_paged(case["q"][l], k_pages[l], v_pages[l], bt, case["k_tree"][l], case["v_tree"][l],
-                                      case["prefix_len"], case["n_nodes"], buf.anc_bits, scale, buf.out[l], buf.attn_ws,
-                                      buf.status)
+        tv.tree_verify_attn_paged_layers(case["q"], k_pages, v_pages, bt, case["k_tree"], case["v_tree"], case["prefix_len"],
+                                         case["n_nodes"], buf.anc_bits, scale, buf.out, buf.attn_ws, buf.status,
+                                         flags=tv.TV_ATTN_STABLE_INPUTS)
         m[2].record()
         tv.tree_accept(case["logits"], case["tokens"], case["retrieve"] if given_rows else buf.retrieve, case["n_nodes"],
                        buf.argmax_tok, buf.accept_len, buf.best_path, buf.accepted_nodes, buf.next_token, buf.accept_ws,

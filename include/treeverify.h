@@ -102,6 +102,8 @@ TV_API int tree_build_mask(const int32_t* parent, const int32_t* n_nodes,
 
 /* Flags of tree_verify_attn_layers. */
 enum {
+  TV_ATTN_LAUNCH_PER_LAYER = 2, /* one launch per layer, exactly as L calls of tree_verify_attn would issue them (for
+                                 comparison; the default is one launch for all layers) */
   TV_ATTN_STABLE_INPUTS = 1   /* the caller promises: the kernel directly in front of this call on the stream does
                                  not write prefix_len, n_nodes or rows [0, prefix_len) of the cache - or it does, but
                                  lets no successor start before it has completed.  tree_build_mask in front (the
@@ -220,6 +222,25 @@ TV_API int tree_verify_attn_paged(const tv_bf16* q,
                      tv_bf16* out, float* lse,
                      void* workspace, size_t workspace_bytes,
                      int32_t* status, tv_stream stream);
+
+/*
+ * tree_verify_attn_paged for all L layers of a step in one launch: k_pages,
+ * v_pages [L,n_pages,Hkv,128,d] with layer stride page_layer_stride (elements;
+ * the layout kv_commit_paged writes), one block table for all layers.
+ * Otherwise as tree_verify_attn_layers (flags: TV_ATTN_STABLE_INPUTS, which
+ * here also covers the block table).
+ */
+TV_API int tree_verify_attn_paged_layers(const tv_bf16* q,
+                     const tv_bf16* k_pages, const tv_bf16* v_pages,
+                     const int32_t* block_table,
+                     const tv_bf16* k_tree, const tv_bf16* v_tree,
+                     const int32_t* prefix_len, const int32_t* n_nodes,
+                     const uint32_t* anc_bits,
+                     int L, int B, int Nmax, int Hq, int Hkv, int d, int n_pages, int max_blocks, float scale,
+                     int64_t q_layer_stride, int64_t page_layer_stride, int64_t tree_layer_stride,
+                     tv_bf16* out, int64_t out_layer_stride, float* lse,
+                     void* workspace, size_t workspace_bytes,
+                     int32_t* status, unsigned flags, tv_stream stream);
 
 /* Scratch needed by tree_accept (bytes). */
 TV_API size_t tv_accept_workspace_bytes(int B, int Nmax, int V);

@@ -14,9 +14,10 @@ LIB_PATH = os.path.join(_PKG, "libtreeverify.so")
 TV_OK, TV_ERR_INVALID_ARG, TV_ERR_CUDA, TV_ERR_WORKSPACE = 0, 1, 2, 3
 TV_ST_BAD_TREE, TV_ST_BAD_INDEX, TV_ST_CAPACITY, TV_ST_TIMEOUT, TV_ST_PATHS_TRUNCATED = 1, 2, 4, 8, 16
 TV_ATTN_STABLE_INPUTS = 1
+TV_ATTN_LAUNCH_PER_LAYER = 2
 
 EXPORTS = ["tv_last_error", "tv_version", "tv_launch_count", "tree_build_mask", "tv_attn_workspace_bytes", "tree_verify_attn",
-           "tree_verify_attn_layers",
+           "tree_verify_attn_layers", "tree_verify_attn_paged_layers",
            "tv_accept_workspace_bytes", "tree_accept", "tree_node_scores", "tree_merge_partials", "tv_accept_noalloc_max_bytes", "tree_accept_noalloc",
            "tv_sample_workspace_bytes", "tree_accept_sample",
            "kv_commit", "kv_commit_inplace", "tree_verify_attn_paged", "kv_commit_paged", "tv_step_staging_bytes",
@@ -67,6 +68,9 @@ def load():
     lib.tree_verify_attn_layers.restype = _c_int
     lib.tree_verify_attn_layers.argtypes = ([_c_vp] * 8 + [_c_int] * 7 + [_c_f] + [_c_i64] * 3 + [_c_vp, _c_i64, _c_vp, _c_vp, _c_sz,
                                             _c_vp, ctypes.c_uint, _c_vp])
+    lib.tree_verify_attn_paged_layers.restype = _c_int
+    lib.tree_verify_attn_paged_layers.argtypes = ([_c_vp] * 9 + [_c_int] * 8 + [_c_f] + [_c_i64] * 3 + [_c_vp, _c_i64, _c_vp, _c_vp,
+                                                  _c_sz, _c_vp, ctypes.c_uint, _c_vp])
     lib.tv_accept_workspace_bytes.restype = _c_sz
     lib.tv_accept_workspace_bytes.argtypes = [_c_int] * 3
     lib.tree_accept.restype = _c_int
@@ -183,6 +187,21 @@ def tree_verify_attn_layers(q, k_cache, v_cache, k_tree, v_tree, prefix_len, n_n
                                           out.stride(0), None if lse is None else lse.data_ptr(), _ptr(workspace),
                                           workspace.numel() * workspace.element_size(), _ptr(status), int(flags),
                                           _stream(stream)))
+
+
+def tree_verify_attn_paged_layers(q, k_pages, v_pages, block_table, k_tree, v_tree, prefix_len, n_nodes, anc_bits, scale,
+                                  out, workspace, status, lse=None, flags=0, stream=None):
+    """All layers over a paged cache: k_pages, v_pages [L,n_pages,Hkv,128,d], one block table [B,max_blocks]."""
+    L, B, Nmax, Hq, d = q.shape
+    _, n_pages, Hkv, _, _ = k_pages.shape
+    assert lse is None or lse.is_contiguous()
+    _check(load().tree_verify_attn_paged_layers(q.data_ptr(), k_pages.data_ptr(), v_pages.data_ptr(), _ptr(block_table),
+                                                k_tree.data_ptr(), v_tree.data_ptr(), _ptr(prefix_len), _ptr(n_nodes),
+                                                _ptr(anc_bits), L, B, Nmax, Hq, Hkv, d, n_pages, block_table.shape[1],
+                                                float(scale), q.stride(0), k_pages.stride(0), k_tree.stride(0),
+                                                out.data_ptr(), out.stride(0), None if lse is None else lse.data_ptr(),
+                                                _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                                _ptr(status), int(flags), _stream(stream)))
 
 
 def tv_debug_attn_expire(q, k_cache, v_cache, k_tree, v_tree, prefix_len, n_nodes, anc_bits, scale, out, workspace, status,

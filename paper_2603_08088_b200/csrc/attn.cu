@@ -1690,7 +1690,7 @@ extern "C" int tree_verify_attn_layers(const tv_bf16* q,
   TV_REQUIRE(L >= 0 && L <= 65535, "tree_verify_attn_layers: need 0 <= L <= 65535");
   TV_REQUIRE(q_layer_stride % 8 == 0 && cache_layer_stride % 8 == 0 && tree_layer_stride % 8 == 0 && out_layer_stride % 8 == 0,
              "tree_verify_attn_layers: layer strides must be multiples of 8 elements");
-  TV_REQUIRE((flags & ~(unsigned)TV_ATTN_STABLE_INPUTS) == 0, "tree_verify_attn_layers: unknown flag");
+  TV_REQUIRE((flags & ~(unsigned)(TV_ATTN_STABLE_INPUTS | TV_ATTN_LAUNCH_PER_LAYER)) == 0, "tree_verify_attn_layers: unknown flag");
   AttnOptions opt;
   opt.early = (flags & TV_ATTN_STABLE_INPUTS) != 0;
   LayerStrides ls;
@@ -1698,6 +1698,50 @@ extern "C" int tree_verify_attn_layers(const tv_bf16* q,
   ls.cache = cache_layer_stride;
   ls.tree = tree_layer_stride;
   ls.out = out_layer_stride;
+  if (flags & TV_ATTN_LAUNCH_PER_LAYER) {      // exactly what L calls of tree_verify_attn issue
+    for (int l = 0; l < L; ++l) {
+      const int rc = attn_entry(q + (size_t)l * ls.q, k_cache + (size_t)l * ls.cache, v_cache + (size_t)l * ls.cache, nullptr,
+                                0, 0, k_tree ? k_tree + (size_t)l * ls.tree : nullptr,
+                                v_tree ? v_tree + (size_t)l * ls.tree : nullptr, prefix_len, n_nodes, anc_bits, 1,
+                                LayerStrides{}, B, Nmax, Hq, Hkv, d, Scap, scale, out + (size_t)l * ls.out,
+                                lse ? lse + (size_t)l * B * Hq * Nmax : nullptr, workspace, workspace_bytes, status, opt,
+                                stream);
+      if (rc != TV_OK) return rc;
+      opt.early = true;      // behind a tree_verify_attn launch of this very call the inputs are stable
+    }
+    return TV_OK;
+  }
   return attn_entry(q, k_cache, v_cache, nullptr, 0, 0, k_tree, v_tree, prefix_len, n_nodes, anc_bits, L, ls, B, Nmax, Hq,
                     Hkv, d, Scap, scale, out, lse, workspace, workspace_bytes, status, opt, stream);
+}
+
+extern "C" int tree_verify_attn_paged_layers(const tv_bf16* q,
+                                             const tv_bf16* k_pages, const tv_bf16* v_pages,
+                                             const int32_t* block_table,
+                                             const tv_bf16* k_tree, const tv_bf16* v_tree,
+                                             const int32_t* prefix_len, const int32_t* n_nodes,
+                                             const uint32_t* anc_bits,
+                                             int L, int B, int Nmax, int Hq, int Hkv, int d, int n_pages, int max_blocks,
+                                             float scale,
+                                             int64_t q_layer_stride, int64_t page_layer_stride, int64_t tree_layer_stride,
+                                             tv_bf16* out, int64_t out_layer_stride, float* lse,
+                                             void* workspace, size_t workspace_bytes,
+                                             int32_t* status, unsigned flags, tv_stream stream) {
+  TV_REQUIRE(block_table && k_tree && v_tree, "tree_verify_attn_paged_layers: NULL pointer");
+  TV_REQUIRE(n_pages >= 1 && max_blocks >= 1 && max_blocks <= (1 << 20) && (long long)n_pages * Hkv < (1ll << 31),
+             "tree_verify_attn_paged_layers: need n_pages >= 1, 1 <= max_blocks <= 2^20, n_pages * Hkv < 2^31");
+  TV_REQUIRE(L >= 0 && L <= 65535, "tree_verify_attn_paged_layers: need 0 <= L <= 65535");
+  TV_REQUIRE(q_layer_stride % 8 == 0 && page_layer_stride % 8 == 0 && tree_layer_stride % 8 == 0 && out_layer_stride % 8 == 0,
+             "tree_verify_attn_paged_layers: layer strides must be multiples of 8 elements");
+  TV_REQUIRE((flags & ~(unsigned)TV_ATTN_STABLE_INPUTS) == 0, "tree_verify_attn_paged_layers: unknown flag");
+  AttnOptions opt;
+  opt.early = (flags & TV_ATTN_STABLE_INPUTS) != 0;
+  LayerStrides ls;
+  ls.q = q_layer_stride;
+  ls.cache = page_layer_stride;
+  ls.tree = tree_layer_stride;
+  ls.out = out_layer_stride;
+  return attn_entry(q, k_pages, v_pages, block_table, n_pages, max_blocks, k_tree, v_tree, prefix_len, n_nodes, anc_bits, L,
+                    ls, B, Nmax, Hq, Hkv, d, max_blocks * kTileN, scale, out, lse, workspace, workspace_bytes, status, opt,
+                    stream);
 }

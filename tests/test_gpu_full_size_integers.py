@@ -12,7 +12,7 @@ import torch
 import paper_2603_08088_b200 as tv
 from oracle import tree_verify_oracle as orc
 from workloads import CONFIGS, make_case, bf16_bits
-from gpu_util import i32
+from gpu_util import i32, f32, oracle_attention_slice, ATTN_ATOL
 
 pytestmark = pytest.mark.gpu
 
@@ -43,6 +43,17 @@ def test_full_size_step_integers_and_committed_bytes(ci):
     if not given_rows:
         assert np.array_equal(i32(buf.retrieve), mk["retrieve"]) and np.array_equal(i32(buf.n_paths), mk["n_paths"])
     rows = i32(d["retrieve"]) if given_rows else mk["retrieve"]
+
+    # ---- attention of the one launch that covers all layers: sampled (layer, sequence, KV head) slices against the
+    # oracle (its own mask), first and last layers included
+    G = cfg.Hq // cfg.Hkv
+    for (l, b, hk) in {(0, 0, 0), (cfg.L - 1, cfg.B - 1, cfg.Hkv - 1), (cfg.L // 2, cfg.B // 2, 3)}:
+        case_np = {"q": bf16_bits(d["q"][l:l + 1]), "k_cache": bf16_bits(k_before[l:l + 1]), "v_cache": bf16_bits(v_before[l:l + 1]),
+                   "k_tree": bf16_bits(d["k_tree"][l:l + 1]), "v_tree": bf16_bits(d["v_tree"][l:l + 1]),
+                   "prefix_len": S0, "n_nodes": n_nodes}
+        ref_out, _ = oracle_attention_slice(case_np, 0, b, hk, G, mk["dense"][:, 0], cfg.d ** -0.5)
+        got = f32(buf.out[l, b:b + 1, :, hk * G:(hk + 1) * G])
+        assert np.abs(got - ref_out).max() <= ATTN_ATOL, f"attention of layer {l}, sequence {b}, KV head {hk}"
 
     # ---- argmax over the full vocabulary, gather, acceptance
     am = orc.argmax_rows(bf16_bits(d["logits"]), n_nodes)

@@ -196,3 +196,49 @@ def test_paged_commit_flags():
     assert rst.tolist() == [orc.ST_CAPACITY, orc.ST_BAD_INDEX, orc.ST_BAD_INDEX, orc.ST_BAD_TREE]
     assert np.array_equal(i32(st), rst) and np.array_equal(i32(Sd), rS)
     assert np.array_equal(asu(kpd), rk) and np.array_equal(asu(vpd), rv) and np.array_equal(rk, asu(kp))
+
+
+def test_paged_layers_call_equals_layer_by_layer_calls():
+    """All layers over the paged cache in one launch (tree_verify_attn_paged_layers) against one
+    tree_verify_attn_paged call per layer (the units are cut at other places, so the two agree to the rounding of
+    the partials, not bit for bit) and against the oracle."""
+    cfg = CONFIGS[4].scaled(B=5, L=3, Hq=8, Hkv=2, S_lo=60, S_hi=900, Scap=1024, V=0)
+    case = make_case(cfg, seed=4400, ragged_nodes=True, with_logits=False)
+    dev = "cuda"
+    L, B, N, Hq, d = cfg.L, cfg.B, cfg.N, cfg.Hq, cfg.d
+    kps, vps, bt = [], [], None
+    for l in range(L):                                # one block table for all layers
+        kp, bt = to_pages(case["k_cache"][l], None, np.random.default_rng(5))
+        vp, _ = to_pages(case["v_cache"][l], None, np.random.default_rng(5))
+        kps.append(kp)
+        vps.append(vp)
+    k_pages, v_pages = torch.stack(kps).to(dev), torch.stack(vps).to(dev)
+    g = to_device(case)
+    btd = bt.to(dev)
+    bits = torch.zeros(B, N, (N + 31) // 32, dtype=torch.int32, device=dev)
+    status = torch.zeros(B, dtype=torch.int32, device=dev)
+    tv.tree_build_mask(g["parent"], g["n_nodes"], N - 1, 1, bits, status)
+    ws = torch.zeros(tv.tv_attn_workspace_bytes(B, N, Hq, cfg.Hkv, d, cfg.Scap), dtype=torch.uint8, device=dev)
+    one = torch.zeros(L, B, N, Hq, d, dtype=torch.bfloat16, device=dev)
+    lse_one = torch.zeros(L, B, Hq, N, dtype=torch.float32, device=dev)
+    for l in range(L):
+        tv.tree_verify_attn_paged(g["q"][l], k_pages[l], v_pages[l], btd, g["k_tree"][l], g["v_tree"][l], g["prefix_len"],
+                                  g["n_nodes"], bits, d ** -0.5, one[l], ws, status, lse=lse_one[l])
+    allq = torch.full_like(one, 3.0)
+    lse_all = torch.full_like(lse_one, 3.0)
+    tv.tree_verify_attn_paged_layers(g["q"], k_pages, v_pages, btd, g["k_tree"], g["v_tree"], g["prefix_len"], g["n_nodes"],
+                                     bits, d ** -0.5, allq, ws, status, lse=lse_all)
+    torch.cuda.synchronize()
+    assert (i32(status) == 0).all()
+    assert (allq.float() - one.float()).abs().max().item() <= 2.0 ** -7
+    both_inf = torch.isinf(lse_all) & torch.isinf(lse_one)
+    assert torch.equal(torch.isinf(lse_all), torch.isinf(lse_one))
+    assert torch.where(both_inf, torch.zeros_like(lse_all), lse_all - lse_one).abs().max().item() <= 1e-4
+    # and against the oracle, layer by layer
+    case_np = case_to_numpy(case)
+    vis = oracle_visibility(case["parent"], case["n_nodes"], bits_gpu=bits)
+    for l in range(L):
+        ref_out, ref_lse = orc.tree_attention(case_np["q"][l], case_np["k_cache"][l], case_np["v_cache"][l],
+                                              case_np["k_tree"][l], case_np["v_tree"][l], case_np["prefix_len"],
+                                              case_np["n_nodes"], vis[:, 0], d ** -0.5)
+        assert_attention_close(allq[l], lse_all[l], ref_out, ref_lse, f"layer {l}")
