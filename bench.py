@@ -362,33 +362,6 @@ def run_ours(args, cfg):
             graph_leg = {"error": f"{type(exc).__name__}: {exc}"[:200]}
             torch.cuda.synchronize()
 
-    # ---- the same step loop kept running for --sustain seconds (this rank's own clock): what the step costs once
-    # the board has reached its power limit, with the clocks seen over that region
-    sustained = None
-    if args.sustain > 0:
-        n_sus = max(args.steps, int(args.sustain / max(elapsed_ms / args.steps * 1e-3, 1e-6)) + 1)
-        every = max(1, n_sus // 64)                       # per-stage events on a subset of the steps
-        sm = {i: [ev() for _ in range(4)] for i in range(0, n_sus, every)}
-        sus_sampler = ClockSampler(local, period_s=0.02)
-        torch.cuda.synchronize()
-        sus_sampler.start()
-        s0, s1 = ev(), ev()
-        s0.record()
-        for i in range(n_sus):
-            one_step(sm.get(i))
-        s1.record()
-        torch.cuda.synchronize()
-        sus_clocks = sus_sampler.stop()
-        sus_ms = s0.elapsed_time(s1)
-        late = [m for i, m in sm.items() if i >= n_sus // 2]          # stages over the second half of the region
-        sustained = {"seconds": sus_ms * 1e-3, "steps": n_sus, "value": n_sus / (sus_ms * 1e-3), "unit": UNIT + " per GPU",
-                     "ms_per_step": sus_ms / n_sus,
-                     "attn_per_layer_us": sum(m[1].elapsed_time(m[2]) for m in late) / (len(late) * cfg.L) * 1e3,
-                     "accept_commit_us": sum(m[2].elapsed_time(m[3]) for m in late) / len(late) * 1e3,
-                     "clocks": sus_clocks}
-        if (buf.status.cpu().numpy() & 15).any():
-            raise SystemExit(f"bench.py: fatal status in the sustained run: {buf.status.cpu().numpy()}")
-
     # ---- multi-layer workloads: the same layers issued as L separate tree_verify_attn calls, back to back (what a
     # caller whose layers depend on each other has to issue: every call is a launch of its own with its own pipeline
     # fill, tail and merges, and reads nothing before the call in front has finished)
@@ -439,6 +412,37 @@ def run_ours(args, cfg):
         b2b_us = b0.elapsed_time(b1) / n_b2b * 1e3
         attn_b2b = {"launches": n_b2b, "us": b2b_us, "input_copies": n_sets}
 
+    # ---- the same step loop kept running for --sustain seconds (rank 0's own clock, run last so that no
+    # other leg is timed on a board that is still at its power limit): what the step costs once the board has
+    # reached that limit, with the clocks seen over the region
+    def run_sustained():
+        sustained = None
+        if args.sustain <= 0:
+            return None
+        n_sus = max(args.steps, int(args.sustain / max(elapsed_ms / args.steps * 1e-3, 1e-6)) + 1)
+        every = max(1, n_sus // 64)                       # per-stage events on a subset of the steps
+        sm = {i: [ev() for _ in range(4)] for i in range(0, n_sus, every)}
+        sus_sampler = ClockSampler(local, period_s=0.02)
+        torch.cuda.synchronize()
+        sus_sampler.start()
+        s0, s1 = ev(), ev()
+        s0.record()
+        for i in range(n_sus):
+            one_step(sm.get(i))
+        s1.record()
+        torch.cuda.synchronize()
+        sus_clocks = sus_sampler.stop()
+        sus_ms = s0.elapsed_time(s1)
+        late = [m for i, m in sm.items() if i >= n_sus // 2]          # stages over the second half of the region
+        sustained = {"seconds": sus_ms * 1e-3, "steps": n_sus, "value": n_sus / (sus_ms * 1e-3), "unit": UNIT + " per GPU",
+                     "ms_per_step": sus_ms / n_sus,
+                     "attn_per_layer_us": sum(m[1].elapsed_time(m[2]) for m in late) / (len(late) * cfg.L) * 1e3,
+                     "accept_commit_us": sum(m[2].elapsed_time(m[3]) for m in late) / len(late) * 1e3,
+                     "clocks": sus_clocks}
+        if (buf.status.cpu().numpy() & 15).any():
+            raise SystemExit(f"bench.py: fatal status in the sustained run: {buf.status.cpu().numpy()}")
+        return sustained
+
     if rank != 0:
         return
     peak, peak_kind = measured_peaks()
@@ -467,9 +471,6 @@ def run_ours(args, cfg):
     }
     if graph_leg is not None:
         line["graph_replay"] = graph_leg
-    if sustained is not None:
-        sustained["attn_hbm_frac"] = alg_bytes / (sustained["attn_per_layer_us"] * 1e-6) / 1e9 / peak
-        line["sustained"] = sustained
     if attn_single is not None:
         attn_single["hbm_gbs"] = alg_bytes / (attn_single["us_per_layer"] * 1e-6) / 1e9
         attn_single["frac"] = attn_single["hbm_gbs"] / peak
@@ -496,6 +497,10 @@ def run_ours(args, cfg):
         sec, desc, threads = oracle_sample_seconds(cfg, args.seed)
         line["cpu_baseline"] = {"value": 1.0 / sec, "unit": UNIT, "cores": threads, "kind": "oracle",
                                 "sample": desc, "est_seconds_per_step": sec}
+    sustained = run_sustained()
+    if sustained is not None:
+        sustained["attn_hbm_frac"] = alg_bytes / (sustained["attn_per_layer_us"] * 1e-6) / 1e9 / peak
+        line["sustained"] = sustained
     print(json.dumps(line))
 
 
