@@ -27,7 +27,8 @@
 // is fetched cold every time.  Cold paths are therefore written as loops, not
 // unrolled, and the timeline marks are compiled out unless -DTV_TRACE is given.
 //
-// Work split.  All key tiles of all (b, hk) units form one linear space that
+// Work split.  All key tiles of all (layer, b, hk) units of the launch - one
+// layer, or all layers of a step - form one linear space that
 // is cut evenly over the CTA groups (a group = the CTAs that hold the row
 // tiles of the same unit and walk the same keys together, so the second reader
 // hits L2).  A unit cut in pieces leaves partials (normalised O in bf16, m, l) in the
@@ -534,11 +535,11 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       tr.mark(0);
       uint64_t kv_policy;      // the committed prefix is streamed once: first in line for eviction from L2
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(kv_policy));
-      // Overlap with the kernel in front (programmatic dependent launch): the committed prefix, prefix_len and
-      // n_nodes are not written by a tree_verify_attn call, the one kernel that lets this one start early, so
-      // the first prefix tiles are requested at once; Q and the tree's K/V - what a preceding kernel may still
-      // be producing - wait for that kernel to finish.  Only then may the next kernel be scheduled, so that at
-      // most two launches are in flight and the two halves of the workspace suffice.
+      // Overlap with the kernel in front (programmatic dependent launch).  With the caller's promise (prm.early)
+      // that this kernel leaves prefix_len, n_nodes, the block table and the committed rows alone, the first
+      // prefix tiles are requested at once; Q and the tree's K/V - what a preceding kernel may still be
+      // producing - wait for that kernel to finish.  Only then may the next kernel be scheduled, so that at
+      // most two launches are in flight.
       // status[] may still be written by the kernel in front (tree_build_mask stores it last), so a flag found
       // before the wait is kept here and raised after it.
       bool synced = false;
