@@ -336,3 +336,47 @@ def test_attention_full_size_sampled_heads(ci, samples):
         err = np.abs(got_out[b:b + 1, :, hk * G:(hk + 1) * G] - ref_out).max()
         assert err <= ATTN_ATOL, f"(b={b}, hk={hk}): {err}"
         assert np.abs(got_lse[b:b + 1, hk * G:(hk + 1) * G] - ref_lse).max() <= 2e-3
+
+
+def test_layers_call_one_launch_many_layers_and_its_limits():
+    """tree_verify_attn_layers: all layers in one launch (as many as the workspace has counters for), against the
+    oracle layer by layer; the same call as one launch per layer agrees to the rounding of the partials."""
+    L = 35
+    cfg = CONFIGS[0].scaled(B=3, L=L, S_lo=0, S_hi=600, Scap=640, N=15, Hq=8, Hkv=2, V=0)
+    case = make_case(cfg, seed=77, ragged_nodes=True, with_logits=False)
+    d = to_device(case)
+    B, N, Hq, Hkv, dh = cfg.B, cfg.N, cfg.Hq, cfg.Hkv, cfg.d
+    bits = torch.zeros(B, N, 1, dtype=torch.int32, device="cuda")
+    status = torch.zeros(B, dtype=torch.int32, device="cuda")
+    tv.tree_build_mask(d["parent"], d["n_nodes"], N - 1, 1, bits, status)
+    need = tv.tv_attn_workspace_bytes(B, N, Hq, Hkv, dh, cfg.Scap)
+    ws = torch.zeros(need, dtype=torch.uint8, device="cuda")
+
+    def run(flags, workspace):
+        out = torch.full((L, B, N, Hq, dh), 3.0, dtype=torch.bfloat16, device="cuda")
+        lse = torch.full((L, B, Hq, N), 3.0, dtype=torch.float32, device="cuda")
+        n0 = tv.tv_launch_count()
+        tv.tree_verify_attn_layers(d["q"], d["k_cache"], d["v_cache"], d["k_tree"], d["v_tree"], d["prefix_len"],
+                                   d["n_nodes"], bits, dh ** -0.5, out, workspace, status, lse=lse, flags=flags)
+        torch.cuda.synchronize()
+        assert (status.cpu().numpy() == 0).all()
+        return out, lse, tv.tv_launch_count() - n0
+
+    out, lse, launches = run(tv.TV_ATTN_STABLE_INPUTS, ws)
+    assert launches == 2                                    # the workspace holds the counters of 32 layers
+    vis = oracle_visibility(case["parent"], case["n_nodes"], bits_gpu=bits)
+    cn = case_to_numpy(case)
+    for l in range(L):
+        ref_out, ref_lse = orc.tree_attention(cn["q"][l], cn["k_cache"][l], cn["v_cache"][l], cn["k_tree"][l],
+                                              cn["v_tree"][l], cn["prefix_len"], cn["n_nodes"], vis[:, 0], dh ** -0.5)
+        assert_attention_close(out[l], lse[l], ref_out, ref_lse, f"layer {l}")
+    out2, lse2, launches2 = run(tv.TV_ATTN_LAUNCH_PER_LAYER, ws)
+    assert launches2 == L
+    assert (out.float() - out2.float()).abs().max().item() <= 2.0 ** -5
+    # room for the counters of a single layer: still correct, one launch per layer
+    per_layer = (B * Hkv * 2 * 8 + 255) // 256 * 256
+    small = torch.zeros(need - 31 * per_layer, dtype=torch.uint8, device="cuda")
+    out3, lse3, launches3 = run(0, small)
+    assert launches3 == L and torch.equal(out3, out2) and torch.equal(lse3, lse2)
+    with pytest.raises(tv.TreeVerifyError):                 # not even one layer of counters
+        run(0, torch.zeros(need - 32 * per_layer, dtype=torch.uint8, device="cuda"))
