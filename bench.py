@@ -29,10 +29,11 @@ METRIC = "tree_verify_steps_per_sec"
 UNIT = "steps/s"
 # DRAM bytes per tree_verify_attn launch from ncu (dram__bytes_read.sum + dram__bytes_write.sum), as a ratio to
 # the algorithmic bytes.  Captured on gqa8b_ragged (161.8 MB / 160.1 MB) and long_context (549.0 MB / 547.4 MB),
-# see profiles/tree_attn_kernel_*.md; full_step_32l and llama7b_layer hold too much memory / too little work for
-# a full capture and take the ragged-batch ratio, since traffic grows with the same sum of (prefix + tree) keys.
+# see profiles/tree_attn_kernel_*.md; full_step_32l holds too much memory for a full capture and takes the ratio of
+# a 4-layer launch of its own shape (613.5 MB / 616.1 MB); llama7b_layer holds too little work for
+# a capture larger than L2 and takes the ragged-batch ratio; traffic grows with the sum of (prefix + tree) keys.
 L2_BYTES = 126 * 1024 * 1024
-NCU_TRAFFIC_RATIO = {"gqa8b_ragged": 1.010, "long_context": 1.003, "full_step_32l": 1.010, "llama7b_layer": 1.010}
+NCU_TRAFFIC_RATIO = {"gqa8b_ragged": 1.010, "long_context": 1.003, "full_step_32l": 0.996, "llama7b_layer": 1.010}
 
 
 def measured_peaks():
@@ -459,7 +460,8 @@ def run_ours(args, cfg):
         "metric": METRIC, "value": total_steps / (elapsed_ms * 1e-3), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": elapsed_ms / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": cfg.name, "B": cfg.B, "L": cfg.L, "N": cfg.N, "D": cfg.D, "Hq": cfg.Hq,
+        "config": {"workload": cfg.name + (f" with {cfg.L} layers" if args.layers > 0 else ""), "B": cfg.B, "L": cfg.L,
+                   "N": cfg.N, "D": cfg.D, "Hq": cfg.Hq,
                    "Hkv": cfg.Hkv, "d": cfg.d, "V": cfg.V, "prefix": [cfg.S_lo, cfg.S_hi],
                    "sum_prefix": int(S_host.sum()), "parallelism": f"sequence-sharded x{world}",
                    "l2": l2_note},
@@ -743,6 +745,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="full_step_32l", choices=[c.name for c in CONFIGS])
     ap.add_argument("--seed", type=int, default=4000)
+    ap.add_argument("--layers", type=int, default=0,
+                    help="override the workload's layer count (a smaller case of the same shape, e.g. for an ncu capture)")
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
     ap.add_argument("--budget-sweep", action="store_true",
                     help="also time tree_verify_attn over the node budgets of the paper's sweep (extra key in the JSON line)")
@@ -760,6 +764,8 @@ def main():
                     help="also time one member of an R-way context split of the workload (extra key in the JSON line)")
     args = ap.parse_args()
     cfg = get_config(args.workload)
+    if args.layers > 0:
+        cfg = cfg.scaled(L=args.layers)
     if args.impl == "reference":
         run_reference(args, cfg)
     else:
