@@ -471,10 +471,12 @@ def run_ours(args, cfg):
         "mean_accept_len": mean_accept,
         "roofline": {"bound": "hbm", "kernel": "tree_verify_attn", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
-                     "traffic": (int(NCU_TRAFFIC_RATIO[cfg.name] * alg_bytes) if cfg.name in NCU_TRAFFIC_RATIO else None),
+                     # one launch covers all cfg.L layers of the step
+                     "traffic": (int(NCU_TRAFFIC_RATIO[cfg.name] * alg_bytes * cfg.L) if cfg.name in NCU_TRAFFIC_RATIO else None),
                      "traffic_source": "ncu dram bytes, scaled by algorithmic bytes from the captured config",
-                     "algorithmic_bytes_per_launch": alg_bytes,
-                     "avg_launch_us": attn_ms * 1e3,
+                     "layers_per_launch": cfg.L,
+                     "algorithmic_bytes_per_launch": alg_bytes * cfg.L,
+                     "avg_launch_us": attn_ms * 1e3 * cfg.L,
                      "tensor_tflops": attn_flops(cfg, S_host) / (attn_ms * 1e-3) / 1e12},
         "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e,
     }
