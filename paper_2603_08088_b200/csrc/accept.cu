@@ -181,9 +181,17 @@ accept_kernel(const ArgPair* __restrict__ partial, int n_chunks,
     int tok = -1;
     if (i < n) {
       const ArgPair* pp = partial + ((size_t)b * Nmax + i) * n_chunks;
-      float bv = pp[0].val;
-      int bi = pp[0].idx;
-      for (int c = 1; c < n_chunks; ++c) take_better(bv, bi, pp[c].val, pp[c].idx);
+      float bv = -INFINITY;
+      int bi = 0x7fffffff;
+      for (int c0 = 0; c0 < n_chunks; c0 += 8) {       // eight pairs requested together, folded in chunk order
+        ArgPair p8[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+          if (c0 + k < n_chunks) p8[k] = pp[c0 + k];
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+          if (c0 + k < n_chunks) take_better(bv, bi, p8[k].val, p8[k].idx);
+      }
       tok = bi;
     }
     am[i] = tok;
