@@ -30,6 +30,9 @@ TV_API int tv_debug_attn_simt(const tv_bf16* q, const tv_bf16* k_cache, const tv
  * tree_verify_attn with the limit of every bounded wait inside the kernel set
  * to wait_limit_ns (the product uses 2 s).  mode bit 0: the producer warp
  * issues no copy at all, so the first wait of the MMA-issuing warp expires.
+ * mode bit 1: the pieces of units that are cut between CTAs store their
+ * partials but never announce them, so the poll of the piece that merges
+ * expires (a launch without a cut unit is then an ordinary launch).
  * The launch then ends by itself: every role leaves its loop, the tensor
  * memory is freed, and TV_ST_TIMEOUT is ORed into status[b] of every
  * sequence (out and lse are unspecified).  Nothing traps or faults; the next

@@ -328,7 +328,8 @@ struct AttnParams {
   int early;                     // the caller promises that the kernel in front leaves prefix_len, n_nodes, the block
                                  // table and the committed rows alone: they are read before the grid-dependency wait
   unsigned long long wait_limit_ns;   // limit of every bounded wait
-  int debug;                     // bit 0: the producer issues no copy at all (exercises the expiry of the waits)
+  int debug;                     // bit 0: the producer issues no copy at all; bit 1: pieces of cut units store their
+                                 // partials but never announce them (both exercise the expiry of a bounded wait)
   int L;                         // layers in this launch: their units form one tile space, layer after layer
   long long out_layer_stride;    // elements between the outputs of two layers (lse is dense, [L,B,Hq,Nmax])
 };
@@ -1199,7 +1200,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
               ok = epi_sync();
               if (!ok) break;
               TV_PROF_T(ep[5]);
-              if (threadIdx.x == 128) {
+              if (threadIdx.x == 128 && !(prm.debug & 2)) {      // (debug bit 1: the piece is never announced)
                 const unsigned long long seen = *reinterpret_cast<volatile unsigned long long*>(ctr + 1);
                 bump_counter(ctr + 1, seen, prm.epoch);
               }
@@ -1626,7 +1627,8 @@ extern "C" TV_API void tv_debug_set_attn_trace(unsigned long long* device_buffer
 }
 
 // Test aid for the failure path: tree_verify_attn with the limit of every bounded wait set to wait_limit_ns and,
-// with mode bit 0, a producer warp that issues no copy at all, so that the first wait of the MMA issuer expires.
+// with mode bit 0, a producer warp that issues no copy at all, so that the first wait of the MMA issuer expires;
+// with mode bit 1, pieces of cut units that never announce their partials, so that the poll of the merging piece expires.
 // The launch must then end by itself with TV_ST_TIMEOUT in status[] of every sequence and leave the GPU usable.
 extern "C" TV_API int tv_debug_attn_expire(const tv_bf16* q, const tv_bf16* k_cache, const tv_bf16* v_cache,
                                            const tv_bf16* k_tree, const tv_bf16* v_tree, const int32_t* prefix_len,
