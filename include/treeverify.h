@@ -110,7 +110,7 @@ enum {
                                  usual step) satisfies it; kv_commit in front does not. */
 };
 
-/* Scratch needed by tree_verify_attn for these dimensions (bytes). */
+/* Scratch needed by tree_verify_attn and tree_verify_attn_layers for these dimensions (bytes). */
 TV_API size_t tv_attn_workspace_bytes(int B, int Nmax, int Hq, int Hkv, int d, int Scap);
 
 /*
@@ -178,14 +178,21 @@ TV_API int tree_verify_attn(const tv_bf16* q,
  * the same mask and the same prefix lengths).  Layer l reads q, k_cache,
  * v_cache, k_tree, v_tree (both NULL: in-cache layout) at l times the given
  * layer stride (elements), writes out at l * out_layer_stride and lse (dense
- * [L,B,Hq,Nmax], or NULL).  Everything else is as for tree_verify_attn, which
- * this call equals layer by layer.
- * What it adds is launch overlap that a single call cannot take by itself:
- * the launch of layer l + 1 is scheduled while layer l drains and requests
- * its first committed-prefix tiles at once - inside one call the library
- * knows that the kernel in front is its own and leaves those inputs alone.
- * With TV_ATTN_STABLE_INPUTS in flags the caller extends that promise to the
- * kernel in front of the call, and layer 0 overlaps it too.
+ * [L,B,Hq,Nmax], or NULL).  Arguments, limits and results are those of
+ * tree_verify_attn, layer by layer (outputs agree with L single calls to the
+ * rounding of the split-KV partials: units are cut at other places).
+ * What it adds: the inputs of all layers are there when the call is made, so
+ * all layers run in ONE launch - their (sequence, KV head) units form one
+ * tile space that is cut evenly over the SMs - with one pipeline fill, one
+ * tail and at most one cut unit per SM for the whole step instead of per
+ * layer.  The workspace of tv_attn_workspace_bytes holds the counters of 32
+ * layers per launch; more layers (or a smaller workspace, down to the
+ * counters of one layer) are served by more launches.  A caller whose layers
+ * depend on each other has to issue single-layer calls instead.
+ * flags: TV_ATTN_STABLE_INPUTS lets the launch read prefix_len, n_nodes and
+ * committed-prefix rows while the kernel in front still runs (see the flag);
+ * TV_ATTN_LAUNCH_PER_LAYER issues one launch per layer, as L single calls
+ * would (for comparison).
  */
 TV_API int tree_verify_attn_layers(const tv_bf16* q,
                      const tv_bf16* k_cache, const tv_bf16* v_cache,
