@@ -110,6 +110,32 @@ def attn_flops(cfg, prefix_len):
     return 4 * cfg.Hq * cfg.N * cfg.d * keys
 
 
+def input_copies(cfg):
+    """(copies of a step's inputs that are used in turn, bytes of one copy, note for the JSON line).  A step whose
+    inputs fit the 126 MB L2 would be timed L2-warm: such workloads cycle through copies of the big inputs (same
+    values, distinct memory), enough of them to exceed L2 between two uses of one copy."""
+    e = 2
+    per_layer = cfg.B * (cfg.N * cfg.Hq * cfg.d + 2 * cfg.N * cfg.Hkv * cfg.d + 2 * cfg.Hkv * cfg.Scap * cfg.d)   # q, tree K/V, cache
+    step_bytes = e * (cfg.L * per_layer + cfg.B * cfg.N * cfg.V)                                                  # + logits
+    n_sets = 1 if step_bytes > 2 * L2_BYTES else min(8, int(2 * L2_BYTES // max(step_bytes, 1)) + 2)
+    if n_sets == 1:
+        note = "inputs larger than L2 (each step streams the whole KV cache and the logits)"
+    elif n_sets * step_bytes > L2_BYTES:
+        note = (f"{n_sets} copies of the inputs ({step_bytes / 1e6:.0f} MB each) used in turn, so that a copy has left "
+                "L2 before it is read again")
+    else:
+        note = (f"L2-resident: {n_sets} copies of the inputs ({step_bytes / 1e6:.2f} MB each) used in turn still fit L2; "
+                "a launch-latency-scale workload")
+    return n_sets, step_bytes, note
+
+
+def workload_config(cfg, world, sum_prefix, layers_overridden):
+    """The `config` object of the JSON line: the workload, the same on both arms."""
+    return {"workload": cfg.name + (f" with {cfg.L} layers" if layers_overridden else ""), "B": cfg.B, "L": cfg.L,
+            "N": cfg.N, "D": cfg.D, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "d": cfg.d, "V": cfg.V, "prefix": [cfg.S_lo, cfg.S_hi],
+            "sum_prefix": int(sum_prefix), "parallelism": f"sequence-sharded x{world}", "l2": input_copies(cfg)[2]}
+
+
 # --------------------------------------------------------------------------- oracle legs
 def oracle_sample_seconds(cfg, seed):
     """Times the CPU oracle, as it stands, on a bounded sample of the workload and
@@ -183,8 +209,10 @@ def run_reference(args, cfg):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": len(ests), "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": cfg.name, "B": cfg.B, "L": cfg.L, "N": cfg.N, "Hq": cfg.Hq, "Hkv": cfg.Hkv,
-                   "d": cfg.d, "V": cfg.V, "prefix": [cfg.S_lo, cfg.S_hi]},
+        # the same workload object as the CUDA arm prints (prefix lengths of the same seed; no cache is drawn for it)
+        "config": workload_config(cfg, int(os.environ.get("WORLD_SIZE", "1")),
+                                  make_case(cfg.scaled(L=1), args.seed, device="cpu", with_cache=False,
+                                            with_logits=False)["prefix_len"].sum().item(), args.layers > 0),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -214,17 +242,9 @@ def run_ours(args, cfg):
     # A step whose inputs fit the 126 MB L2 would be timed L2-warm: such workloads cycle through copies of the big
     # inputs (same values, distinct memory), enough of them to exceed L2 between two uses of one copy.
     big = ("q", "k_cache", "v_cache", "k_tree", "v_tree") + (("logits",) if has_accept else ())
-    step_bytes = sum(case[k].numel() * case[k].element_size() for k in big)
-    n_sets = 1 if step_bytes > 2 * L2_BYTES else min(8, int(2 * L2_BYTES // max(step_bytes, 1)) + 2)
+    n_sets, step_bytes, l2_note = input_copies(cfg)
+    assert step_bytes == sum(case[k].numel() * case[k].element_size() for k in big)
     sets = [case] + [dict(case, **{k: case[k].clone() for k in big}) for _ in range(n_sets - 1)]
-    if n_sets == 1:
-        l2_note = "inputs larger than L2 (each step streams the whole KV cache and the logits)"
-    elif n_sets * step_bytes > L2_BYTES:
-        l2_note = (f"{n_sets} copies of the inputs ({step_bytes / 1e6:.0f} MB each) used in turn, so that a copy has left "
-                   "L2 before it is read again")
-    else:
-        l2_note = (f"L2-resident: {n_sets} copies of the inputs ({step_bytes / 1e6:.2f} MB each) used in turn still fit L2; "
-                   "a launch-latency-scale workload")
     step_no = [0]
 
     def rest():
@@ -460,11 +480,7 @@ def run_ours(args, cfg):
         "metric": METRIC, "value": total_steps / (elapsed_ms * 1e-3), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": elapsed_ms / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": cfg.name + (f" with {cfg.L} layers" if args.layers > 0 else ""), "B": cfg.B, "L": cfg.L,
-                   "N": cfg.N, "D": cfg.D, "Hq": cfg.Hq,
-                   "Hkv": cfg.Hkv, "d": cfg.d, "V": cfg.V, "prefix": [cfg.S_lo, cfg.S_hi],
-                   "sum_prefix": int(S_host.sum()), "parallelism": f"sequence-sharded x{world}",
-                   "l2": l2_note},
+        "config": workload_config(cfg, world, S_host.sum(), args.layers > 0),
         "sequence_steps_per_sec": total_steps * cfg.B / (elapsed_ms * 1e-3),
         "stage_us": {"mask": mask_us, "attn_per_layer": attn_ms * 1e3, "accept_commit": tail_us},
         "step_ms": {"median": per_step_ms[len(per_step_ms) // 2], "min": per_step_ms[0], "max": per_step_ms[-1]},
