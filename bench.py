@@ -440,8 +440,8 @@ def run_ours(args, cfg):
         b2b_us = b0.elapsed_time(b1) / n_b2b * 1e3
         attn_b2b = {"launches": n_b2b, "us": b2b_us, "input_copies": n_sets}
 
-    # ---- the same step loop kept running for --sustain seconds (rank 0's own clock, run last so that no
-    # other leg is timed on a board that is still at its power limit): what the step costs once the board has
+    # ---- the same step loop kept running for --sustain seconds (this rank's own clock; the legs that
+    # are timed on their own come before it or rest first): what the step costs once the board has
     # reached that limit, with the clocks seen over the region
     def run_sustained():
         sustained = None
@@ -470,6 +470,8 @@ def run_ours(args, cfg):
         if (buf.status.cpu().numpy() & 15).any():
             raise SystemExit(f"bench.py: fatal status in the sustained run: {buf.status.cpu().numpy()}")
         return sustained
+
+    sustained = run_sustained()       # every rank, so that the ranks stay together; the legs behind it rest first
 
     if rank != 0:
         return
@@ -527,7 +529,6 @@ def run_ours(args, cfg):
         sec, desc, threads = oracle_sample_seconds(cfg, args.seed)
         line["cpu_baseline"] = {"value": 1.0 / sec, "unit": UNIT, "cores": threads, "kind": "oracle",
                                 "sample": desc, "est_seconds_per_step": sec}
-    sustained = run_sustained()
     if sustained is not None:
         sustained["attn_hbm_frac"] = alg_bytes / (sustained["attn_per_layer_us"] * 1e-6) / 1e9 / peak
         line["sustained"] = sustained
