@@ -52,8 +52,9 @@ argmax_scan_kernel(const tv_bf16* __restrict__ logits, const int32_t* __restrict
   tv::pdl_enter();
   const int tid = threadIdx.x;
   const bool vec_ok = ((V & 7) == 0) && ((reinterpret_cast<uintptr_t>(logits) & 15u) == 0);
-  __shared__ float sv[kScanThreads / 32];
-  __shared__ int si[kScanThreads / 32];
+  __shared__ float sv[2][kScanThreads / 32];      // two sets, taken in turn: one barrier per item suffices
+  __shared__ int si[2][kScanThreads / 32];
+  int set = 0;
   const uint4 kLowest = make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);     // bf16 -inf
 
   // item -> (row, chunk, active); padded rows are never read
@@ -134,18 +135,18 @@ argmax_scan_kernel(const tv_bf16* __restrict__ logits, const int32_t* __restrict
         take_better(best, best_i, ov, oi);
       }
       if ((tid & 31) == 0) {
-        sv[tid >> 5] = best;
-        si[tid >> 5] = best_i;
+        sv[set][tid >> 5] = best;
+        si[set][tid >> 5] = best_i;
       }
       __syncthreads();
       if (tid == 0) {
-        for (int w = 1; w < kScanThreads / 32; ++w) take_better(best, best_i, sv[w], si[w]);
+        for (int w = 1; w < kScanThreads / 32; ++w) take_better(best, best_i, sv[set][w], si[set][w]);
         ArgPair out;
         out.val = best;
         out.idx = best_i;
         partial[(size_t)row * n_chunks + chunk] = out;
       }
-      __syncthreads();       // sv / si are reused by the next item
+      set ^= 1;              // the next item writes the other set; this one is rewritten only after the next barrier
     }
     item = nitem;
     row = nrow;
