@@ -421,6 +421,32 @@ def run_ours(args, cfg):
         torch.cuda.synchronize()
         attn_single = {"calls": reps * cfg.L, "us_per_layer": c0.elapsed_time(c1) / (reps * cfg.L) * 1e3}
 
+    # ---- the kernel's memory side alone (test entry point of treeverify_debug.h): the same launch, schedule and TMA
+    # copies, every shared-memory slot handed back as soon as it has landed, no MMA, no softmax, no output
+    stream_only = None
+    if True:                       # every rank, like the legs around it, so that the ranks stay together
+        rest()
+        for c in sets:
+            c["prefix_len"].copy_(prefix0)
+
+        def stream_pass(i):
+            c = sets[i % n_sets]
+            tv.tv_debug_attn_stream_only(c["q"], c["k_cache"], c["v_cache"], c["k_tree"], c["v_tree"], c["prefix_len"],
+                                         c["n_nodes"], buf.anc_bits, buf.out, buf.attn_ws, buf.status)
+
+        n_so = 5 if cfg.L > 1 else 120
+        for i in range(3):
+            stream_pass(i)
+        torch.cuda.synchronize()
+        s0, s1 = ev(), ev()
+        s0.record()
+        for i in range(n_so):
+            stream_pass(i)
+        s1.record()
+        torch.cuda.synchronize()
+        stream_only = {"calls": n_so, "us_per_layer": s0.elapsed_time(s1) / (n_so * cfg.L) * 1e3,
+                       "note": "tv_debug_attn_stream_only: the launch's K/V stream with nothing computed"}
+
     # ---- one-layer workloads: the attention launches alone, back to back on one stream (the step loop above is
     # bound by the host's launch path when a step is a handful of short kernels); inputs cycle through the copies
     attn_b2b = None
@@ -515,6 +541,10 @@ def run_ours(args, cfg):
         attn_single["hbm_gbs"] = alg_bytes / (attn_single["us_per_layer"] * 1e-6) / 1e9
         attn_single["frac"] = attn_single["hbm_gbs"] / peak
         line["attn_single_call"] = attn_single
+    if stream_only is not None:
+        stream_only["hbm_gbs"] = alg_bytes / (stream_only["us_per_layer"] * 1e-6) / 1e9
+        stream_only["frac"] = stream_only["hbm_gbs"] / peak
+        line["attn_stream_only"] = stream_only
     if attn_b2b is not None:
         attn_b2b["hbm_gbs"] = alg_bytes / (attn_b2b["us"] * 1e-6) / 1e9
         attn_b2b["frac"] = attn_b2b["hbm_gbs"] / peak

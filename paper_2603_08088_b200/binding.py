@@ -103,6 +103,10 @@ def load():
         lib.tv_debug_attn_expire.restype = _c_int
         lib.tv_debug_attn_expire.argtypes = ([_c_vp] * 8 + [_c_int] * 6 + [_c_f, _c_vp, _c_vp, _c_vp, _c_sz, _c_vp,
                                               ctypes.c_ulonglong, _c_int, _c_vp])
+    if hasattr(lib, "tv_debug_attn_stream_only"):
+        lib.tv_debug_attn_stream_only.restype = _c_int
+        lib.tv_debug_attn_stream_only.argtypes = ([_c_vp] * 8 + [_c_int] * 7 + [_c_i64] * 3 + [_c_vp, _c_i64, _c_vp, _c_sz,
+                                                   _c_vp, _c_vp])
     if hasattr(lib, "tv_debug_attn_simt"):
         lib.tv_debug_attn_simt.restype = _c_int
         lib.tv_debug_attn_simt.argtypes = [_c_vp] * 8 + [_c_int] * 6 + [_c_f, _c_vp, _c_vp, _c_vp]
@@ -215,6 +219,19 @@ def tv_debug_attn_expire(q, k_cache, v_cache, k_tree, v_tree, prefix_len, n_node
                                        float(scale), _ptr(out), _ptr(lse), _ptr(workspace),
                                        workspace.numel() * workspace.element_size(), _ptr(status), int(wait_limit_ns),
                                        int(mode), _stream(stream)))
+
+
+def tv_debug_attn_stream_only(q, k_cache, v_cache, k_tree, v_tree, prefix_len, n_nodes, anc_bits, out, workspace, status,
+                              stream=None):
+    """Tuning aid (treeverify_debug.h): the K/V stream of tree_verify_attn_layers alone - same launch, schedule and
+    copies, no MMA, no softmax, no output.  Shapes as in tree_verify_attn_layers."""
+    L, B, Nmax, Hq, d = q.shape
+    _, _, Hkv, Scap, _ = k_cache.shape
+    _check(load().tv_debug_attn_stream_only(q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(), k_tree.data_ptr(),
+                                            v_tree.data_ptr(), _ptr(prefix_len), _ptr(n_nodes), _ptr(anc_bits), L, B, Nmax,
+                                            Hq, Hkv, d, Scap, q.stride(0), k_cache.stride(0), k_tree.stride(0),
+                                            out.data_ptr(), out.stride(0), _ptr(workspace),
+                                            workspace.numel() * workspace.element_size(), _ptr(status), _stream(stream)))
 
 
 def tv_debug_attn_simt(q, k_cache, v_cache, k_tree, v_tree, prefix_len, n_nodes, anc_bits, scale, out,

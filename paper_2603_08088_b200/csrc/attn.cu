@@ -329,7 +329,9 @@ struct AttnParams {
                                  // table and the committed rows alone: they are read before the grid-dependency wait
   unsigned long long wait_limit_ns;   // limit of every bounded wait
   int debug;                     // bit 0: the producer issues no copy at all; bit 1: pieces of cut units store their
-                                 // partials but never announce them (both exercise the expiry of a bounded wait)
+                                 // partials but never announce them (both exercise the expiry of a bounded wait);
+                                 // bit 2: the K/V stream alone - the issuing warp only hands every slot back as
+                                 // soon as it is full, no MMA, no softmax, no output (what the memory side can do)
   int L;                         // layers in this launch: their units form one tile space, layer after layer
   long long out_layer_stride;    // elements between the outputs of two layers (lse is dense, [L,B,Hq,Nmax])
 };
@@ -689,6 +691,20 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         ok = mbar_wait(bar(L::Q_FULL), item_idx & 1, abort_flag, wait_limit);
         if (!ok) break;
         tr.mark(0x1000u | item_idx);
+        if (prm.debug & 4) {       // stream only: every tile of the item is released as soon as it has landed
+#pragma unroll 1
+          for (int f = 0; f < 2 * nt && ok; ++f) {
+            const uint32_t ff = fill + f;
+            ok = mbar_wait(bar(L::KV_FULL + ff % kSlots), (ff / kSlots) & 1, abort_flag, wait_limit);
+            if (ok && elect_one()) mbar_arrive(bar(L::KV_EMPTY + ff % kSlots));
+            __syncwarp();
+          }
+          if (elect_one()) mbar_arrive(bar(L::Q_EMPTY));
+          __syncwarp();
+          fill += 2 * nt;
+          ++item_idx;
+          continue;
+        }
         {
           const uint32_t slot = fill % kSlots;
           ok = mbar_wait(bar(L::KV_FULL + slot), (fill / kSlots) & 1, abort_flag, wait_limit);
@@ -775,7 +791,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         S = S < 0 ? 0 : (S > prm.Scap ? prm.Scap : S);
         if (S + prm.n_nodes[b] > prm.Scap) atomicOr(prm.status + b, TV_ST_CAPACITY);
       }
-    if (wg_active && !*abort_flag) {
+    if (wg_active && !*abort_flag && !(prm.debug & 4)) {
       int g = g_begin;
       Item it;
       uint32_t fill = 0, tj = 0, epi_phase = 0, item_cnt = 0;   // tj: key tiles handled so far (all items)
@@ -1641,6 +1657,28 @@ extern "C" TV_API int tv_debug_attn_expire(const tv_bf16* q, const tv_bf16* k_ca
   opt.debug = mode;
   return attn_entry(q, k_cache, v_cache, nullptr, 0, 0, k_tree, v_tree, prefix_len, n_nodes, anc_bits, 1, LayerStrides{}, B,
                     Nmax, Hq, Hkv, d, Scap, scale, out, lse, workspace, workspace_bytes, status, opt, stream);
+}
+
+extern "C" TV_API int tv_debug_attn_stream_only(const tv_bf16* q, const tv_bf16* k_cache, const tv_bf16* v_cache,
+                                                const tv_bf16* k_tree, const tv_bf16* v_tree, const int32_t* prefix_len,
+                                                const int32_t* n_nodes, const uint32_t* anc_bits, int L, int B, int Nmax,
+                                                int Hq, int Hkv, int d, int Scap, int64_t q_layer_stride,
+                                                int64_t cache_layer_stride, int64_t tree_layer_stride, tv_bf16* out,
+                                                int64_t out_layer_stride, void* workspace, size_t workspace_bytes,
+                                                int32_t* status, tv_stream stream) {
+  TV_REQUIRE(L >= 0 && L <= 65535, "tv_debug_attn_stream_only: need 0 <= L <= 65535");
+  TV_REQUIRE(q_layer_stride % 8 == 0 && cache_layer_stride % 8 == 0 && tree_layer_stride % 8 == 0 && out_layer_stride % 8 == 0,
+             "tv_debug_attn_stream_only: layer strides must be multiples of 8 elements");
+  AttnOptions opt;
+  opt.early = true;
+  opt.debug = 4;
+  LayerStrides ls;
+  ls.q = q_layer_stride;
+  ls.cache = cache_layer_stride;
+  ls.tree = tree_layer_stride;
+  ls.out = out_layer_stride;
+  return attn_entry(q, k_cache, v_cache, nullptr, 0, 0, k_tree, v_tree, prefix_len, n_nodes, anc_bits, L, ls, B, Nmax, Hq,
+                    Hkv, d, Scap, 1.0f, out, nullptr, workspace, workspace_bytes, status, opt, stream);
 }
 
 extern "C" size_t tv_attn_workspace_bytes(int B, int Nmax, int Hq, int Hkv, int d, int Scap) {

@@ -31,7 +31,8 @@ def test_header_symbols_are_exported(lib):
         assert hasattr(lib, n), f"{n} declared in treeverify.h but not exported"
     assert set(names) == set(tv.EXPORTS)
     debug = _declared_symbols("treeverify_debug.h")            # test and tuning aids: declared apart, exported too
-    assert set(debug) == {"tv_debug_attn_simt", "tv_debug_attn_expire", "tv_debug_set_attn_trace"}
+    assert set(debug) == {"tv_debug_attn_simt", "tv_debug_attn_expire", "tv_debug_attn_stream_only",
+                          "tv_debug_set_attn_trace"}
     for n in debug:
         assert hasattr(lib, n), f"{n} declared in treeverify_debug.h but not exported"
     assert not set(debug) & set(names)
