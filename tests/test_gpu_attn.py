@@ -91,6 +91,52 @@ def test_attention_parity_small(name, ci, over, simt):
             assert np.isneginf(f32(lse)[b, :, n[b]:]).all()
 
 
+GROUPS = [
+    # (query heads per KV head, KV heads, nodes, d): group sizes that do not divide the 128-row tile leave rows of
+    # every tile unused (128 // G nodes per tile), and large groups put few nodes into a tile
+    (3, 2, 50, 128), (5, 1, 30, 128), (6, 2, 64, 64), (7, 4, 26, 128), (12, 1, 21, 128), (24, 1, 11, 64),
+    (128, 1, 3, 128), (7, 1, 129, 128),
+]
+
+
+@pytest.mark.parametrize("G,Hkv,N,d", GROUPS, ids=[f"G{g}_kv{h}_N{n}_d{d}" for g, h, n, d in GROUPS])
+def test_group_sizes_that_do_not_divide_the_row_tile(G, Hkv, N, d):
+    cfg = CONFIGS[0].scaled(B=3, Hq=G * Hkv, Hkv=Hkv, d=d, S_lo=0, S_hi=700, Scap=1024, N=N, D=min(6, N - 1), V=0,
+                            tree="uniform")
+    case = make_case(cfg, seed=4200 + G, ragged_nodes=True, with_logits=False)
+    dcase = to_device(case)
+    case_np = case_to_numpy(case)
+    n = case["n_nodes"].numpy()
+    out, lse, bits, dense = gpu_attention(dcase, 0)
+    ref_out, ref_lse = oracle_attention(case_np, dense.cpu().numpy(), 0)
+    assert_attention_close(out, lse, ref_out, ref_lse, f"G={G}")
+    got = f32(out)
+    for b in range(cfg.B):
+        assert (got[b, n[b]:] == 0).all()
+    # all layers in one launch and the paged layout walk the same row tiles
+    L = 2
+    cfg2 = cfg.scaled(L=L)
+    case2 = make_case(cfg2, seed=4300 + G, ragged_nodes=True, with_logits=False)
+    g2 = to_device(case2)
+    B, Hq = cfg.B, cfg.Hq
+    bits2 = torch.zeros(B, N, (N + 31) // 32, dtype=torch.int32, device="cuda")
+    st = torch.zeros(B, dtype=torch.int32, device="cuda")
+    tv.tree_build_mask(g2["parent"], g2["n_nodes"], N - 1, 1, bits2, st)
+    ws = torch.zeros(max(256, tv.tv_attn_workspace_bytes(B, N, Hq, Hkv, d, cfg.Scap)), dtype=torch.uint8, device="cuda")
+    out2 = torch.full((L, B, N, Hq, d), 3.0, dtype=torch.bfloat16, device="cuda")
+    lse2 = torch.zeros(L, B, Hq, N, device="cuda")
+    tv.tree_verify_attn_layers(g2["q"], g2["k_cache"], g2["v_cache"], g2["k_tree"], g2["v_tree"], g2["prefix_len"],
+                               g2["n_nodes"], bits2, d ** -0.5, out2, ws, st, lse=lse2)
+    torch.cuda.synchronize()
+    assert (st.cpu().numpy() == 0).all()
+    vis = oracle_visibility(case2["parent"], case2["n_nodes"], bits_gpu=bits2)
+    cn = case_to_numpy(case2)
+    for l in range(L):
+        r_out, r_lse = orc.tree_attention(cn["q"][l], cn["k_cache"][l], cn["v_cache"][l], cn["k_tree"][l], cn["v_tree"][l],
+                                          cn["prefix_len"], cn["n_nodes"], vis[:, 0], d ** -0.5)
+        assert_attention_close(out2[l], lse2[l], r_out, r_lse, f"G={G}, layer {l}")
+
+
 BUDGETS = [(16, 10), (32, 10), (64, 4), (64, 16), (128, 10), (200, 12), (256, 10), (256, 16)]
 
 
