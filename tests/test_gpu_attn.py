@@ -137,6 +137,28 @@ def test_group_sizes_that_do_not_divide_the_row_tile(G, Hkv, N, d):
         assert_attention_close(out2[l], lse2[l], r_out, r_lse, f"G={G}, layer {l}")
 
 
+@pytest.mark.parametrize("B", [33, 70, 512])
+def test_many_sequences_up_to_the_maximum(B):
+    """The schedule table is built 32 sequences at a time and searched per work item; the library takes up to
+    512 sequences.  Short ragged sequences, so that most CTAs walk many units."""
+    cfg = CONFIGS[0].scaled(B=B, Hq=4, Hkv=2, d=64, S_lo=0, S_hi=300, Scap=384, N=9, D=4, V=0, tree="uniform")
+    case = make_case(cfg, seed=9000 + B, ragged_nodes=True, with_logits=False)
+    dcase = to_device(case)
+    out, lse, bits, dense = gpu_attention(dcase, 0)
+    ref_out, ref_lse = oracle_attention(case_to_numpy(case), dense.cpu().numpy(), 0)
+    assert_attention_close(out, lse, ref_out, ref_lse, f"B={B}")
+    if B == 512:                # one more sequence is refused, nothing is launched
+        big = CONFIGS[0].scaled(B=513, Hq=4, Hkv=2, d=64, S_lo=0, S_hi=10, Scap=128, N=9, D=4, V=0, tree="uniform")
+        g = to_device(make_case(big, seed=1, with_logits=False))
+        ws = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
+        st = torch.zeros(513, dtype=torch.int32, device="cuda")
+        o = torch.zeros(513, 9, 4, 64, dtype=torch.bfloat16, device="cuda")
+        b513 = torch.zeros(513, 9, 1, dtype=torch.int32, device="cuda")
+        with pytest.raises(tv.TreeVerifyError):
+            tv.tree_verify_attn(g["q"][0], g["k_cache"][0], g["v_cache"][0], g["k_tree"][0], g["v_tree"][0], g["prefix_len"],
+                                g["n_nodes"], b513, 0.125, o, ws, st)
+
+
 BUDGETS = [(16, 10), (32, 10), (64, 4), (64, 16), (128, 10), (200, 12), (256, 10), (256, 16)]
 
 
