@@ -157,6 +157,32 @@ def test_commit_bytes_exact(d, Hkv):
     assert st.tolist() == [orc.ST_CAPACITY, 0, orc.ST_BAD_INDEX, orc.ST_BAD_INDEX, orc.ST_CAPACITY]
 
 
+def test_many_sequences_accept_and_commit_at_the_row_limit():
+    """tree_accept takes up to 65535 (sequence, node) rows: 512 sequences of 127 slots here, ragged, a small
+    vocabulary; the commit behind it moves the accepted rows of all 512 sequences.  One row more is refused."""
+    B, N, V = 512, 127, 301
+    cfg = CONFIGS[0].scaled(B=B, N=N, D=5, V=V, S_lo=1, S_hi=8, Scap=32, L=1, Hq=2, Hkv=1, d=64, tree="uniform")
+    case = make_case(cfg, seed=31337, ragged_nodes=True, with_cache=False)
+    got, ref = check_accept(case["logits"], case["tokens"], case["retrieve"], case["n_nodes"])
+    assert (ref["accept_len"] > 0).any()
+    # commit of those paths: L = 2 layers, every byte
+    rng = np.random.default_rng(5)
+    L, Hkv, d, Scap, Dp1 = 2, 1, 64, 24, case["retrieve"].shape[2]
+    u16 = lambda *s: rng.integers(0, 2 ** 16, size=s).astype(np.uint16)
+    case_np = dict(k_cache=u16(L, B, Hkv, Scap, d), v_cache=u16(L, B, Hkv, Scap, d),
+                   k_tree=u16(L, B, N, Hkv, d), v_tree=u16(L, B, N, Hkv, d))
+    S = rng.integers(0, Scap - Dp1, size=B).astype(np.int32)
+    kc, vc, S2, st = gpu_commit(case_np, ref["accepted_nodes"], ref["accept_len"], S, ref["status"])
+    rk, rv, rS, rst = orc.kv_commit(case_np["k_cache"], case_np["v_cache"], case_np["k_tree"], case_np["v_tree"],
+                                    ref["accepted_nodes"], ref["accept_len"], S, ref["status"])
+    assert np.array_equal(kc, rk) and np.array_equal(vc, rv) and np.array_equal(S2, rS) and np.array_equal(st, rst)
+    # 512 x 128 = 65536 rows: refused before anything is launched
+    z = lambda *sh: torch.zeros(sh, dtype=torch.int32, device="cuda")
+    with pytest.raises(tv.TreeVerifyError):
+        tv.tree_accept(torch.zeros(B, 128, 8, dtype=torch.bfloat16, device="cuda"), z(B, 128), z(B, 1, 2), z(B), z(B, 128), z(B),
+                       z(B), z(B, 2), z(B), torch.zeros(1 << 20, dtype=torch.uint8, device="cuda"), z(B))
+
+
 def test_node_scores_parity():
     """tree_node_scores against the oracle: bit-exact fp32 values of the gathered bf16 logits."""
     cfg = CONFIGS[4].scaled(S_lo=1, S_hi=8, Scap=32, L=1, B=6, V=153600)
