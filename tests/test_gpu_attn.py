@@ -159,6 +159,24 @@ def test_many_sequences_up_to_the_maximum(B):
                                 g["n_nodes"], b513, 0.125, o, ws, st)
 
 
+@pytest.mark.parametrize("d,G", [(128, 4), (64, 1), (128, 8)])
+def test_prefix_lengths_on_and_around_tile_boundaries(d, G):
+    """Prefixes of 0, 127, 128, 129, 255, 256, 257 keys and one that fills the cache to its last row: the ragged
+    last prefix tile has 127, 0 (it does not exist), 1 ... valid keys.  Rows behind each prefix hold NaN."""
+    S = np.array([0, 127, 128, 129, 255, 256, 257, 512], dtype=np.int32)
+    B, Scap, N = len(S), 512, 33
+    cfg = CONFIGS[0].scaled(B=B, Hq=2 * G, Hkv=2, d=d, S_lo=0, S_hi=Scap, Scap=Scap, N=N, D=6, V=0, tree="uniform")
+    case = make_case(cfg, seed=777 + d + G, ragged_nodes=True, with_logits=False)
+    case["prefix_len"] = torch.from_numpy(S.copy())
+    nan = torch.tensor(float("nan"), dtype=torch.bfloat16)
+    for b in range(B):
+        case["k_cache"][:, b, :, S[b]:] = nan
+        case["v_cache"][:, b, :, S[b]:] = nan
+    out, lse, bits, dense = gpu_attention(to_device(case), 0)
+    ref_out, ref_lse = oracle_attention(case_to_numpy(case), dense.cpu().numpy(), 0)
+    assert_attention_close(out, lse, ref_out, ref_lse, f"d={d} G={G}")
+
+
 BUDGETS = [(16, 10), (32, 10), (64, 4), (64, 16), (128, 10), (200, 12), (256, 10), (256, 16)]
 
 
