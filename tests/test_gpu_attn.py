@@ -259,19 +259,25 @@ MOVES = [
     ("first_tile_of_the_item_second_half", 100, 8, 80),
     ("tree_tile_second_half", 40, 128, 40 + 100),
     ("whole_tile_then_ragged_tile", 370, 8, 340),
+    # full, unmasked prefix tiles: the fast path's row-sum check has to reject the tile and the careful path redo it
+    ("full_tile_first_half", 600, 8, 260),
+    ("full_tile_second_half", 600, 8, 350),
+    ("opening_tile_early_key", 600, 8, 5),
+    ("opening_tile_late_key", 600, 8, 120),
+    ("last_full_tile_last_key", 640, 8, 639),
 ]
 
 
 @pytest.mark.parametrize("name,S,N,big", MOVES, ids=[m[0] for m in MOVES])
 @pytest.mark.parametrize("d", [64, 128])
-def test_reference_maximum_moving_inside_a_masked_tile(name, S, N, big, d):
+def test_reference_maximum_moving_inside_a_tile(name, S, N, big, d):
     """The softmax keeps a lazy reference maximum and rescales only when the maximum grows by more than 2^8.
     Masked key tiles are worked through in two halves of 64 keys; here one key in the SECOND half of such a
     tile scores 2^12 above everything before it, so the reference moves after the first half has already
     produced its probabilities: they have to move with it.  All other scores are 0, so every visible key
     before the dominant one has weight 1 and that one 2^12.2: the output is a known mixture."""
     parent = chain_tree(N)                          # node i sees nodes 0..i: tree key j is visible to rows >= j
-    case = _tree_case(parent, S, 2, 1, d, 384, seed=S + N)
+    case = _tree_case(parent, S, 2, 1, d, 384 if S < 384 else 768, seed=S + N)
     case["k_cache"].zero_()
     case["k_tree"].zero_()
     case["q"].fill_(1.0)
