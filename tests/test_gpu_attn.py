@@ -265,6 +265,9 @@ MOVES = [
     ("opening_tile_early_key", 600, 8, 5),
     ("opening_tile_late_key", 600, 8, 120),
     ("last_full_tile_last_key", 640, 8, 639),
+    # a jump of about 2^367: 2^x overflows in the fast path, the factor of the rescale underflows to zero
+    ("extreme_jump_in_a_full_tile", 600, 8, 350),
+    ("extreme_jump_in_the_tree_tile", 40, 128, 40 + 100),
 ]
 
 
@@ -282,6 +285,8 @@ def test_reference_maximum_moving_inside_a_tile(name, S, N, big, d):
     case["k_tree"].zero_()
     case["q"].fill_(1.0)
     amp = 0.75 * (128 / d) ** 0.5                   # score = d * amp / sqrt(d); 12.24 in log2 units for both head dims
+    if name.startswith("extreme"):
+        amp *= 30.0
     if big < S:
         case["k_cache"][0, 0, 0, big] = amp
     else:
