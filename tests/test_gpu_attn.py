@@ -477,3 +477,39 @@ def test_layers_call_one_launch_many_layers_and_its_limits():
     assert launches3 == L and torch.equal(out3, out2) and torch.equal(lse3, lse2)
     with pytest.raises(tv.TreeVerifyError):                 # not even one layer of counters
         run(0, torch.zeros(need - 32 * per_layer, dtype=torch.uint8, device="cuda"))
+
+
+def test_layers_call_with_padded_layer_strides_is_bit_equal_to_the_dense_call():
+    """The layer strides are arguments of their own: tensors whose layers lie further apart than their size
+    (a view into a larger allocation) give the same bits as dense ones."""
+    L = 3
+    cfg = CONFIGS[0].scaled(B=3, L=L, S_lo=0, S_hi=500, Scap=512, N=40, Hq=8, Hkv=2, d=128, V=0)
+    case = to_device(make_case(cfg, seed=61, ragged_nodes=True, with_logits=False))
+    B, N, Hq, Hkv, d, Scap = cfg.B, cfg.N, cfg.Hq, cfg.Hkv, cfg.d, cfg.Scap
+    bits = torch.zeros(B, N, (N + 31) // 32, dtype=torch.int32, device="cuda")
+    st = torch.zeros(B, dtype=torch.int32, device="cuda")
+    tv.tree_build_mask(case["parent"], case["n_nodes"], N - 1, 1, bits, st)
+    ws = torch.zeros(tv.tv_attn_workspace_bytes(B, N, Hq, Hkv, d, Scap), dtype=torch.uint8, device="cuda")
+
+    def padded(t, pad):
+        per = t[0].numel()
+        big = torch.full((L * (per + pad),), 7.0, dtype=t.dtype, device=t.device)
+        v = torch.as_strided(big, t.shape, (per + pad,) + t[0].stride())
+        v.copy_(t)
+        return v
+
+    def run(q, kc, vc, kt, vt, out):
+        tv.tree_verify_attn_layers(q, kc, vc, kt, vt, case["prefix_len"], case["n_nodes"], bits, d ** -0.5, out, ws, st)
+        torch.cuda.synchronize()
+        assert (st.cpu().numpy() == 0).all()
+        return out
+
+    dense = run(case["q"], case["k_cache"], case["v_cache"], case["k_tree"], case["v_tree"],
+                torch.zeros(L, B, N, Hq, d, dtype=torch.bfloat16, device="cuda"))
+    out_p = padded(torch.zeros(L, B, N, Hq, d, dtype=torch.bfloat16, device="cuda"), 24)
+    got = run(padded(case["q"], 8), padded(case["k_cache"], 4096), padded(case["v_cache"], 4096), padded(case["k_tree"], 16),
+              padded(case["v_tree"], 16), out_p)
+    assert torch.equal(got, dense)
+    per = B * N * Hq * d                       # the gaps between the layers of the output were left alone
+    gaps = torch.as_strided(out_p, (L, 24), (per + 24, 1), per)
+    assert (gaps == 7.0).all()
